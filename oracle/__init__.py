@@ -1,0 +1,145 @@
+"""ctypes front end of the fp64 CPU oracle (``oracle/sbp_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+CPU-baseline leg of the benchmark.  It shares nothing with the CUDA library and
+never imports it.  ``build()`` compiles the C file with gcc; every wrapper only
+marshals numpy arrays, the arithmetic lives in the C file.
+
+Paper passages each wrapped function follows are cited in the C source.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sbp_oracle.c")
+_LIB_PATH = os.path.join(_HERE, "libsbp_oracle.so")
+
+MASK_RANDOM = 0
+MASK_GRID = 1
+FLAG_SHARE_MASK = 1
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle shared object beside its source (gcc -O2 -fopenmp)."""
+    if (not force and os.path.exists(_LIB_PATH)
+            and os.path.getmtime(_LIB_PATH) >= os.path.getmtime(_SRC)):
+        return _LIB_PATH
+    cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+           "-ffp-contract=off", "-o", _LIB_PATH, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    lib = ctypes.CDLL(_LIB_PATH)
+    i64, u64, u32, dbl, vp = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_uint32,
+                              ctypes.c_double, ctypes.c_void_p)
+    lib.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+    lib.oracle_philox4x32_10.restype = None
+    lib.oracle_keep_count.argtypes = [ctypes.c_int, i64, i64, dbl]
+    lib.oracle_keep_count.restype = i64
+    lib.oracle_sample_keep.argtypes = [ctypes.c_int, i64, i64, i64, dbl, u64, u64, i64, u32, vp, vp]
+    lib.oracle_sample_keep.restype = i64
+    lib.oracle_forward_cache.argtypes = [vp, i64, vp, i64, vp]
+    lib.oracle_forward_cache.restype = None
+    lib.oracle_linear_backward.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp]
+    lib.oracle_linear_backward.restype = None
+    lib.oracle_full_backward.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, vp]
+    lib.oracle_full_backward.restype = None
+    lib.oracle_num_threads.argtypes = []
+    lib.oracle_num_threads.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def philox4x32_10(counter, key):
+    """One Philox4x32-10 block: 4 counter words, 2 key words -> 4 output words."""
+    c = np.asarray(counter, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    assert c.shape == (4,) and k.shape == (2,)
+    out = np.zeros(4, dtype=np.uint32)
+    _load().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def keep_count(mode: int, H: int, W: int, keep_ratio: float) -> int:
+    return int(_load().oracle_keep_count(mode, H, W, float(keep_ratio)))
+
+
+def sample_keep(mode: int, B: int, H: int, W: int, keep_ratio: float, seed: int = 0,
+                step: int = 0, sample_offset: int = 0, flags: int = 0):
+    """Returns (keep_rows int32 [M_keep], keep_offsets int32 [B+1])."""
+    cap = keep_count(mode, H, W, keep_ratio)
+    if cap < 0:
+        raise ValueError("arguments outside the sampler's domain")
+    rows = np.zeros(max(B * cap, 1), dtype=np.int32)
+    offs = np.zeros(B + 1, dtype=np.int32)
+    n = _load().oracle_sample_keep(mode, B, H, W, float(keep_ratio), seed, step,
+                                   sample_offset, flags, _ptr(rows), _ptr(offs))
+    if n < 0:
+        raise ValueError("arguments outside the sampler's domain")
+    return rows[:n].copy(), offs
+
+
+def forward_cache(X: np.ndarray, keep_rows: np.ndarray) -> np.ndarray:
+    """Byte-exact gather of the kept rows of a 2-D array of any dtype."""
+    X = np.ascontiguousarray(X)
+    assert X.ndim == 2
+    rows = np.ascontiguousarray(keep_rows, dtype=np.int32)
+    out = np.empty((rows.shape[0], X.shape[1]), dtype=X.dtype)
+    _load().oracle_forward_cache(_ptr(X), X.shape[1] * X.dtype.itemsize, _ptr(rows),
+                                 rows.shape[0], _ptr(out))
+    return out
+
+
+def linear_backward(X_keep, dY, W, keep_rows, want=("dW", "db", "dX")):
+    """SBP backward of one linear layer in fp64.  Returns dict of requested outputs."""
+    X_keep, dY, W = _f64(X_keep), _f64(dY), _f64(W)
+    rows = np.ascontiguousarray(keep_rows, dtype=np.int32)
+    M, C_out = dY.shape
+    C_in = W.shape[0]
+    M_keep = rows.shape[0]
+    assert W.shape == (C_in, C_out) and X_keep.shape == (M_keep, C_in)
+    dW = np.empty((C_in, C_out)) if "dW" in want else None
+    db = np.empty(C_out) if "db" in want else None
+    dX = np.empty((M, C_in)) if "dX" in want else None
+    _load().oracle_linear_backward(_ptr(X_keep), _ptr(dY), _ptr(W), _ptr(rows), M_keep, M,
+                                   C_in, C_out, _ptr(dW), _ptr(db), _ptr(dX))
+    return {k: v for k, v in (("dW", dW), ("db", db), ("dX", dX)) if v is not None}
+
+
+def full_backward(X, dY, W, want=("dW", "db", "dX")):
+    """Full (no SBP) backward of the same layer in fp64."""
+    X, dY, W = _f64(X), _f64(dY), _f64(W)
+    M, C_out = dY.shape
+    C_in = W.shape[0]
+    assert X.shape == (M, C_in) and W.shape == (C_in, C_out)
+    dW = np.empty((C_in, C_out)) if "dW" in want else None
+    db = np.empty(C_out) if "db" in want else None
+    dX = np.empty((M, C_in)) if "dX" in want else None
+    _load().oracle_full_backward(_ptr(X), _ptr(dY), _ptr(W), M, C_in, C_out,
+                                 _ptr(dW), _ptr(db), _ptr(dX))
+    return {k: v for k, v in (("dW", dW), ("db", db), ("dX", dX)) if v is not None}

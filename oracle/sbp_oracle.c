@@ -1,0 +1,315 @@
+/*
+ * CPU oracle for the Stochastic Backpropagation (SBP) linear-layer hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the
+ * CUDA library is checked against; it shares no code with the CUDA path and is
+ * never on the product path.  Floating point is fp64 throughout; the index
+ * work is exact integer arithmetic.
+ *
+ * What each function follows (paper: "An In-depth Study of Stochastic
+ * Backpropagation", arXiv 2210.00129):
+ *   - keep / drop index sets and the keep ratio r:      Sec. 3.2.1 (text after Eq. 3)
+ *   - random and grid-wise mask sampling:               Sec. 4 ("How to sample the
+ *                                                       gradient keep mask?"), Supp. A.4
+ *   - forward cache of the kept rows:                   Algorithm 1, Sec. 3.1
+ *   - dW, dX of a linear / point-wise layer under SBP:  Eq. 5 and the text after it
+ *   - full backward for the invariants:                 Eq. 3
+ *   - no gradient rescaling:                            Eq. 1
+ * The paper names no random generator; the sampler uses Philox4x32-10
+ * (Salmon, Moraes, Dror, Shaw: "Parallel Random Numbers: As Easy as 1, 2, 3",
+ * SC'11), written here from that paper's definition of the round function.
+ *
+ * Parity pins: every function here is pinned by tests that do not call it to
+ * check itself (published Philox known answers, brute-force selection, hand
+ * computed integer cases, reduction to library matrix products, enumeration
+ * of all masks).  Nothing in this file is "parity unpinned".
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_MASK_RANDOM 0
+#define ORACLE_MASK_GRID   1
+#define ORACLE_FLAG_SHARE_MASK 1u
+
+/* ------------------------------------------------------------------ */
+/* Philox4x32-10 (SC'11, Sec. 3.3 and Table 2 of that paper)            */
+/* ------------------------------------------------------------------ */
+
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint64_t MUL_A = 0xD2511F53u;   /* multiplier applied to word 0 */
+    const uint64_t MUL_B = 0xCD9E8D57u;   /* multiplier applied to word 2 */
+    const uint32_t WEYL_0 = 0x9E3779B9u;  /* key schedule increments */
+    const uint32_t WEYL_1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) { k0 += WEYL_0; k1 += WEYL_1; }
+        uint64_t pa = MUL_A * (uint64_t)c0;
+        uint64_t pb = MUL_B * (uint64_t)c2;
+        uint32_t hi_a = (uint32_t)(pa >> 32), lo_a = (uint32_t)pa;
+        uint32_t hi_b = (uint32_t)(pb >> 32), lo_b = (uint32_t)pb;
+        uint32_t n0 = hi_b ^ c1 ^ k0;
+        uint32_t n1 = lo_b;
+        uint32_t n2 = hi_a ^ c3 ^ k1;
+        uint32_t n3 = lo_a;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The 32-bit random word attached to position n of global sample gid.
+ * Counter layout: word0 = n / 4, word1 = global sample id, word2 = step,
+ * word3 = stream tag (0 = random-mask keys, 1 = grid phase); key = seed.
+ * Position n takes output word n mod 4. */
+static uint32_t position_word(uint64_t seed, uint32_t step, uint32_t gid, uint32_t n)
+{
+    uint32_t ctr[4] = { n >> 2, gid, step, 0u };
+    uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    return out[n & 3u];
+}
+
+static uint32_t grid_phase_word(uint64_t seed, uint32_t step, uint32_t gid)
+{
+    uint32_t ctr[4] = { 0u, gid, step, 1u };
+    uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    return out[0];
+}
+
+/* ------------------------------------------------------------------ */
+/* keep ratio -> number of kept positions (Sec. 3.2.1: r = #kept / #all) */
+/* ------------------------------------------------------------------ */
+
+/* which member of the 2x2 grid family a ratio selects; 0 when none */
+static int grid_family(double r)
+{
+    if (r == 0.25) return 1;
+    if (r == 0.5)  return 2;
+    if (r == 0.75) return 3;
+    if (r == 1.0)  return 4;
+    return 0;
+}
+
+/* is (h, w) kept by grid family member fam at phase p ? */
+static int grid_keeps(int fam, uint32_t p, int64_t h, int64_t w)
+{
+    switch (fam) {
+    case 1: return ((h & 1) == (int64_t)(p >> 1)) && ((w & 1) == (int64_t)(p & 1));
+    case 2: return (((h + w) & 1) == (int64_t)p);
+    case 3: return !(((h & 1) == (int64_t)(p >> 1)) && ((w & 1) == (int64_t)(p & 1)));
+    case 4: return 1;
+    }
+    return 0;
+}
+
+/* Random mode: the exact per-sample count K = clamp(floor(r*N + 1/2), 1, N).
+ * Grid mode: the largest count any phase can give (capacity per sample).
+ * Returns -1 for arguments outside the method's domain. */
+int64_t oracle_keep_count(int mode, int64_t H, int64_t W, double r)
+{
+    if (H <= 0 || W <= 0 || !(r > 0.0) || !(r <= 1.0)) return -1;
+    int64_t N = H * W;
+    if (mode == ORACLE_MASK_RANDOM) {
+        int64_t K = (int64_t)floor(r * (double)N + 0.5);
+        if (K < 1) K = 1;
+        if (K > N) K = N;
+        return K;
+    }
+    if (mode == ORACLE_MASK_GRID) {
+        int fam = grid_family(r);
+        if (!fam) return -1;
+        int phases = (fam == 2) ? 2 : (fam == 4 ? 1 : 4);
+        int64_t best = 0;
+        for (int p = 0; p < phases; ++p) {
+            int64_t cnt = 0;
+            for (int64_t h = 0; h < H; ++h)
+                for (int64_t w = 0; w < W; ++w)
+                    cnt += grid_keeps(fam, (uint32_t)p, h, w);
+            if (cnt > best) best = cnt;
+        }
+        return best;
+    }
+    return -1;
+}
+
+/* ------------------------------------------------------------------ */
+/* keep-index sampling (Sec. 4; Supp. A.4: one fresh mask per step)     */
+/* ------------------------------------------------------------------ */
+
+static int cmp_u64(const void* a, const void* b)
+{
+    uint64_t x = *(const uint64_t*)a, y = *(const uint64_t*)b;
+    return (x > y) - (x < y);
+}
+
+/* Writes the global row ids b*N + n of the kept positions, ascending, and the
+ * per-sample prefix keep_offsets[0..B].  Returns M_keep, or -1 on bad input.
+ * Random mode: every position gets the 64-bit score (word << 32) | n; the K
+ * positions with the smallest scores are kept (all K-subsets equally likely).
+ * Grid mode: a periodic 2x2 lattice whose phase is drawn per sample. */
+int64_t oracle_sample_keep(int mode, int64_t B, int64_t H, int64_t W, double r,
+                           uint64_t seed, uint64_t step, int64_t sample_offset,
+                           uint32_t flags, int32_t* keep_rows, int32_t* keep_offsets)
+{
+    if (B <= 0 || H <= 0 || W <= 0) return -1;
+    int64_t N = H * W;
+    if (oracle_keep_count(mode, H, W, r) < 0) return -1;
+    if (step >> 32) return -1;
+    if (sample_offset < 0 || ((uint64_t)(sample_offset + B - 1) >> 32)) return -1;
+    if (B * N >= ((int64_t)1 << 31)) return -1;
+
+    int64_t out = 0;
+    keep_offsets[0] = 0;
+    if (mode == ORACLE_MASK_RANDOM) {
+        int64_t K = oracle_keep_count(mode, H, W, r);
+        uint64_t* score = (uint64_t*)malloc((size_t)N * sizeof(uint64_t));
+        unsigned char* kept = (unsigned char*)malloc((size_t)N);
+        for (int64_t b = 0; b < B; ++b) {
+            uint32_t gid = (flags & ORACLE_FLAG_SHARE_MASK) ? 0u : (uint32_t)(sample_offset + b);
+            for (int64_t n = 0; n < N; ++n) {
+                uint64_t u = position_word(seed, (uint32_t)step, gid, (uint32_t)n);
+                score[n] = (u << 32) | (uint64_t)n;
+            }
+            qsort(score, (size_t)N, sizeof(uint64_t), cmp_u64);
+            memset(kept, 0, (size_t)N);
+            for (int64_t k = 0; k < K; ++k) kept[score[k] & 0xffffffffu] = 1;
+            for (int64_t n = 0; n < N; ++n)
+                if (kept[n]) keep_rows[out++] = (int32_t)(b * N + n);
+            keep_offsets[b + 1] = (int32_t)out;
+        }
+        free(score); free(kept);
+    } else {
+        int fam = grid_family(r);
+        uint32_t phases = (fam == 2) ? 2u : (fam == 4 ? 1u : 4u);
+        for (int64_t b = 0; b < B; ++b) {
+            uint32_t gid = (flags & ORACLE_FLAG_SHARE_MASK) ? 0u : (uint32_t)(sample_offset + b);
+            uint32_t p = grid_phase_word(seed, (uint32_t)step, gid) % phases;
+            for (int64_t h = 0; h < H; ++h)
+                for (int64_t w = 0; w < W; ++w)
+                    if (grid_keeps(fam, p, h, w)) keep_rows[out++] = (int32_t)(b * N + h * W + w);
+            keep_offsets[b + 1] = (int32_t)out;
+        }
+    }
+    return out;
+}
+
+/* ------------------------------------------------------------------ */
+/* forward cache (Algorithm 1: only inputs[keep] is retained)           */
+/* ------------------------------------------------------------------ */
+
+/* Byte-exact row gather: X_keep[m, :] = X[keep_rows[m], :], rows of row_bytes. */
+void oracle_forward_cache(const void* X, int64_t row_bytes, const int32_t* keep_rows,
+                          int64_t M_keep, void* X_keep)
+{
+    for (int64_t m = 0; m < M_keep; ++m)
+        memcpy((char*)X_keep + m * row_bytes,
+               (const char*)X + (int64_t)keep_rows[m] * row_bytes, (size_t)row_bytes);
+}
+
+/* ------------------------------------------------------------------ */
+/* SBP backward of a linear layer (Eq. 5; bias gradient by the same     */
+/* masking of dY; nothing is rescaled, Eq. 1)                           */
+/* ------------------------------------------------------------------ */
+
+/* X_keep [M_keep, C_in], dY [M, C_out] (full; only kept rows are read),
+ * W [C_in, C_out] row-major (Y = X W), keep_rows ascending global row ids.
+ *   dW[i, j] = sum_m X_keep[m, i] * dY[keep_rows[m], j]
+ *   db[j]    = sum_m dY[keep_rows[m], j]
+ *   dX[keep_rows[m], i] = sum_j dY[keep_rows[m], j] * W[i, j];  other rows +0.0
+ * Any of dW, db, dX may be NULL.  Sums run over m (resp. j) in ascending order. */
+void oracle_linear_backward(const double* X_keep, const double* dY, const double* W,
+                            const int32_t* keep_rows, int64_t M_keep, int64_t M,
+                            int64_t C_in, int64_t C_out,
+                            double* dW, double* db, double* dX)
+{
+    if (dW) {
+        #pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < C_in; ++i) {
+            double* dWi = dW + i * C_out;
+            for (int64_t j = 0; j < C_out; ++j) dWi[j] = 0.0;
+            for (int64_t m = 0; m < M_keep; ++m) {
+                double x = X_keep[m * C_in + i];
+                const double* g = dY + (int64_t)keep_rows[m] * C_out;
+                for (int64_t j = 0; j < C_out; ++j) dWi[j] += x * g[j];
+            }
+        }
+    }
+    if (db) {
+        for (int64_t j = 0; j < C_out; ++j) db[j] = 0.0;
+        for (int64_t m = 0; m < M_keep; ++m) {
+            const double* g = dY + (int64_t)keep_rows[m] * C_out;
+            for (int64_t j = 0; j < C_out; ++j) db[j] += g[j];
+        }
+    }
+    if (dX) {
+        #pragma omp parallel for schedule(static)
+        for (int64_t t = 0; t < M * C_in; ++t) dX[t] = 0.0;
+        #pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M_keep; ++m) {
+            const double* g = dY + (int64_t)keep_rows[m] * C_out;
+            double* o = dX + (int64_t)keep_rows[m] * C_in;
+            for (int64_t i = 0; i < C_in; ++i) {
+                const double* w = W + i * C_out;
+                double acc = 0.0;
+                for (int64_t j = 0; j < C_out; ++j) acc += g[j] * w[j];
+                o[i] = acc;
+            }
+        }
+    }
+}
+
+/* Full backward of the same layer (Eq. 3): dW = X^T dY, db = column sums of
+ * dY, dX = dY W^T, over all M rows. */
+void oracle_full_backward(const double* X, const double* dY, const double* W,
+                          int64_t M, int64_t C_in, int64_t C_out,
+                          double* dW, double* db, double* dX)
+{
+    if (dW) {
+        #pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < C_in; ++i) {
+            double* dWi = dW + i * C_out;
+            for (int64_t j = 0; j < C_out; ++j) dWi[j] = 0.0;
+            for (int64_t m = 0; m < M; ++m) {
+                double x = X[m * C_in + i];
+                const double* g = dY + m * C_out;
+                for (int64_t j = 0; j < C_out; ++j) dWi[j] += x * g[j];
+            }
+        }
+    }
+    if (db) {
+        for (int64_t j = 0; j < C_out; ++j) db[j] = 0.0;
+        for (int64_t m = 0; m < M; ++m)
+            for (int64_t j = 0; j < C_out; ++j) db[j] += dY[m * C_out + j];
+    }
+    if (dX) {
+        #pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            const double* g = dY + m * C_out;
+            for (int64_t i = 0; i < C_in; ++i) {
+                const double* w = W + i * C_out;
+                double acc = 0.0;
+                for (int64_t j = 0; j < C_out; ++j) acc += g[j] * w[j];
+                dX[m * C_in + i] = acc;
+            }
+        }
+    }
+}
+
+/* threads the row loops above will use */
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
