@@ -1,0 +1,169 @@
+/*
+ * sbp.h - C ABI of the B200 (sm_100a) Stochastic Backpropagation linear-layer library.
+ *
+ * Stochastic Backpropagation (SBP; "An In-depth Study of Stochastic
+ * Backpropagation", arXiv 2210.00129) runs the forward pass of a linear /
+ * point-wise layer on every spatial position but caches, and back-propagates
+ * through, only a randomly kept subset of positions.  This library is the hot
+ * path of that method for one layer Y = X W:
+ *
+ *   sbp_sample_keep      draw the kept positions of every sample      (Sec. 3.2.1, Sec. 4)
+ *   sbp_forward_cache    X_keep = X[keep_rows, :]                     (Algorithm 1)
+ *   sbp_linear_backward  dW = X_keep^T dY_keep, db = sum dY_keep,
+ *                        dX = scatter(dY_keep W^T), zeros elsewhere   (Eq. 5)
+ *
+ * Nothing is rescaled by 1/r: Eq. 1 keeps the plain 1/B factor.
+ *
+ * Conventions
+ *   - M = B*N rows, N = H*W positions per sample, row id = b*N + h*W + w.
+ *   - All matrices are row-major, dense (no padding), inner stride 1.
+ *     W is [C_in, C_out] (the paper's orientation, Y = X W).
+ *   - "dev" pointers are CUDA device pointers owned by the caller; the library
+ *     allocates and frees nothing and keeps no pointer after a call returns.
+ *     Device buffers must be 16-byte aligned.
+ *   - Calls enqueue work on the caller's stream (a cudaStream_t passed as
+ *     void*, NULL = default stream) and return without synchronising.
+ *   - Errors detectable on the host are returned before anything is launched.
+ *     Conditions only the device can see (bad indices under SBP_FLAG_VALIDATE,
+ *     a bounded wait that ran out) are written to the optional status word.
+ *   - No call throws; every call returns an sbp_status.
+ */
+#ifndef SBP_H_
+#define SBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SBP_OK = 0,
+    SBP_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, size or ratio out of range */
+    SBP_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for */
+    SBP_ERR_WORKSPACE = 3,     /* workspace missing or too small */
+    SBP_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
+    SBP_ERR_TIMEOUT = 5,       /* device status word: a bounded wait inside a kernel expired */
+    SBP_ERR_BAD_INDICES = 6    /* device status word: keep_rows not ascending / out of range */
+} sbp_status;
+
+typedef enum { SBP_F32 = 0, SBP_BF16 = 1 } sbp_dtype;
+
+/* Sec. 4, "How to sample the gradient keep mask?": uniformly random positions,
+ * or a structured periodic ("grid-wise") mask. */
+typedef enum { SBP_MASK_RANDOM = 0, SBP_MASK_GRID = 1 } sbp_mask_mode;
+
+enum {
+    SBP_FLAG_SHARE_MASK = 1,  /* every sample of the call uses sample 0's mask (one mask per iteration, Supp. A.4) */
+    SBP_FLAG_ACCUMULATE = 2,  /* dW += and db += instead of overwrite (gradient accumulation) */
+    SBP_FLAG_VALIDATE = 4,    /* check keep_rows on the device before use; result in the status word */
+    SBP_FLAG_PLAIN_FMA = 8    /* bf16 only: use the CUDA-core FMA kernels instead of the tensor-core ones */
+};
+
+const char* sbp_status_string(sbp_status s);
+
+/*
+ * Kept positions per sample for keep ratio r = #kept / #all (Sec. 3.2.1).
+ * Pure host function.
+ *   SBP_MASK_RANDOM: the exact count K = clamp(floor(r*H*W + 1/2), 1, H*W).
+ *   SBP_MASK_GRID:   the largest count any phase of the mask gives (buffer capacity
+ *                    per sample); r must be one of 0.25, 0.5, 0.75, 1.0.
+ * Returns -1 when H, W <= 0, r outside (0, 1], or the ratio has no grid mask.
+ */
+int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_ratio);
+
+/*
+ * Draw the keep set of each of B samples (Sec. 3.2.1 index sets; Sec. 4 masks;
+ * Supp. A.4: a fresh mask every training step).
+ *
+ * SBP_MASK_RANDOM: position n of global sample g = sample_offset + b gets the
+ *   32-bit word u = Philox4x32-10(counter = {n/4, g, step, 0}, key = seed)[n mod 4];
+ *   the K positions with the smallest 64-bit scores (u << 32 | n) are kept, so
+ *   every K-subset is equally likely.  Pass H = N, W = 1 for unstructured rows.
+ * SBP_MASK_GRID: a 2x2-periodic lattice with a random phase p per sample,
+ *   p = Philox4x32-10({0, g, step, 1}, seed)[0] mod (#phases):
+ *     r = 0.25  keep (h mod 2, w mod 2) == (p / 2, p mod 2)      (4 phases)
+ *     r = 0.5   keep (h + w) mod 2 == p                           (2 phases)
+ *     r = 0.75  complement of the r = 0.25 mask                   (4 phases)
+ *     r = 1.0   keep everything
+ * The mask depends only on (seed, step, g, n): it does not change with how a
+ * batch is split over calls or devices.
+ *
+ * Outputs (dev): keep_rows, capacity B * sbp_keep_count(...), receives the global
+ * row ids b*N + n of kept positions in ascending order (entries past the total
+ * are left untouched); keep_offsets[B + 1] receives the per-sample prefix,
+ * keep_offsets[B] = M_keep.
+ *
+ * Errors: SBP_ERR_INVALID_ARG for null/misaligned outputs, B, H, W <= 0,
+ * B*H*W >= 2^31, r outside (0, 1], step >= 2^32, sample ids >= 2^32 or < 0;
+ * SBP_ERR_UNSUPPORTED for a grid ratio outside the four above;
+ * SBP_ERR_CUDA if the launch fails.
+ */
+sbp_status sbp_sample_keep(sbp_mask_mode mode, int64_t B, int64_t H, int64_t W,
+                           double keep_ratio, uint64_t seed, uint64_t step,
+                           int64_t sample_offset, uint32_t flags,
+                           int32_t* keep_rows /* dev */, int32_t* keep_offsets /* dev */,
+                           void* stream);
+
+/*
+ * Forward cache (Algorithm 1: only inputs[keep] is retained for backward):
+ *   X_keep[m, :] = X[keep_rows[m], :]   for m < M_keep, a bit-exact copy.
+ * X is [M, C]; X_keep is [M_keep_cap, C]; rows M_keep <= m < M_keep_cap are set
+ * to zero (sbp_linear_backward relies on those padding rows being finite).
+ * M_keep is *M_keep_dev when that device pointer is non-NULL (e.g. &keep_offsets[B]),
+ * else M_keep_cap.  Dropped rows of X are never read.
+ * Requires C * sizeof(element) to be a multiple of 16 (else SBP_ERR_UNSUPPORTED).
+ * keep_rows entries must lie in [0, M); they are not checked here.
+ */
+sbp_status sbp_forward_cache(sbp_dtype dt, const void* X /* dev */, int64_t M, int64_t C,
+                             const int32_t* keep_rows /* dev */,
+                             const int32_t* M_keep_dev /* dev, nullable */,
+                             int64_t M_keep_cap, void* X_keep /* dev */, void* stream);
+
+/* Scratch bytes sbp_linear_backward needs for these sizes (never 0). */
+size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap,
+                                           int64_t C_in, int64_t C_out);
+
+/*
+ * SBP backward of one linear layer (Eq. 5 and the text after it; bias gradient
+ * by the same masking of dY; no rescaling, Eq. 1):
+ *   dW[i, j]            = sum_{m < M_keep} X_keep[m, i] * dY[keep_rows[m], j]     fp32 [C_in, C_out]
+ *   db[j]               = sum_{m < M_keep} dY[keep_rows[m], j]                    fp32 [C_out]
+ *   dX[keep_rows[m], :] = dY[keep_rows[m], :] * W^T                                dt   [M, C_in]
+ *   every other row of dX = +0.0
+ * Inputs: X_keep [M_keep_cap, C_in] (from sbp_forward_cache; rows past M_keep must
+ * be finite), dY [M, C_out] (the full upstream gradient; only kept rows are read),
+ * W [C_in, C_out], keep_rows strictly ascending ids in [0, M).  M_keep is
+ * *M_keep_dev if non-NULL, else M_keep_cap.  Any of dW, db, dX may be NULL to skip
+ * that product.
+ *
+ * SBP_BF16: inputs bf16, products accumulated in fp32 on the tensor cores, dX
+ * rounded to bf16 (nearest even).  SBP_F32: plain fp32 FMA arithmetic.
+ * C_in and C_out must be multiples of 8 (bf16) / 4 (fp32), else SBP_ERR_UNSUPPORTED.
+ *
+ * flags: SBP_FLAG_ACCUMULATE adds into dW and db; SBP_FLAG_VALIDATE first checks
+ * keep_rows on the device and, on failure, writes SBP_ERR_BAD_INDICES to
+ * *status_word and makes the compute kernels return without touching outputs
+ * (needs a status word); SBP_FLAG_PLAIN_FMA forces the CUDA-core kernels.
+ * workspace: at least sbp_linear_backward_workspace_bytes(...) bytes, 256-byte
+ * aligned, used only during the call's kernels (SBP_ERR_WORKSPACE if short).
+ * status_word (dev, nullable): must be zero before the call; receives the first
+ * device-side error (SBP_ERR_TIMEOUT, SBP_ERR_BAD_INDICES), else stays zero.
+ * Results are deterministic: no floating-point atomics are used.
+ */
+sbp_status sbp_linear_backward(sbp_dtype dt,
+                               const void* X_keep /* dev */, const void* dY /* dev */,
+                               const void* W /* dev */,
+                               const int32_t* keep_rows /* dev */,
+                               const int32_t* M_keep_dev /* dev, nullable */,
+                               int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
+                               float* dW /* dev, nullable */, float* db /* dev, nullable */,
+                               void* dX /* dev, nullable */,
+                               uint32_t flags, void* workspace /* dev */, size_t workspace_bytes,
+                               int32_t* status_word /* dev, nullable */, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SBP_H_ */
