@@ -1,0 +1,244 @@
+// Keep-index sampler (Sec. 3.2.1 index sets; Sec. 4 random and grid-wise masks).
+//
+// One thread block per sample.  Random mode finds the K-th smallest 64-bit score
+// (philox word << 32 | position) with a four-pass, 8-bit radix select over the philox words -
+// which are recomputed on every pass, never stored - and then emits the kept positions in
+// ascending order with a block-wide prefix sum.  Grid mode evaluates the lattice predicate and
+// uses the same ordered compaction; per-sample offsets come from closed-form counts.
+#include "sbp_common.cuh"
+
+namespace sbp {
+namespace {
+
+constexpr int kSampThreads = 512;
+constexpr int kSampWarps = kSampThreads / 32;
+
+struct SampShared {
+    uint32_t hist[256];
+    uint32_t warp_sums_a[kSampWarps];
+    uint32_t warp_sums_b[kSampWarps];
+    uint32_t sel_digit;
+    uint32_t sel_below;
+    uint64_t red64[kSampWarps];
+};
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t n = __shfl_up_sync(0xffffffffu, v, d);
+        if (lane >= d) v += n;
+    }
+    return v;
+}
+
+// Exclusive prefix over the block of per-thread counts; returns (exclusive prefix, block total).
+__device__ __forceinline__ uint2 block_excl_scan(uint32_t v, uint32_t* warp_sums) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t incl = warp_incl_scan(v, lane);
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    uint32_t ws = (lane < kSampWarps) ? warp_sums[lane] : 0u;
+    const uint32_t ws_incl = warp_incl_scan(ws, lane);
+    const uint32_t total = __shfl_sync(0xffffffffu, ws_incl, kSampWarps - 1);
+    const uint32_t warp_base = __shfl_sync(0xffffffffu, ws_incl - ws, warp);
+    __syncthreads();
+    return make_uint2(warp_base + incl - v, total);
+}
+
+// words of the four positions 4q .. 4q+3 of sample gid
+__device__ __forceinline__ PhiloxWords position_words(uint32_t q, uint32_t gid, uint32_t step,
+                                                      uint32_t k0, uint32_t k1) {
+    return philox4x32_10(q, gid, step, 0u, k0, k1);
+}
+
+__global__ void __launch_bounds__(kSampThreads)
+sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint32_t step,
+                          uint32_t first_sample, int share_mask,
+                          int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
+    __shared__ SampShared sh;
+    const uint32_t b = blockIdx.x;
+    const uint32_t gid = share_mask ? 0u : first_sample + b;
+    const uint32_t groups = (N + 3u) >> 2;
+    const int64_t row_base = (int64_t)b * N;
+    int32_t* out = keep_rows + (int64_t)b * K;
+    if (threadIdx.x == 0) {
+        keep_offsets[b + 1] = (int32_t)((b + 1) * (int64_t)K);
+        if (b == 0) keep_offsets[0] = 0;
+    }
+
+    // ---- radix select: threshold word `prefix` and how many positions equal to it are kept ----
+    uint32_t prefix = 0, known = 0, remaining = K;
+    if (K < N) {
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int i = threadIdx.x; i < 256; i += kSampThreads) sh.hist[i] = 0;
+            __syncthreads();
+            for (uint32_t q = threadIdx.x; q < groups; q += kSampThreads) {
+                const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t n = 4u * q + e;
+                    if (n < N && (pw.w[e] & known) == prefix) atomicAdd(&sh.hist[(pw.w[e] >> shift) & 0xffu], 1u);
+                }
+            }
+            __syncthreads();
+            // exclusive scan over the 256 bins; the bin where the running count crosses `remaining` wins
+            const uint32_t cnt = (threadIdx.x < 256) ? sh.hist[threadIdx.x] : 0u;
+            const uint2 sc = block_excl_scan(cnt, sh.warp_sums_a);
+            if (threadIdx.x < 256 && sc.x < remaining && remaining <= sc.x + cnt) {
+                sh.sel_digit = threadIdx.x;
+                sh.sel_below = sc.x;
+            }
+            __syncthreads();
+            prefix |= sh.sel_digit << shift;
+            known |= 0xffu << shift;
+            remaining -= sh.sel_below;
+            __syncthreads();
+        }
+    }
+    const bool keep_all = (K >= N);
+    const uint32_t threshold = prefix;       // kept: word < threshold, plus the first `remaining` equal to it
+
+    // ---- ordered compaction, kSampThreads*4 positions per sweep ----
+    uint32_t eq_seen = 0, written = 0;
+    for (uint32_t q0 = 0; q0 < groups; q0 += kSampThreads) {
+        const uint32_t q = q0 + threadIdx.x;
+        uint32_t lt_mask = 0, eq_mask = 0;
+        if (q < groups) {
+            if (keep_all) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) if (4u * q + e < N) lt_mask |= 1u << e;
+            } else {
+                const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (4u * q + e < N) {
+                        if (pw.w[e] < threshold) lt_mask |= 1u << e;
+                        else if (pw.w[e] == threshold) eq_mask |= 1u << e;
+                    }
+                }
+            }
+        }
+        uint32_t keep_mask = lt_mask;
+        if (!keep_all) {
+            const uint2 se = block_excl_scan(__popc(eq_mask), sh.warp_sums_a);
+            uint32_t rank = eq_seen + se.x;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (eq_mask & (1u << e)) {
+                    if (rank < remaining) keep_mask |= 1u << e;
+                    ++rank;
+                }
+            }
+            eq_seen += se.y;
+        }
+        const uint2 sk = block_excl_scan(__popc(keep_mask), sh.warp_sums_b);
+        uint32_t pos = written + sk.x;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (keep_mask & (1u << e)) out[pos++] = (int32_t)(row_base + 4u * q + e);
+        }
+        written += sk.y;
+    }
+}
+
+// ---- grid-wise masks: 2x2-periodic lattice with a per-sample phase ----
+__device__ __forceinline__ uint32_t grid_phase(int family, uint32_t gid, uint32_t step, uint32_t k0, uint32_t k1) {
+    if (family == 4) return 0u;
+    const uint32_t word = philox4x32_10(0u, gid, step, 1u, k0, k1).w[0];
+    return family == 2 ? (word & 1u) : (word & 3u);
+}
+
+__device__ __forceinline__ uint32_t grid_count(int family, uint32_t p, uint32_t H, uint32_t W) {
+    const uint32_t quarter = ((H + 1u - (p >> 1)) >> 1) * ((W + 1u - (p & 1u)) >> 1);
+    switch (family) {
+        case 1: return quarter;
+        case 2: return (H * W + 1u - p) >> 1;
+        case 3: return H * W - quarter;
+        default: return H * W;
+    }
+}
+
+__device__ __forceinline__ bool grid_keeps(int family, uint32_t p, uint32_t h, uint32_t w) {
+    const bool on_lattice = ((h & 1u) == (p >> 1)) && ((w & 1u) == (p & 1u));
+    switch (family) {
+        case 1: return on_lattice;
+        case 2: return ((h + w) & 1u) == p;
+        case 3: return !on_lattice;
+        default: return true;
+    }
+}
+
+__global__ void __launch_bounds__(kSampThreads)
+sample_keep_grid_kernel(int family, uint32_t H, uint32_t W, uint32_t k0, uint32_t k1, uint32_t step,
+                        uint32_t first_sample, int share_mask,
+                        int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
+    __shared__ SampShared sh;
+    const uint32_t b = blockIdx.x;
+    const uint32_t N = H * W;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    // offset of this sample = sum of the closed-form counts of the samples before it
+    uint64_t before = 0;
+    if (share_mask) {
+        before = (uint64_t)b * grid_count(family, grid_phase(family, 0u, step, k0, k1), H, W);
+    } else {
+        uint64_t part = 0;
+        for (uint32_t s = threadIdx.x; s < b; s += kSampThreads)
+            part += grid_count(family, grid_phase(family, first_sample + s, step, k0, k1), H, W);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+        if (lane == 0) sh.red64[warp] = part;
+        __syncthreads();
+        for (int i = 0; i < kSampWarps; ++i) before += sh.red64[i];
+        __syncthreads();
+    }
+    const uint32_t gid = share_mask ? 0u : first_sample + b;
+    const uint32_t p = grid_phase(family, gid, step, k0, k1);
+    const uint32_t mine = grid_count(family, p, H, W);
+    if (threadIdx.x == 0) {
+        keep_offsets[b + 1] = (int32_t)(before + mine);
+        if (b == 0) keep_offsets[0] = 0;
+    }
+    int32_t* out = keep_rows + before;
+    const int64_t row_base = (int64_t)b * N;
+    const uint32_t groups = (N + 3u) >> 2;
+    uint32_t written = 0;
+    for (uint32_t q0 = 0; q0 < groups; q0 += kSampThreads) {
+        const uint32_t q = q0 + threadIdx.x;
+        uint32_t keep_mask = 0;
+        if (q < groups) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t n = 4u * q + e;
+                if (n < N && grid_keeps(family, p, n / W, n % W)) keep_mask |= 1u << e;
+            }
+        }
+        const uint2 sk = block_excl_scan(__popc(keep_mask), sh.warp_sums_b);
+        uint32_t pos = written + sk.x;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (keep_mask & (1u << e)) out[pos++] = (int32_t)(row_base + 4u * q + e);
+        written += sk.y;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, int64_t W, int64_t K,
+                               uint64_t seed, uint32_t step, uint32_t first_sample, bool share_mask,
+                               int32_t* keep_rows, int32_t* keep_offsets, cudaStream_t stream) {
+    const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
+    const dim3 grid((unsigned)B), block(kSampThreads);
+    if (mode == SBP_MASK_RANDOM) {
+        sample_keep_random_kernel<<<grid, block, 0, stream>>>((uint32_t)(H * W), (uint32_t)K, k0, k1, step,
+                                                              first_sample, share_mask ? 1 : 0,
+                                                              keep_rows, keep_offsets);
+    } else {
+        sample_keep_grid_kernel<<<grid, block, 0, stream>>>(grid_family, (uint32_t)H, (uint32_t)W, k0, k1, step,
+                                                            first_sample, share_mask ? 1 : 0,
+                                                            keep_rows, keep_offsets);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace sbp

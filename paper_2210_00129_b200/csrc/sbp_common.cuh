@@ -1,0 +1,99 @@
+// Shared device/host helpers of the SBP library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/sbp.h"
+
+namespace sbp {
+
+constexpr int kNumSMs = 148;            // B200: 2 dies x 74 SMs; grids are sized in multiples of this
+
+// Status codes are shared with the C header; device code writes them to the caller's status word.
+__device__ __forceinline__ void report_device_error(int32_t* status_word, int32_t code) {
+    if (status_word != nullptr) atomicCAS(status_word, 0, code);
+}
+
+// Number of valid kept rows: the device-side count when given, else the host capacity.
+__device__ __forceinline__ int64_t load_m_keep(const int32_t* M_keep_dev, int64_t M_keep_cap) {
+    if (M_keep_dev == nullptr) return M_keep_cap;
+    int64_t v = (int64_t)__ldg(M_keep_dev);
+    if (v < 0) v = 0;
+    return v < M_keep_cap ? v : M_keep_cap;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies with a Weyl key
+// schedule.  Device-side implementation used by the keep-index sampler.
+// ---------------------------------------------------------------------------------------------
+struct PhiloxWords { uint32_t w[4]; };
+
+__device__ __forceinline__ PhiloxWords philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                     uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t lo0 = 0xD2511F53u * c0;
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0);
+        const uint32_t lo1 = 0xCD9E8D57u * c2;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2);
+        const uint32_t t0 = hi1 ^ c1 ^ k0;
+        const uint32_t t2 = hi0 ^ c3 ^ k1;
+        c0 = t0; c1 = lo1; c2 = t2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    PhiloxWords out;
+    out.w[0] = c0; out.w[1] = c1; out.w[2] = c2; out.w[3] = c3;
+    return out;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Launch entry points of the individual kernels (defined in their own .cu files).
+// None synchronises.
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, int64_t W, int64_t K,
+                               uint64_t seed, uint32_t step, uint32_t first_sample, bool share_mask,
+                               int32_t* keep_rows, int32_t* keep_offsets, cudaStream_t stream);
+
+cudaError_t launch_gather_rows(const void* X, int64_t row_bytes, const int32_t* keep_rows,
+                               const int32_t* M_keep_dev, int64_t M_keep_cap, void* X_keep,
+                               cudaStream_t stream);
+
+cudaError_t launch_validate_keep_rows(const int32_t* keep_rows, const int32_t* M_keep_dev,
+                                      int64_t M_keep_cap, int64_t M, int32_t* status_word,
+                                      cudaStream_t stream);
+
+// partial column sums of the kept rows of dY -> db (deterministic two-pass reduction)
+size_t db_workspace_bytes(int64_t M_keep_cap, int64_t C_out);
+cudaError_t launch_db(sbp_dtype dt, const void* dY, const int32_t* keep_rows, const int32_t* M_keep_dev,
+                      int64_t M_keep_cap, int64_t C_out, float* db, bool accumulate, float* workspace,
+                      const int32_t* status_word, cudaStream_t stream);
+
+// out[i] = (accumulate ? out[i] : 0) + sum_s partials[s*n + i], summed in ascending s
+cudaError_t launch_reduce_partials(const float* partials, int splits, int64_t n, float* out,
+                                   bool accumulate, const int32_t* status_word, cudaStream_t stream);
+
+// plain-FMA (CUDA-core) products for fp32 and for bf16 shapes the tensor-core kernels do not take
+size_t simt_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+cudaError_t launch_simt_dw(sbp_dtype dt, const void* X_keep, const void* dY, const int32_t* keep_rows,
+                           const int32_t* M_keep_dev, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
+                           float* dW, bool accumulate, float* workspace, const int32_t* status_word,
+                           cudaStream_t stream);
+cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const int32_t* keep_rows,
+                           const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
+                           int64_t C_out, void* dX, const int32_t* status_word, cudaStream_t stream);
+
+// tcgen05 / TMEM bf16 products
+bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+sbp_status launch_tc_dw(const void* X_keep, const void* dY, const int32_t* keep_rows,
+                        const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
+                        int64_t C_out, float* dW, bool accumulate, float* workspace,
+                        int32_t* status_word, cudaStream_t stream);
+sbp_status launch_tc_dx(const void* dY, const void* W, const int32_t* keep_rows,
+                        const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
+                        int64_t C_out, void* dX, int32_t* status_word, cudaStream_t stream);
+
+}  // namespace sbp
