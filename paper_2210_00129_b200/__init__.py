@@ -1,5 +1,125 @@
 """B200-native Stochastic Backpropagation (SBP) linear-layer hot path.
 
-The compute lives in a C-ABI CUDA library (``include/sbp.h``); this package is
-its thin Python binding plus the seeded input generators (``synth``).
+The compute lives in a C-ABI CUDA library (``include/sbp.h``, built in-tree as
+``libsbp_b200.so``); this module is its thin Python binding: the functions below carry the
+same names as the C entry points and only marshal arguments (torch tensors -> device
+pointers, the current torch stream -> ``cudaStream_t``).  Every step of the path runs in the
+library's kernels; there is no fallback - a missing library raises at the first call.
+
+``synth`` (seeded input generators) is importable without the library.
 """
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsbp_b200.so")
+
+# enums of include/sbp.h
+SBP_OK, SBP_ERR_INVALID_ARG, SBP_ERR_UNSUPPORTED, SBP_ERR_WORKSPACE = 0, 1, 2, 3
+SBP_ERR_CUDA, SBP_ERR_TIMEOUT, SBP_ERR_BAD_INDICES = 4, 5, 6
+SBP_F32, SBP_BF16 = 0, 1
+SBP_MASK_RANDOM, SBP_MASK_GRID = 0, 1
+SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
+
+EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache",
+           "sbp_linear_backward_workspace_bytes", "sbp_linear_backward")
+
+_lib = None
+
+
+class SbpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (sbp_status {status})")
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libsbp_b200.so``; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2210_00129_b200.build` "
+                           "(the SBP path has no implementation outside this CUDA library)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i64, u64, u32, dbl, vp, sz, ci = (ctypes.c_int64, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_double,
+                                      ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int)
+    lib.sbp_status_string.argtypes = [ci]
+    lib.sbp_status_string.restype = ctypes.c_char_p
+    lib.sbp_keep_count.argtypes = [ci, i64, i64, dbl]
+    lib.sbp_keep_count.restype = i64
+    lib.sbp_sample_keep.argtypes = [ci, i64, i64, i64, dbl, u64, u64, i64, u32, vp, vp, vp]
+    lib.sbp_sample_keep.restype = ci
+    lib.sbp_forward_cache.argtypes = [ci, vp, i64, i64, vp, vp, i64, vp, vp]
+    lib.sbp_forward_cache.restype = ci
+    lib.sbp_linear_backward_workspace_bytes.argtypes = [ci, i64, i64, i64, i64]
+    lib.sbp_linear_backward_workspace_bytes.restype = sz
+    lib.sbp_linear_backward.argtypes = [ci, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp, u32, vp, sz, vp, vp]
+    lib.sbp_linear_backward.restype = ci
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / raw integer address / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != SBP_OK:
+        raise SbpError(status, where)
+
+
+def status_string(status: int) -> str:
+    return load_library().sbp_status_string(int(status)).decode()
+
+
+def sbp_keep_count(mode: int, H: int, W: int, keep_ratio: float) -> int:
+    return int(load_library().sbp_keep_count(mode, H, W, float(keep_ratio)))
+
+
+def sbp_sample_keep(mode, B, H, W, keep_ratio, seed, step, sample_offset, flags, keep_rows, keep_offsets,
+                    stream=None, check=True) -> int:
+    """Fill ``keep_rows`` / ``keep_offsets`` (int32 CUDA tensors) on the current stream."""
+    s = load_library().sbp_sample_keep(mode, B, H, W, float(keep_ratio), seed, step, sample_offset, flags,
+                                       _ptr(keep_rows), _ptr(keep_offsets), _stream(stream))
+    if check:
+        _check(s, "sbp_sample_keep")
+    return s
+
+
+def sbp_forward_cache(dt, X, M, C, keep_rows, M_keep_dev, M_keep_cap, X_keep, stream=None, check=True) -> int:
+    s = load_library().sbp_forward_cache(dt, _ptr(X), M, C, _ptr(keep_rows), _ptr(M_keep_dev), M_keep_cap,
+                                         _ptr(X_keep), _stream(stream))
+    if check:
+        _check(s, "sbp_forward_cache")
+    return s
+
+
+def sbp_linear_backward_workspace_bytes(dt, M, M_keep_cap, C_in, C_out) -> int:
+    return int(load_library().sbp_linear_backward_workspace_bytes(dt, M, M_keep_cap, C_in, C_out))
+
+
+def sbp_linear_backward(dt, X_keep, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW, db, dX,
+                        flags, workspace, workspace_bytes, status_word=None, stream=None, check=True) -> int:
+    s = load_library().sbp_linear_backward(dt, _ptr(X_keep), _ptr(dY), _ptr(W), _ptr(keep_rows), _ptr(M_keep_dev),
+                                           M, M_keep_cap, C_in, C_out, _ptr(dW), _ptr(db), _ptr(dX), flags,
+                                           _ptr(workspace), workspace_bytes, _ptr(status_word), _stream(stream))
+    if check:
+        _check(s, "sbp_linear_backward")
+    return s

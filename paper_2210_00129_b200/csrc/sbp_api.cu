@@ -1,0 +1,179 @@
+// The extern "C" boundary declared in include/sbp.h: argument checks, kernel choice, launches.
+#include <math.h>
+
+#include "sbp_common.cuh"
+
+namespace {
+
+using namespace sbp;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int grid_family_of(double r) {
+    if (r == 0.25) return 1;
+    if (r == 0.5) return 2;
+    if (r == 0.75) return 3;
+    if (r == 1.0) return 4;
+    return 0;
+}
+
+inline bool ratio_ok(double r) { return r > 0.0 && r <= 1.0; }   // false for NaN
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline bool use_tensor_cores(sbp_dtype dt, uint32_t flags, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
+    return dt == SBP_BF16 && !(flags & SBP_FLAG_PLAIN_FMA) && tc_shapes_supported(M, M_keep_cap, C_in, C_out);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sbp_status_string(sbp_status s) {
+    switch (s) {
+        case SBP_OK: return "ok";
+        case SBP_ERR_INVALID_ARG: return "invalid argument";
+        case SBP_ERR_UNSUPPORTED: return "unsupported request";
+        case SBP_ERR_WORKSPACE: return "workspace missing or too small";
+        case SBP_ERR_CUDA: return "CUDA call failed";
+        case SBP_ERR_TIMEOUT: return "bounded device wait expired";
+        case SBP_ERR_BAD_INDICES: return "keep_rows not strictly ascending or out of range";
+    }
+    return "unknown status";
+}
+
+int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_ratio) {
+    if (H <= 0 || W <= 0 || !ratio_ok(keep_ratio)) return -1;
+    const int64_t N = H * W;
+    if (mode == SBP_MASK_RANDOM) {
+        int64_t K = (int64_t)floor(keep_ratio * (double)N + 0.5);
+        if (K < 1) K = 1;
+        if (K > N) K = N;
+        return K;
+    }
+    if (mode == SBP_MASK_GRID) {
+        const int64_t quarter_max = ((H + 1) / 2) * ((W + 1) / 2);   // phase (0, 0) holds the most lattice points
+        const int64_t quarter_min = (H / 2) * (W / 2);               // phase (1, 1) the fewest
+        switch (grid_family_of(keep_ratio)) {
+            case 1: return quarter_max;
+            case 2: return (N + 1) / 2;
+            case 3: return N - quarter_min;
+            case 4: return N;
+            default: return -1;
+        }
+    }
+    return -1;
+}
+
+sbp_status sbp_sample_keep(sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, double keep_ratio,
+                           uint64_t seed, uint64_t step, int64_t sample_offset, uint32_t flags,
+                           int32_t* keep_rows, int32_t* keep_offsets, void* stream) {
+    if (mode != SBP_MASK_RANDOM && mode != SBP_MASK_GRID) return SBP_ERR_INVALID_ARG;
+    if (keep_rows == nullptr || keep_offsets == nullptr) return SBP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(keep_rows) & 3u) || (reinterpret_cast<uintptr_t>(keep_offsets) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || !ratio_ok(keep_ratio)) return SBP_ERR_INVALID_ARG;
+    if (H >= (1ll << 31) || W >= (1ll << 31) || H * W >= (1ll << 31) || B >= (1ll << 31) ||
+        B * (H * W) >= (1ll << 31))
+        return SBP_ERR_INVALID_ARG;
+    if (step >> 32) return SBP_ERR_INVALID_ARG;
+    if (sample_offset < 0 || ((uint64_t)(sample_offset + B - 1) >> 32)) return SBP_ERR_INVALID_ARG;
+    const int family = grid_family_of(keep_ratio);
+    if (mode == SBP_MASK_GRID && family == 0) return SBP_ERR_UNSUPPORTED;
+    const int64_t K = sbp_keep_count(mode, H, W, keep_ratio);
+    const cudaError_t e = launch_sample_keep((int)mode, family, B, H, W, K, seed, (uint32_t)step,
+                                             (uint32_t)sample_offset, (flags & SBP_FLAG_SHARE_MASK) != 0,
+                                             keep_rows, keep_offsets, (cudaStream_t)stream);
+    return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
+sbp_status sbp_forward_cache(sbp_dtype dt, const void* X, int64_t M, int64_t C, const int32_t* keep_rows,
+                             const int32_t* M_keep_dev, int64_t M_keep_cap, void* X_keep, void* stream) {
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (X == nullptr || X_keep == nullptr || keep_rows == nullptr) return SBP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(X_keep)) return SBP_ERR_INVALID_ARG;
+    if (M <= 0 || C <= 0 || M_keep_cap < 0 || M >= (1ll << 31) || M_keep_cap > M) return SBP_ERR_INVALID_ARG;
+    const int64_t row_bytes = C * (dt == SBP_BF16 ? 2 : 4);
+    if (row_bytes % 16 != 0) return SBP_ERR_UNSUPPORTED;
+    const cudaError_t e = launch_gather_rows(X, row_bytes, keep_rows, M_keep_dev, M_keep_cap, X_keep,
+                                             (cudaStream_t)stream);
+    return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
+size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
+                                           int64_t C_out) {
+    if (M <= 0 || M_keep_cap < 0 || C_in <= 0 || C_out <= 0) return 256;
+    const size_t db_part = align_up(db_workspace_bytes(M_keep_cap, C_out), 256);
+    size_t dw_part = simt_dw_workspace_bytes(M_keep_cap, C_in, C_out);
+    if (dt == SBP_BF16 && tc_shapes_supported(M, M_keep_cap, C_in, C_out)) {
+        const size_t t = tc_dw_workspace_bytes(M_keep_cap, C_in, C_out);
+        if (t > dw_part) dw_part = t;
+    }
+    return db_part + align_up(dw_part, 256) + 256;
+}
+
+sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY, const void* W,
+                               const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M,
+                               int64_t M_keep_cap, int64_t C_in, int64_t C_out, float* dW, float* db, void* dX,
+                               uint32_t flags, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                               void* stream_v) {
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (dY == nullptr || keep_rows == nullptr) return SBP_ERR_INVALID_ARG;
+    if (M <= 0 || M >= (1ll << 31) || M_keep_cap < 0 || M_keep_cap > M || C_in <= 0 || C_out <= 0 ||
+        C_in >= (1ll << 24) || C_out >= (1ll << 24))
+        return SBP_ERR_INVALID_ARG;
+    if (dW != nullptr && X_keep == nullptr) return SBP_ERR_INVALID_ARG;
+    if (dX != nullptr && W == nullptr) return SBP_ERR_INVALID_ARG;
+    if (!aligned16(X_keep) || !aligned16(dY) || !aligned16(W) || !aligned16(dW) || !aligned16(db) ||
+        !aligned16(dX) || (reinterpret_cast<uintptr_t>(keep_rows) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    if ((flags & SBP_FLAG_VALIDATE) && status_word == nullptr) return SBP_ERR_INVALID_ARG;
+    const int64_t mult = (dt == SBP_BF16) ? 8 : 4;
+    if (C_in % mult != 0 || C_out % mult != 0) return SBP_ERR_UNSUPPORTED;
+    const bool need_ws = (dW != nullptr) || (db != nullptr);
+    if (need_ws) {
+        if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+            workspace_bytes < sbp_linear_backward_workspace_bytes(dt, M, M_keep_cap, C_in, C_out))
+            return SBP_ERR_WORKSPACE;
+    }
+    const bool accumulate = (flags & SBP_FLAG_ACCUMULATE) != 0;
+    float* ws_db = static_cast<float*>(workspace);
+    float* ws_dw = need_ws ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
+                                                      align_up(db_workspace_bytes(M_keep_cap, C_out), 256))
+                           : nullptr;
+
+    if (flags & SBP_FLAG_VALIDATE) {
+        if (launch_validate_keep_rows(keep_rows, M_keep_dev, M_keep_cap, M, status_word, stream) != cudaSuccess)
+            return SBP_ERR_CUDA;
+    }
+    const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
+    if (db != nullptr) {
+        if (launch_db(dt, dY, keep_rows, M_keep_dev, M_keep_cap, C_out, db, accumulate, ws_db, status_word,
+                      stream) != cudaSuccess)
+            return SBP_ERR_CUDA;
+    }
+    if (dW != nullptr) {
+        if (tc) {
+            const sbp_status s = launch_tc_dw(X_keep, dY, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW,
+                                              accumulate, ws_dw, status_word, stream);
+            if (s != SBP_OK) return s;
+        } else if (launch_simt_dw(dt, X_keep, dY, keep_rows, M_keep_dev, M_keep_cap, C_in, C_out, dW, accumulate,
+                                  ws_dw, status_word, stream) != cudaSuccess) {
+            return SBP_ERR_CUDA;
+        }
+    }
+    if (dX != nullptr) {
+        if (tc) {
+            const sbp_status s = launch_tc_dx(dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dX,
+                                              status_word, stream);
+            if (s != SBP_OK) return s;
+        } else if (launch_simt_dx(dt, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dX, status_word,
+                                  stream) != cudaSuccess) {
+            return SBP_ERR_CUDA;
+        }
+    }
+    return SBP_OK;
+}
+
+}  // extern "C"
