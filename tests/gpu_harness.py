@@ -46,7 +46,7 @@ def run_forward_cache(dtype, X_dev, keep_rows_dev, M_keep_cap, M_keep_dev=None):
 def run_backward(dtype, X_keep_dev, dY_dev, W_dev, keep_rows_dev, M_keep_cap, M_keep_dev=None, flags=0,
                  want=("dW", "db", "dX"), init=None, with_status=True):
     M, C_out = dY_dev.shape
-    C_in = W_dev.shape[0]
+    C_in = W_dev.shape[0] if W_dev is not None else X_keep_dev.shape[1]
     code = dt_code(dtype)
     nbytes = sbp.sbp_linear_backward_workspace_bytes(code, M, M_keep_cap, C_in, C_out)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
