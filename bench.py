@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the SBP linear-layer hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: draw the keep set,
+build the forward cache, run the SBP backward (db, dW, dX).  Default workload: the ViT-B/16 MLP
+fc1 layer (bf16, B=64, 14x14 tokens, 768 -> 3072, keep ratio 0.5, random mask).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints one JSON line (rank 0).  ``value`` counts the backward FLOPs of the kept rows
+(4 * M_keep * C_in * C_out per step and GPU) over device time, with inputs resident in HBM;
+``e2e`` is the same metric through ``sbp_step_host`` with pinned host tensors (copies timed).
+With N > 1 (torchrun) every rank processes its own shard of the batch (its own sample ids);
+the path has no exchange step, so no collective is issued and scaling is weak.
+``--impl reference`` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2210_00129_b200 import synth  # noqa: E402
+
+METRIC = "sbp_backward_tflops_kept_rows"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+WORKLOADS = {
+    # name: dtype, B, H, W, C_in, C_out, keep ratio, mask mode
+    "vit_b16_fc1": dict(dtype="bf16", B=64, H=14, W=14, C_in=768, C_out=3072, keep_ratio=0.5, mode=0),
+    "vit_b16_fc2": dict(dtype="bf16", B=64, H=14, W=14, C_in=3072, C_out=768, keep_ratio=0.5, mode=0),
+    "vit_b16_fc1_b128": dict(dtype="bf16", B=128, H=14, W=14, C_in=768, C_out=3072, keep_ratio=0.5, mode=0),
+    "vit_b16_qkv_b128": dict(dtype="bf16", B=128, H=14, W=14, C_in=768, C_out=2304, keep_ratio=0.5, mode=0),
+    "vit_b16_proj_b128": dict(dtype="bf16", B=128, H=14, W=14, C_in=768, C_out=768, keep_ratio=0.5, mode=0),
+    "convnext_b_s1_pw1": dict(dtype="bf16", B=64, H=56, W=56, C_in=128, C_out=512, keep_ratio=0.5, mode=0),
+    "convnext_b_s1_pw2": dict(dtype="bf16", B=64, H=56, W=56, C_in=512, C_out=128, keep_ratio=0.5, mode=0),
+    "convnext_b_s3_pw1_grid": dict(dtype="bf16", B=64, H=14, W=14, C_in=512, C_out=2048, keep_ratio=0.5, mode=1),
+    "det_s1_pw1": dict(dtype="bf16", B=2, H=200, W=334, C_in=128, C_out=512, keep_ratio=0.5, mode=0),
+    "single_fp32": dict(dtype="f32", B=2, H=16, W=1, C_in=32, C_out=64, keep_ratio=0.5, mode=0),
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason sampler running beside the timed region."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, power = [], [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # samples under load: the upper half of the clock readings while kernels were running
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def bytes_of(dtype):
+    return 2 if dtype == "bf16" else 4
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm / CPU baseline: the fp64 oracle, as it stands, on a bounded sample
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_step(w, B_s, data_seed):
+    """One whole step of the oracle on the first B_s samples of the workload; returns (seconds, flops)."""
+    import oracle
+    N = w["H"] * w["W"]
+    M = B_s * N
+    X, Wt, dY = synth.layer_inputs(w["dtype"], M, w["C_in"], w["C_out"], data_seed)
+    Xf, Wf, dYf = (synth.to_f64(a, w["dtype"]) for a in (X, Wt, dY))
+    t0 = time.perf_counter()
+    keep, _ = oracle.sample_keep(w["mode"], B_s, w["H"], w["W"], w["keep_ratio"], 0, 0, 0)
+    Xk = oracle.forward_cache(Xf, keep)
+    oracle.linear_backward(Xk, dYf, Wf, keep)
+    dt = time.perf_counter() - t0
+    return dt, 4.0 * len(keep) * w["C_in"] * w["C_out"]
+
+
+def pick_oracle_sample(w, target_s=12.0):
+    """Samples of the batch the oracle gets: sized from a one-sample probe to ~target_s seconds."""
+    import oracle
+    oracle.build()
+    t1, _ = oracle_sample_step(w, 1, 999)
+    B_s = int(max(1, min(w["B"], target_s / max(t1, 1e-4))))
+    return B_s
+
+
+def run_reference(args, w, name):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    # bounded sample: the whole run (probe + warm-up + K steps) stays near a minute and a half
+    B_s = pick_oracle_sample(w, target_s=min(6.0, 90.0 / (args.steps + 2)))
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(w, B_s, 1000)
+    times, flops = [], 0.0
+    for _ in range(args.steps):
+        dt, fl = oracle_sample_step(w, B_s, 1000)
+        times.append(dt); flops = fl
+    total = sum(times)
+    value = flops * args.steps / total / 1e12
+    cores = oracle.num_threads()
+    sample = f"first {B_s} of {w['B']} samples of {name} per step (whole path: sampler, cache, dW, db, dX)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, **{k: w[k] for k in ("B", "H", "W", "C_in", "C_out", "keep_ratio")},
+                       "mask": "grid" if w["mode"] else "random"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# CUDA arm
+# ----------------------------------------------------------------------------------------------
+def run_cuda(args, w, name):
+    import torch
+    import torch.distributed as dist
+    import paper_2210_00129_b200 as sbp
+    from paper_2210_00129_b200 import build as sbp_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        sbp_build.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    sbp.load_library()
+
+    dtype, B, H, W_, C_in, C_out, r, mode = (w[k] for k in ("dtype", "B", "H", "W", "C_in", "C_out", "keep_ratio", "mode"))
+    code = sbp.SBP_BF16 if dtype == "bf16" else sbp.SBP_F32
+    es = bytes_of(dtype)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    N = H * W_
+    M = B * N
+    cap = sbp.sbp_keep_count(mode, H, W_, r)
+    cap_total = B * cap
+    sample_offset = rank * B
+
+    def to_dev(a):
+        t = torch.from_numpy(a).cuda()
+        return t.view(torch.bfloat16) if dtype == "bf16" else t
+
+    # ---- buffer sets: rotate so that consecutive steps never find their inputs in the 126 MB L2 ----
+    set_bytes = (M * C_in + M * C_out + C_in * C_out + cap_total * C_in + M * C_in) * es + C_in * C_out * 4
+    n_sets = max(2, int(np.ceil(3 * 126e6 / set_bytes)) + 1)
+    n_sets = min(n_sets, 64)
+    sets = []
+    Xh, Wh, dYh = synth.layer_inputs(dtype, M, C_in, C_out, 1002 + rank)
+    for i in range(n_sets):
+        s = dict(X=to_dev(Xh), W=to_dev(Wh), dY=to_dev(dYh))
+        if i:   # same distribution, different bits per set: roll the seeded tensors
+            s["X"] = torch.roll(s["X"], i, 0); s["dY"] = torch.roll(s["dY"], i, 0)
+        # index and cache buffers hold a full batch so the same sets also serve the keep = 1.0 comparison
+        s["rows"] = torch.zeros(M, dtype=torch.int32, device="cuda")
+        s["offs"] = torch.zeros(B + 1, dtype=torch.int32, device="cuda")
+        s["Xk"] = torch.zeros((M, C_in), dtype=tdt, device="cuda")
+        s["dW"] = torch.zeros((C_in, C_out), dtype=torch.float32, device="cuda")
+        s["db"] = torch.zeros(C_out, dtype=torch.float32, device="cuda")
+        s["dX"] = torch.zeros((M, C_in), dtype=tdt, device="cuda")
+        sets.append(s)
+    ws_bytes = max(sbp.sbp_linear_backward_workspace_bytes(code, M, cap_total, C_in, C_out),
+                   sbp.sbp_linear_backward_workspace_bytes(code, M, M, C_in, C_out))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    sid = stream.cuda_stream
+
+    def step(i, keep_ratio=r, events=None):
+        s = sets[i % n_sets]
+        cnt = s["offs"][B:B + 1]
+        capk = B * sbp.sbp_keep_count(mode, H, W_, keep_ratio) if keep_ratio != r else cap_total
+        sbp.sbp_sample_keep(mode, B, H, W_, keep_ratio, 0, i, sample_offset, 0, s["rows"], s["offs"], stream=sid)
+        sbp.sbp_forward_cache(code, s["X"], M, C_in, s["rows"], cnt, capk, s["Xk"], stream=sid)
+        if events is not None:
+            events[0].record(stream)
+        sbp.sbp_linear_backward(code, None, s["dY"], None, s["rows"], cnt, M, capk, C_in, C_out, None, s["db"], None,
+                                0, ws, ws_bytes, status, stream=sid)
+        sbp.sbp_linear_backward(code, s["Xk"], s["dY"], None, s["rows"], cnt, M, capk, C_in, C_out, s["dW"], None, None,
+                                0, ws, ws_bytes, status, stream=sid)
+        if events is not None:
+            events[1].record(stream)
+        sbp.sbp_linear_backward(code, None, s["dY"], s["W"], s["rows"], cnt, M, capk, C_in, C_out, None, None, s["dX"],
+                                0, ws, ws_bytes, status, stream=sid)
+        if events is not None:
+            events[2].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(k_steps, keep_ratio=r, per_kernel=False):
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k_steps)] if per_kernel else None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(k_steps):
+            step(i, keep_ratio, evs[i] if evs else None)
+        e1.record(stream)
+        barrier()
+        total_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        dx_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / k_steps if evs else None
+        dwdb_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / k_steps if evs else None
+        return total_ms, dx_ms, dwdb_ms
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert int(status.item()) == 0, "device status word set during warm-up"
+    M_keep = int(sets[0]["offs"][B].item())
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+    total_ms, dx_ms, dwdb_ms = timed(args.steps, per_kernel=True)
+    if sampler:
+        clocks = sampler.stop()
+    assert int(status.item()) == 0, "device status word set during the timed steps"
+
+    flops_step = 4.0 * M_keep * C_in * C_out
+    value = flops_step * args.steps * world / (total_ms * 1e-3) / 1e12
+
+    # ---- same kernels at keep ratio 1.0: backward speed-up and saved-activation memory ----
+    bwd_steps = max(3, args.steps // 4)
+    for i in range(3):
+        step(i, 1.0)
+    full_ms, full_dx, full_dwdb = timed(bwd_steps, keep_ratio=1.0, per_kernel=True)
+    bwd_speedup = (full_dx + full_dwdb) / (dx_ms + dwdb_ms)
+    saved_frac = (M_keep * C_in * es + 4 * M_keep + 4 * (B + 1)) / (M * C_in * es)
+
+    # ---- end to end from pinned host tensors through sbp_step_host ----
+    arena_bytes = sbp.sbp_step_host_arena_bytes(code, mode, B, H, W_, C_in, C_out, r)
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device="cuda")
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    Xp, Wp, dYp = pin(Xh), pin(Wh), pin(dYh)
+    dWp = torch.empty((C_in, C_out), dtype=torch.float32).pin_memory()
+    dbp = torch.empty(C_out, dtype=torch.float32).pin_memory()
+    dXp = torch.empty((M, C_in), dtype=torch.int16 if dtype == "bf16" else torch.float32).pin_memory()
+    stp = torch.zeros(1, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def host_step(i):
+        sbp.sbp_step_host(code, mode, B, H, W_, C_in, C_out, r, 0, i, sample_offset, 0, Xp, dYp, Wp, dWp, dbp, dXp,
+                          None, None, stp, arena, arena_bytes, stream=sid)
+    for i in range(2):
+        host_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        host_step(i)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    assert int(stp.item()) == 0
+    e2e_value = flops_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e12
+    h2d = (M * C_in + M * C_out + C_in * C_out) * es
+    d2h = C_in * C_out * 4 + C_out * 4 + M * C_in * es + 4
+
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        tc_path = dtype == "bf16" and min(C_in, C_out) >= 128 and cap_total >= 64
+        dx_flops = 2.0 * M_keep * C_in * C_out
+        if tc_path:
+            peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+            roofline = {"kernel": "tc_dx_kernel", "bound": "tensor", "achieved": dx_flops / (dx_ms * 1e-3) / 1e12,
+                        "peak": peak, "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step)",
+                        "unit": "TFLOP/s", "traffic": None}
+        else:
+            # plain-FMA path: 128 fp32 FMA lanes x 148 SMs x 2 FLOP at the maximum SM clock
+            peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            roofline = {"kernel": "simt_dx_kernel", "bound": "alu", "achieved": dx_flops / (dx_ms * 1e-3) / 1e12,
+                        "peak": peak, "peak_kind": "derived: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz", "unit": "TFLOP/s",
+                        "traffic": None}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline["dx_ms"] = dx_ms
+        roofline["dw_db_ms"] = dwdb_ms
+
+        B_s = pick_oracle_sample(w)
+        import oracle
+        cpu_s, cpu_flops = oracle_sample_step(w, B_s, 1000)
+        launches_per_step = 2 + sbp.sbp_linear_backward_kernel_count(code, M, cap_total, C_in, C_out, True, True, True, 0)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": name, "B_per_gpu": B, "H": H, "W": W_, "C_in": C_in, "C_out": C_out, "keep_ratio": r,
+                       "mask": "grid" if mode else "random", "M": M, "M_keep": M_keep,
+                       "l2": f"inputs larger than L2: {n_sets} rotating buffer sets of {set_bytes / 1e6:.0f} MB",
+                       "parallelism": f"dp{world} (batch sharded by sample id, no collective)"},
+            "roofline": roofline,
+            "cpu_baseline": {"value": cpu_flops / cpu_s / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+                             "kind": "oracle", "seconds": cpu_s,
+                             "sample": f"first {B_s} of {B} samples of {name}, whole path once, fp64"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps, "api": "sbp_step_host (pinned host tensors)"},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+            "bwd_speedup_vs_keep1": bwd_speedup,
+            "bwd_ms": {"keep": dx_ms + dwdb_ms, "keep1": full_dx + full_dwdb},
+            "saved_activation_frac_vs_keep1": saved_frac,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="vit_b16_fc1", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    args = ap.parse_args()
+    w = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w, args.workload)
+    else:
+        run_cuda(args, w, args.workload)
+
+
+if __name__ == "__main__":
+    main()

@@ -163,6 +163,42 @@ sbp_status sbp_linear_backward(sbp_dtype dt,
                                uint32_t flags, void* workspace /* dev */, size_t workspace_bytes,
                                int32_t* status_word /* dev, nullable */, void* stream);
 
+/*
+ * Number of kernels one sbp_linear_backward call with these arguments enqueues (diagnostic,
+ * pure host function; the paper has no counterpart).  want_* select the outputs requested.
+ */
+int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
+                                     int64_t C_out, int want_dW, int want_db, int want_dX,
+                                     uint32_t flags);
+
+/*
+ * One whole SBP step of a layer for callers whose tensors live in HOST memory: copies X, dY, W
+ * to the device, draws the keep set (Sec. 4), builds the forward cache (Algorithm 1), runs the
+ * backward (Eq. 5) and copies dW, db, dX (and optionally the indices) back, all enqueued on
+ * `stream`; the caller synchronises the stream before reading the host outputs.  Host buffers
+ * should be page-locked so the copies run asynchronously.
+ *
+ * X_host [B*H*W, C_in], dY_host [B*H*W, C_out], W_host [C_in, C_out]: element type dt.
+ * dW_host [C_in, C_out] fp32, db_host [C_out] fp32, dX_host [B*H*W, C_in] dt.
+ * keep_rows_host (nullable, capacity B * sbp_keep_count(...)), keep_offsets_host (nullable,
+ * B + 1 entries), status_host (nullable, one int32: the device status word of the step).
+ * arena (dev): caller-owned scratch of at least sbp_step_host_arena_bytes(...) bytes, 256-byte
+ * aligned; holds the device copies of every tensor during the step.  Nothing is allocated.
+ * flags: SBP_FLAG_SHARE_MASK, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA (accumulation is not offered).
+ * Errors as for the three calls it is built from; SBP_ERR_WORKSPACE for a short arena.
+ */
+size_t sbp_step_host_arena_bytes(sbp_dtype dt, sbp_mask_mode mode, int64_t B, int64_t H, int64_t W,
+                                 int64_t C_in, int64_t C_out, double keep_ratio);
+
+sbp_status sbp_step_host(sbp_dtype dt, sbp_mask_mode mode, int64_t B, int64_t H, int64_t W,
+                         int64_t C_in, int64_t C_out, double keep_ratio, uint64_t seed, uint64_t step,
+                         int64_t sample_offset, uint32_t flags,
+                         const void* X_host, const void* dY_host, const void* W_host,
+                         float* dW_host, float* db_host, void* dX_host,
+                         int32_t* keep_rows_host /* nullable */, int32_t* keep_offsets_host /* nullable */,
+                         int32_t* status_host /* nullable */,
+                         void* arena /* dev */, size_t arena_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,8 @@ SBP_MASK_RANDOM, SBP_MASK_GRID = 0, 1
 SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache",
-           "sbp_linear_backward_workspace_bytes", "sbp_linear_backward")
+           "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
+           "sbp_step_host_arena_bytes", "sbp_step_host")
 
 _lib = None
 
@@ -58,6 +59,13 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_linear_backward_workspace_bytes.restype = sz
     lib.sbp_linear_backward.argtypes = [ci, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp, u32, vp, sz, vp, vp]
     lib.sbp_linear_backward.restype = ci
+    lib.sbp_linear_backward_kernel_count.argtypes = [ci, i64, i64, i64, i64, ci, ci, ci, u32]
+    lib.sbp_linear_backward_kernel_count.restype = ci
+    lib.sbp_step_host_arena_bytes.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl]
+    lib.sbp_step_host_arena_bytes.restype = sz
+    lib.sbp_step_host.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl, u64, u64, i64, u32,
+                                  vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sbp_step_host.restype = ci
     _lib = lib
     return lib
 
@@ -122,4 +130,27 @@ def sbp_linear_backward(dt, X_keep, dY, W, keep_rows, M_keep_dev, M, M_keep_cap,
                                            _ptr(workspace), workspace_bytes, _ptr(status_word), _stream(stream))
     if check:
         _check(s, "sbp_linear_backward")
+    return s
+
+
+def sbp_linear_backward_kernel_count(dt, M, M_keep_cap, C_in, C_out, want_dW=True, want_db=True, want_dX=True,
+                                     flags=0) -> int:
+    return int(load_library().sbp_linear_backward_kernel_count(dt, M, M_keep_cap, C_in, C_out, int(want_dW),
+                                                               int(want_db), int(want_dX), flags))
+
+
+def sbp_step_host_arena_bytes(dt, mode, B, H, W, C_in, C_out, keep_ratio) -> int:
+    return int(load_library().sbp_step_host_arena_bytes(dt, mode, B, H, W, C_in, C_out, float(keep_ratio)))
+
+
+def sbp_step_host(dt, mode, B, H, W, C_in, C_out, keep_ratio, seed, step, sample_offset, flags, X_host, dY_host,
+                  W_host, dW_host, db_host, dX_host, keep_rows_host, keep_offsets_host, status_host, arena,
+                  arena_bytes, stream=None, check=True) -> int:
+    """Whole step from host (ideally pinned) tensors; results land in the host outputs once the stream is synced."""
+    s = load_library().sbp_step_host(dt, mode, B, H, W, C_in, C_out, float(keep_ratio), seed, step, sample_offset,
+                                     flags, _ptr(X_host), _ptr(dY_host), _ptr(W_host), _ptr(dW_host), _ptr(db_host),
+                                     _ptr(dX_host), _ptr(keep_rows_host), _ptr(keep_offsets_host), _ptr(status_host),
+                                     _ptr(arena), arena_bytes, _stream(stream))
+    if check:
+        _check(s, "sbp_step_host")
     return s

@@ -184,6 +184,10 @@ size_t simt_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) 
     return s > 1 ? (size_t)s * (size_t)C_in * (size_t)C_out * sizeof(float) : 0;
 }
 
+int simt_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
+    return simt_dw_splits(M_keep_cap, C_in, C_out) > 1 ? 2 : 1;
+}
+
 cudaError_t launch_simt_dw(sbp_dtype dt, const void* X_keep, const void* dY, const int32_t* keep_rows,
                            const int32_t* M_keep_dev, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
                            float* dW, bool accumulate, float* workspace, const int32_t* status_word,

@@ -176,4 +176,101 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     return SBP_OK;
 }
 
+int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
+                                     int want_dW, int want_db, int want_dX, uint32_t flags) {
+    const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
+    int n = (flags & SBP_FLAG_VALIDATE) ? 1 : 0;
+    if (want_db) n += 2;                                   // strip partials + fixed-order reduce
+    if (want_dW) n += tc ? tc_dw_kernel_count(M_keep_cap, C_in, C_out) : simt_dw_kernel_count(M_keep_cap, C_in, C_out);
+    if (want_dX) n += 1;
+    return n;
+}
+
+namespace {
+struct StepArena {
+    size_t X, dY, W, rows, offs, Xk, dW, db, dX, status, ws, ws_bytes, total;
+};
+StepArena plan_step_arena(sbp_dtype dt, int64_t M, int64_t cap_total, int64_t B, int64_t C_in, int64_t C_out) {
+    const size_t es = (dt == SBP_BF16) ? 2 : 4;
+    StepArena a;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t at = off; off += align_up(bytes, 256); return at; };
+    a.X = take((size_t)M * C_in * es);
+    a.dY = take((size_t)M * C_out * es);
+    a.W = take((size_t)C_in * C_out * es);
+    a.rows = take((size_t)cap_total * 4);
+    a.offs = take((size_t)(B + 1) * 4);
+    a.Xk = take((size_t)cap_total * C_in * es);
+    a.dW = take((size_t)C_in * C_out * 4);
+    a.db = take((size_t)C_out * 4);
+    a.dX = take((size_t)M * C_in * es);
+    a.status = take(4);
+    a.ws_bytes = sbp_linear_backward_workspace_bytes(dt, M, cap_total, C_in, C_out);
+    a.ws = take(a.ws_bytes);
+    a.total = off;
+    return a;
+}
+}  // namespace
+
+size_t sbp_step_host_arena_bytes(sbp_dtype dt, sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, int64_t C_in,
+                                 int64_t C_out, double keep_ratio) {
+    const int64_t cap = sbp_keep_count(mode, H, W, keep_ratio);
+    if (cap < 0 || B <= 0 || C_in <= 0 || C_out <= 0) return 0;
+    return plan_step_arena(dt, B * H * W, B * cap, B, C_in, C_out).total;
+}
+
+sbp_status sbp_step_host(sbp_dtype dt, sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, int64_t C_in,
+                         int64_t C_out, double keep_ratio, uint64_t seed, uint64_t step, int64_t sample_offset,
+                         uint32_t flags, const void* X_host, const void* dY_host, const void* W_host,
+                         float* dW_host, float* db_host, void* dX_host, int32_t* keep_rows_host,
+                         int32_t* keep_offsets_host, int32_t* status_host, void* arena, size_t arena_bytes,
+                         void* stream_v) {
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (X_host == nullptr || dY_host == nullptr || W_host == nullptr || dW_host == nullptr || db_host == nullptr ||
+        dX_host == nullptr)
+        return SBP_ERR_INVALID_ARG;
+    if (flags & SBP_FLAG_ACCUMULATE) return SBP_ERR_UNSUPPORTED;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || C_out <= 0) return SBP_ERR_INVALID_ARG;
+    const int64_t cap = sbp_keep_count(mode, H, W, keep_ratio);
+    if (cap < 0) return (mode == SBP_MASK_GRID && ratio_ok(keep_ratio)) ? SBP_ERR_UNSUPPORTED : SBP_ERR_INVALID_ARG;
+    if (H * W >= (1ll << 31) || B * (H * W) >= (1ll << 31)) return SBP_ERR_INVALID_ARG;
+    const int64_t M = B * H * W, cap_total = B * cap;
+    const StepArena a = plan_step_arena(dt, M, cap_total, B, C_in, C_out);
+    if (arena == nullptr || (reinterpret_cast<uintptr_t>(arena) & 255u) || arena_bytes < a.total)
+        return SBP_ERR_WORKSPACE;
+    const size_t es = (dt == SBP_BF16) ? 2 : 4;
+    char* base = static_cast<char*>(arena);
+    auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+    if (!ok(cudaMemcpyAsync(base + a.X, X_host, (size_t)M * C_in * es, cudaMemcpyHostToDevice, stream)) ||
+        !ok(cudaMemcpyAsync(base + a.dY, dY_host, (size_t)M * C_out * es, cudaMemcpyHostToDevice, stream)) ||
+        !ok(cudaMemcpyAsync(base + a.W, W_host, (size_t)C_in * C_out * es, cudaMemcpyHostToDevice, stream)) ||
+        !ok(cudaMemsetAsync(base + a.status, 0, 4, stream)))
+        return SBP_ERR_CUDA;
+    int32_t* rows = reinterpret_cast<int32_t*>(base + a.rows);
+    int32_t* offs = reinterpret_cast<int32_t*>(base + a.offs);
+    int32_t* status = reinterpret_cast<int32_t*>(base + a.status);
+    sbp_status s = sbp_sample_keep(mode, B, H, W, keep_ratio, seed, step, sample_offset, flags, rows, offs, stream);
+    if (s != SBP_OK) return s;
+    s = sbp_forward_cache(dt, base + a.X, M, C_in, rows, offs + B, cap_total, base + a.Xk, stream);
+    if (s != SBP_OK) return s;
+    s = sbp_linear_backward(dt, base + a.Xk, base + a.dY, base + a.W, rows, offs + B, M, cap_total, C_in, C_out,
+                            reinterpret_cast<float*>(base + a.dW), reinterpret_cast<float*>(base + a.db), base + a.dX,
+                            flags & (SBP_FLAG_VALIDATE | SBP_FLAG_PLAIN_FMA), base + a.ws, a.ws_bytes, status, stream);
+    if (s != SBP_OK) return s;
+    if (!ok(cudaMemcpyAsync(dW_host, base + a.dW, (size_t)C_in * C_out * 4, cudaMemcpyDeviceToHost, stream)) ||
+        !ok(cudaMemcpyAsync(db_host, base + a.db, (size_t)C_out * 4, cudaMemcpyDeviceToHost, stream)) ||
+        !ok(cudaMemcpyAsync(dX_host, base + a.dX, (size_t)M * C_in * es, cudaMemcpyDeviceToHost, stream)))
+        return SBP_ERR_CUDA;
+    if (keep_rows_host != nullptr &&
+        !ok(cudaMemcpyAsync(keep_rows_host, rows, (size_t)cap_total * 4, cudaMemcpyDeviceToHost, stream)))
+        return SBP_ERR_CUDA;
+    if (keep_offsets_host != nullptr &&
+        !ok(cudaMemcpyAsync(keep_offsets_host, offs, (size_t)(B + 1) * 4, cudaMemcpyDeviceToHost, stream)))
+        return SBP_ERR_CUDA;
+    if (status_host != nullptr && !ok(cudaMemcpyAsync(status_host, status, 4, cudaMemcpyDeviceToHost, stream)))
+        return SBP_ERR_CUDA;
+    return SBP_OK;
+}
+
 }  // extern "C"

@@ -77,6 +77,7 @@ cudaError_t launch_reduce_partials(const float* partials, int splits, int64_t n,
 
 // plain-FMA (CUDA-core) products for fp32 and for bf16 shapes the tensor-core kernels do not take
 size_t simt_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+int    simt_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 cudaError_t launch_simt_dw(sbp_dtype dt, const void* X_keep, const void* dY, const int32_t* keep_rows,
                            const int32_t* M_keep_dev, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
                            float* dW, bool accumulate, float* workspace, const int32_t* status_word,
@@ -88,6 +89,7 @@ cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const in
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+int    tc_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 sbp_status launch_tc_dw(const void* X_keep, const void* dY, const int32_t* keep_rows,
                         const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
                         int64_t C_out, float* dW, bool accumulate, float* workspace,

@@ -428,6 +428,10 @@ size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
     return p.splits > 1 ? (size_t)p.splits * (size_t)C_in * (size_t)C_out * sizeof(float) : 0;
 }
 
+int tc_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
+    return plan_dw(M_keep_cap, C_in, C_out).splits > 1 ? 2 : 1;
+}
+
 sbp_status launch_tc_dx(const void* dY, const void* W, const int32_t* keep_rows, const int32_t* M_keep_dev,
                         int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out, void* dX,
                         int32_t* status_word, cudaStream_t stream) {
