@@ -199,6 +199,29 @@ sbp_status sbp_step_host(sbp_dtype dt, sbp_mask_mode mode, int64_t B, int64_t H,
                          int32_t* status_host /* nullable */,
                          void* arena /* dev */, size_t arena_bytes, void* stream);
 
+/*
+ * Bias gradient without any workspace argument (an addition of this library; the paper has no
+ * counterpart):  db[j] (+)= sum_{m < M_keep} dY[keep_rows[m], j], as sbp_linear_backward computes it.
+ *
+ * For callers that cannot allocate device memory and so cannot supply a workspace - operator
+ * plugins that receive only their tensors, code under a memory pool owned and locked by another
+ * framework, services with a fixed device-memory budget.  The split-reduction scratch lives in a
+ * fixed 1 MiB device array inside the library (held by every GPU that loads the library until the
+ * process exits).  The call allocates and frees nothing.
+ *
+ * Limits: C_out <= 4096 (SBP_ERR_WORKSPACE beyond it: the built-in scratch is too small; use
+ * sbp_linear_backward with a workspace).  C_out a multiple of 8 (bf16) / 4 (fp32).
+ * flags: SBP_FLAG_ACCUMULATE or 0.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the array, which
+ * keeps the previous call's contents (nothing in it needs clearing: each call overwrites every
+ * entry it later reads); calls whose kernels may overlap on the GPU (different streams) race on it
+ * and must be ordered by the caller.
+ */
+sbp_status sbp_bias_grad_static(sbp_dtype dt, const void* dY /* dev */, const int32_t* keep_rows /* dev */,
+                                const int32_t* M_keep_dev /* dev, nullable */, int64_t M, int64_t M_keep_cap,
+                                int64_t C_out, float* db /* dev */, uint32_t flags, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,7 @@ SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA 
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
-           "sbp_step_host_arena_bytes", "sbp_step_host")
+           "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static")
 
 _lib = None
 
@@ -66,6 +66,8 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_step_host.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl, u64, u64, i64, u32,
                                   vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sbp_step_host.restype = ci
+    lib.sbp_bias_grad_static.argtypes = [ci, vp, vp, vp, i64, i64, i64, vp, u32, vp]
+    lib.sbp_bias_grad_static.restype = ci
     _lib = lib
     return lib
 
@@ -153,4 +155,14 @@ def sbp_step_host(dt, mode, B, H, W, C_in, C_out, keep_ratio, seed, step, sample
                                      _ptr(arena), arena_bytes, _stream(stream))
     if check:
         _check(s, "sbp_step_host")
+    return s
+
+
+def sbp_bias_grad_static(dt, dY, keep_rows, M_keep_dev, M, M_keep_cap, C_out, db, flags=0, stream=None,
+                         check=True) -> int:
+    """Bias gradient with the library's built-in scratch: for callers that cannot allocate a workspace."""
+    s = load_library().sbp_bias_grad_static(dt, _ptr(dY), _ptr(keep_rows), _ptr(M_keep_dev), M, M_keep_cap, C_out,
+                                            _ptr(db), flags, _stream(stream))
+    if check:
+        _check(s, "sbp_bias_grad_static")
     return s
