@@ -225,36 +225,40 @@ def run_cuda(args, w, name):
     sid = stream.cuda_stream
 
     def step(i, keep_ratio=r, events=None):
+        """One pass of the whole path; `events` (6 per step) bracket its five calls on the launch stream."""
         s = sets[i % n_sets]
         cnt = s["offs"][B:B + 1]
         capk = B * sbp.sbp_keep_count(mode, H, W_, keep_ratio) if keep_ratio != r else cap_total
+        rec = (lambda k: events[k].record(stream)) if events is not None else (lambda k: None)
+        rec(0)
         sbp.sbp_sample_keep(mode, B, H, W_, keep_ratio, 0, i, sample_offset, 0, s["rows"], s["offs"], stream=sid)
+        rec(1)
         sbp.sbp_forward_cache(code, s["X"], M, C_in, s["rows"], cnt, capk, s["Xk"], stream=sid)
-        if events is not None:
-            events[0].record(stream)
+        rec(2)
         sbp.sbp_linear_backward(code, None, s["dY"], None, s["rows"], cnt, M, capk, C_in, C_out, None, s["db"], None,
                                 0, ws, ws_bytes, status, stream=sid)
+        rec(3)
         sbp.sbp_linear_backward(code, s["Xk"], s["dY"], None, s["rows"], cnt, M, capk, C_in, C_out, s["dW"], None, None,
                                 0, ws, ws_bytes, status, stream=sid)
-        if events is not None:
-            events[1].record(stream)
+        rec(4)
         sbp.sbp_linear_backward(code, None, s["dY"], s["W"], s["rows"], cnt, M, capk, C_in, C_out, None, None, s["dX"],
                                 0, ws, ws_bytes, status, stream=sid)
-        if events is not None:
-            events[2].record(stream)
+        rec(5)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(k_steps, keep_ratio=r, per_kernel=False):
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(k_steps)] if per_kernel else None
+    PHASES = ("sample_keep", "forward_cache", "db", "dW", "dX")
+
+    def timed(k_steps, keep_ratio=r):
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(k_steps)]
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
         for i in range(k_steps):
-            step(i, keep_ratio, evs[i] if evs else None)
+            step(i, keep_ratio, evs[i])
         e1.record(stream)
         barrier()
         total_ms = e0.elapsed_time(e1)
@@ -262,9 +266,8 @@ def run_cuda(args, w, name):
             t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             total_ms = float(t.item())
-        dx_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / k_steps if evs else None
-        dwdb_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / k_steps if evs else None
-        return total_ms, dx_ms, dwdb_ms
+        phase_ms = {name: sum(e[k].elapsed_time(e[k + 1]) for e in evs) / k_steps for k, name in enumerate(PHASES)}
+        return total_ms, phase_ms
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -276,7 +279,8 @@ def run_cuda(args, w, name):
     if sampler:
         sampler.start()
         time.sleep(0.3)
-    total_ms, dx_ms, dwdb_ms = timed(args.steps, per_kernel=True)
+    total_ms, phase_ms = timed(args.steps)
+    dx_ms = phase_ms["dX"]
     if sampler:
         clocks = sampler.stop()
     assert int(status.item()) == 0, "device status word set during the timed steps"
@@ -288,8 +292,10 @@ def run_cuda(args, w, name):
     bwd_steps = max(3, args.steps // 4)
     for i in range(3):
         step(i, 1.0)
-    full_ms, full_dx, full_dwdb = timed(bwd_steps, keep_ratio=1.0, per_kernel=True)
-    bwd_speedup = (full_dx + full_dwdb) / (dx_ms + dwdb_ms)
+    full_ms, full_phase = timed(bwd_steps, keep_ratio=1.0)
+    bwd_keep = phase_ms["db"] + phase_ms["dW"] + phase_ms["dX"]
+    bwd_full = full_phase["db"] + full_phase["dW"] + full_phase["dX"]
+    bwd_speedup = bwd_full / bwd_keep
     saved_frac = (M_keep * C_in * es + 4 * M_keep + 4 * (B + 1)) / (M * C_in * es)
 
     # ---- end to end from pinned host tensors through sbp_step_host ----
@@ -341,8 +347,7 @@ def run_cuda(args, w, name):
                         "peak": peak, "peak_kind": "derived: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz", "unit": "TFLOP/s",
                         "traffic": None}
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        roofline["dx_ms"] = dx_ms
-        roofline["dw_db_ms"] = dwdb_ms
+        roofline["launch_ms"] = dx_ms
 
         B_s = pick_oracle_sample(w)
         import oracle
@@ -365,7 +370,8 @@ def run_cuda(args, w, name):
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
             "bwd_speedup_vs_keep1": bwd_speedup,
-            "bwd_ms": {"keep": dx_ms + dwdb_ms, "keep1": full_dx + full_dwdb},
+            "bwd_ms": {"keep": bwd_keep, "keep1": bwd_full},
+            "phase_us": {k: round(v * 1e3, 2) for k, v in phase_ms.items()},
             "saved_activation_frac_vs_keep1": saved_frac,
         }
         print(json.dumps(line))

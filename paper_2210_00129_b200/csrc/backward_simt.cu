@@ -54,6 +54,8 @@ simt_dw_kernel(const T* __restrict__ X_keep, const T* __restrict__ dY, const int
                const int32_t* __restrict__ status_word) {
     __shared__ __align__(16) float As[kTileK][kTile];
     __shared__ __align__(16) float Bs[kTileK][kTile];
+    pdl_launch_dependents();
+    pdl_wait();
     if (status_word != nullptr && *status_word != 0) return;
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int splits = gridDim.z;
@@ -110,6 +112,8 @@ simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t*
     __shared__ __align__(16) float Bs[kTileK][kTile + 4];
     // rows[0] = kept row before the tile (or -1), rows[1 + t] = rows of the tile, M past the last kept row
     __shared__ int64_t rows[kTile + 2];
+    pdl_launch_dependents();
+    pdl_wait();
     if (status_word != nullptr && *status_word != 0) return;
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int64_t m0 = (int64_t)blockIdx.x * kTile;
@@ -197,15 +201,15 @@ cudaError_t launch_simt_dw(sbp_dtype dt, const void* X_keep, const void* dY, con
     float* out = splits > 1 ? workspace : dW;
     const int acc_in_kernel = (splits == 1 && accumulate) ? 1 : 0;
     const int64_t split_stride = C_in * C_out;
+    cudaError_t e;
     if (dt == SBP_BF16)
-        simt_dw_kernel<__nv_bfloat16><<<grid, kSimtThreads, 0, stream>>>(
-            (const __nv_bfloat16*)X_keep, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M_keep_cap,
-            (int)C_in, (int)C_out, out, split_stride, acc_in_kernel, status_word);
+        e = launch_pdl(simt_dw_kernel<__nv_bfloat16>, grid, dim3(kSimtThreads), 0, stream,
+                       (const __nv_bfloat16*)X_keep, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M_keep_cap,
+                       (int)C_in, (int)C_out, out, split_stride, acc_in_kernel, status_word);
     else
-        simt_dw_kernel<float><<<grid, kSimtThreads, 0, stream>>>(
-            (const float*)X_keep, (const float*)dY, keep_rows, M_keep_dev, M_keep_cap,
-            (int)C_in, (int)C_out, out, split_stride, acc_in_kernel, status_word);
-    cudaError_t e = cudaGetLastError();
+        e = launch_pdl(simt_dw_kernel<float>, grid, dim3(kSimtThreads), 0, stream,
+                       (const float*)X_keep, (const float*)dY, keep_rows, M_keep_dev, M_keep_cap,
+                       (int)C_in, (int)C_out, out, split_stride, acc_in_kernel, status_word);
     if (e != cudaSuccess || splits == 1) return e;
     return launch_reduce_partials(workspace, splits, C_in * C_out, dW, accumulate, status_word, stream);
 }
@@ -217,14 +221,12 @@ cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const in
     if (row_tiles < 1) row_tiles = 1;
     const dim3 grid((unsigned)row_tiles, (unsigned)((C_in + kTile - 1) / kTile));
     if (dt == SBP_BF16)
-        simt_dx_kernel<__nv_bfloat16><<<grid, kSimtThreads, 0, stream>>>(
-            (const __nv_bfloat16*)dY, (const __nv_bfloat16*)W, keep_rows, M_keep_dev, M, M_keep_cap,
-            (int)C_in, (int)C_out, (__nv_bfloat16*)dX, status_word);
-    else
-        simt_dx_kernel<float><<<grid, kSimtThreads, 0, stream>>>(
-            (const float*)dY, (const float*)W, keep_rows, M_keep_dev, M, M_keep_cap,
-            (int)C_in, (int)C_out, (float*)dX, status_word);
-    return cudaGetLastError();
+        return launch_pdl(simt_dx_kernel<__nv_bfloat16>, grid, dim3(kSimtThreads), 0, stream,
+                          (const __nv_bfloat16*)dY, (const __nv_bfloat16*)W, keep_rows, M_keep_dev, M, M_keep_cap,
+                          (int)C_in, (int)C_out, (__nv_bfloat16*)dX, status_word);
+    return launch_pdl(simt_dx_kernel<float>, grid, dim3(kSimtThreads), 0, stream,
+                      (const float*)dY, (const float*)W, keep_rows, M_keep_dev, M, M_keep_cap,
+                      (int)C_in, (int)C_out, (float*)dX, status_word);
 }
 
 }  // namespace sbp

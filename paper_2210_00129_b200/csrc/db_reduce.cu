@@ -2,10 +2,10 @@
 // same masking of dY as Eq. 5), and the deterministic reduction of split partial results.
 //
 // db: each block owns a strip of 32 16-byte column vectors and a contiguous share of the kept
-// rows; a warp reads one gathered row strip as 32 x 16-byte vectors (coalesced), the eight warps
-// of a block take different rows, partial sums are combined through shared memory and written
-// to a [splits, C_out] scratch that a second kernel adds up in a fixed order.  HBM-bound: one
-// read of the kept rows of dY.
+// rows; a warp reads one gathered row strip as 32 x 16-byte vectors (coalesced, 512 B), keeps
+// eight such loads in flight, the eight warps of a block take different rows, partial sums are
+// combined through shared memory in a fixed order and written to a [splits, C_out] scratch that
+// a second kernel adds up, again in a fixed order.  HBM-bound: one read of the kept rows of dY.
 #include "sbp_common.cuh"
 
 namespace sbp {
@@ -13,8 +13,8 @@ namespace {
 
 constexpr int kDbThreads = 256;
 constexpr int kDbWarps = kDbThreads / 32;
-constexpr int kDbUnroll = 4;
-constexpr int kDbMaxSplits = 64;
+constexpr int kDbUnroll = 8;
+constexpr int kDbTargetBlocks = 4 * kNumSMs;
 
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {
@@ -36,14 +36,21 @@ template <> struct Vec16<__nv_bfloat16> {
     }
 };
 
-inline int db_splits(int64_t M_keep_cap, int64_t col_vecs) {
+inline int db_splits(int64_t M_keep_cap, int64_t col_vecs, int max_splits) {
     const int64_t strips = (col_vecs + 31) / 32;
-    int64_t s = (2 * (int64_t)kNumSMs + strips - 1) / strips;
-    const int64_t by_rows = (M_keep_cap + 63) / 64;
+    int64_t s = (kDbTargetBlocks + strips - 1) / strips;
+    const int64_t by_rows = (M_keep_cap + 63) / 64;        // at least 64 rows per block
     if (s > by_rows) s = by_rows;
-    if (s > kDbMaxSplits) s = kDbMaxSplits;
+    if (s > max_splits) s = max_splits;
     if (s < 1) s = 1;
     return (int)s;
+}
+
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 
 template <typename T>
@@ -53,6 +60,8 @@ db_partial_kernel(const uint4* __restrict__ dY, uint32_t col_vecs, const int32_t
                   const int32_t* __restrict__ status_word) {
     constexpr int E = Vec16<T>::kElems;
     __shared__ float red[kDbWarps][32 * E];
+    pdl_launch_dependents();
+    pdl_wait();
     if (status_word != nullptr && *status_word != 0) return;
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -67,13 +76,16 @@ db_partial_kernel(const uint4* __restrict__ dY, uint32_t col_vecs, const int32_t
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
     if (cv < col_vecs) {
         for (int64_t m = m_begin + warp; m < m_end; m += kDbWarps * kDbUnroll) {
+            int64_t row[kDbUnroll];
             uint4 v[kDbUnroll];
 #pragma unroll
             for (int u = 0; u < kDbUnroll; ++u) {
                 const int64_t mm = m + u * kDbWarps;
-                v[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (mm < m_end) v[u] = __ldg(dY + (int64_t)__ldg(keep_rows + mm) * col_vecs + cv);
+                row[u] = (mm < m_end) ? (int64_t)__ldg(keep_rows + mm) : -1;
             }
+#pragma unroll
+            for (int u = 0; u < kDbUnroll; ++u)
+                v[u] = (row[u] >= 0) ? ld_stream16(dY + row[u] * col_vecs + cv) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
             for (int u = 0; u < kDbUnroll; ++u) Vec16<T>::accumulate(v[u], acc);
         }
@@ -91,9 +103,12 @@ db_partial_kernel(const uint4* __restrict__ dY, uint32_t col_vecs, const int32_t
     }
 }
 
+// few partials: one thread per float4 of the output, partials added in ascending order
 __global__ void __launch_bounds__(256)
-reduce_partials_kernel(const float4* __restrict__ partials, int splits, int64_t n_vec, float4* __restrict__ out,
-                       int accumulate, const int32_t* __restrict__ status_word) {
+reduce_partials_flat_kernel(const float4* __restrict__ partials, int splits, int64_t n_vec, float4* __restrict__ out,
+                            int accumulate, const int32_t* __restrict__ status_word) {
+    pdl_launch_dependents();
+    pdl_wait();
     if (status_word != nullptr && *status_word != 0) return;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
@@ -106,27 +121,55 @@ reduce_partials_kernel(const float4* __restrict__ partials, int splits, int64_t 
     }
 }
 
+// many partials: 32 float4 columns x 8 interleaved partial lanes per block; each lane adds its
+// partials in ascending order, the eight lane sums are then added in lane order
+__global__ void __launch_bounds__(256)
+reduce_partials_deep_kernel(const float4* __restrict__ partials, int splits, int64_t n_vec, float4* __restrict__ out,
+                            int accumulate, const int32_t* __restrict__ status_word) {
+    __shared__ float4 red[8][32];
+    pdl_launch_dependents();
+    pdl_wait();
+    if (status_word != nullptr && *status_word != 0) return;
+    const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
+    const int64_t i = (int64_t)blockIdx.x * 32 + x;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < n_vec) {
+        for (int k = y; k < splits; k += 8) {
+            const float4 p = __ldg(partials + (int64_t)k * n_vec + i);
+            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+        }
+    }
+    red[y][x] = s;
+    __syncthreads();
+    if (y == 0 && i < n_vec) {
+        float4 t = accumulate ? out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { t.x += red[w][x].x; t.y += red[w][x].y; t.z += red[w][x].z; t.w += red[w][x].w; }
+        out[i] = t;
+    }
+}
+
 }  // namespace
 
-size_t db_workspace_bytes(int64_t M_keep_cap, int64_t C_out) {
-    (void)M_keep_cap;
-    return (size_t)kDbMaxSplits * (size_t)C_out * sizeof(float);
+size_t db_workspace_bytes(sbp_dtype dt, int64_t M_keep_cap, int64_t C_out, int max_splits) {
+    const int64_t col_vecs = C_out / ((dt == SBP_BF16) ? 8 : 4);
+    return (size_t)db_splits(M_keep_cap, col_vecs, max_splits) * (size_t)C_out * sizeof(float);
 }
 
 cudaError_t launch_db(sbp_dtype dt, const void* dY, const int32_t* keep_rows, const int32_t* M_keep_dev,
                       int64_t M_keep_cap, int64_t C_out, float* db, bool accumulate, float* workspace,
-                      const int32_t* status_word, cudaStream_t stream) {
+                      int max_splits, const int32_t* status_word, cudaStream_t stream) {
     const int64_t elems = (dt == SBP_BF16) ? 8 : 4;
     const int64_t col_vecs = C_out / elems;
-    const int splits = db_splits(M_keep_cap, col_vecs);
+    const int splits = db_splits(M_keep_cap, col_vecs, max_splits);
     const dim3 grid((unsigned)((col_vecs + 31) / 32), (unsigned)splits);
+    cudaError_t e;
     if (dt == SBP_BF16)
-        db_partial_kernel<__nv_bfloat16><<<grid, kDbThreads, 0, stream>>>(
-            (const uint4*)dY, (uint32_t)col_vecs, keep_rows, M_keep_dev, M_keep_cap, workspace, status_word);
+        e = launch_pdl(db_partial_kernel<__nv_bfloat16>, grid, dim3(kDbThreads), 0, stream,
+                       (const uint4*)dY, (uint32_t)col_vecs, keep_rows, M_keep_dev, M_keep_cap, workspace, status_word);
     else
-        db_partial_kernel<float><<<grid, kDbThreads, 0, stream>>>(
-            (const uint4*)dY, (uint32_t)col_vecs, keep_rows, M_keep_dev, M_keep_cap, workspace, status_word);
-    cudaError_t e = cudaGetLastError();
+        e = launch_pdl(db_partial_kernel<float>, grid, dim3(kDbThreads), 0, stream,
+                       (const uint4*)dY, (uint32_t)col_vecs, keep_rows, M_keep_dev, M_keep_cap, workspace, status_word);
     if (e != cudaSuccess) return e;
     return launch_reduce_partials(workspace, splits, C_out, db, accumulate, status_word, stream);
 }
@@ -134,12 +177,16 @@ cudaError_t launch_db(sbp_dtype dt, const void* dY, const int32_t* keep_rows, co
 cudaError_t launch_reduce_partials(const float* partials, int splits, int64_t n, float* out,
                                    bool accumulate, const int32_t* status_word, cudaStream_t stream) {
     const int64_t n_vec = n / 4;   // n is a multiple of 4 for every caller
+    if (splits > 8) {
+        const int64_t blocks = (n_vec + 31) / 32;
+        return launch_pdl(reduce_partials_deep_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
+                          (const float4*)partials, splits, n_vec, (float4*)out, accumulate ? 1 : 0, status_word);
+    }
     int64_t blocks = (n_vec + 255) / 256;
     if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
     if (blocks < 1) blocks = 1;
-    reduce_partials_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const float4*)partials, splits, n_vec,
-                                                                (float4*)out, accumulate ? 1 : 0, status_word);
-    return cudaGetLastError();
+    return launch_pdl(reduce_partials_flat_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
+                      (const float4*)partials, splits, n_vec, (float4*)out, accumulate ? 1 : 0, status_word);
 }
 
 }  // namespace sbp

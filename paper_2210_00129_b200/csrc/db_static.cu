@@ -60,13 +60,14 @@ extern "C" sbp_status sbp_bias_grad_static(sbp_dtype dt, const void* dY, const i
     if (C_out % ((dt == SBP_BF16) ? 8 : 4) != 0) return SBP_ERR_UNSUPPORTED;
     // the built-in scratch is sized for kStaticMaxCols columns; wider layers need sbp_linear_backward
     if (C_out > kStaticMaxCols) return SBP_ERR_WORKSPACE;
-    if (sbp::db_workspace_bytes(M_keep_cap, C_out) > kStaticScratchFloats * sizeof(float)) return SBP_ERR_WORKSPACE;
+    if (sbp::db_workspace_bytes(dt, M_keep_cap, C_out, kStaticSplits) > kStaticScratchFloats * sizeof(float))
+        return SBP_ERR_WORKSPACE;
 
     float* scratch = nullptr;
     if (scratch_address(&scratch) != cudaSuccess) return SBP_ERR_CUDA;
     // Nothing in the scratch has to start at zero: the first kernel writes every partial the second reads.
     const cudaError_t e = sbp::launch_db(dt, dY, keep_rows, M_keep_dev, M_keep_cap, C_out, db,
-                                         (flags & SBP_FLAG_ACCUMULATE) != 0, scratch, nullptr,
+                                         (flags & SBP_FLAG_ACCUMULATE) != 0, scratch, kStaticSplits, nullptr,
                                          static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
 }

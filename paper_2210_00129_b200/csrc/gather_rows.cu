@@ -21,6 +21,8 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 __global__ void __launch_bounds__(kGatherThreads)
 gather_rows_kernel(const uint4* __restrict__ X, uint32_t vec_per_row, const int32_t* __restrict__ keep_rows,
                    const int32_t* __restrict__ M_keep_dev, int64_t M_keep_cap, uint4* __restrict__ X_keep) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int64_t total = M_keep_cap * (int64_t)vec_per_row;
     const int64_t valid = M_keep * (int64_t)vec_per_row;
@@ -53,6 +55,8 @@ gather_rows_kernel(const uint4* __restrict__ X, uint32_t vec_per_row, const int3
 __global__ void validate_keep_rows_kernel(const int32_t* __restrict__ keep_rows,
                                           const int32_t* __restrict__ M_keep_dev, int64_t M_keep_cap,
                                           int64_t M, int32_t* status_word) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     if (M_keep_dev != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
         const int64_t raw = (int64_t)__ldg(M_keep_dev);
@@ -78,9 +82,8 @@ cudaError_t launch_gather_rows(const void* X, int64_t row_bytes, const int32_t* 
     int64_t blocks = (total + per_block - 1) / per_block;
     const int64_t max_blocks = (int64_t)kNumSMs * 16;
     if (blocks > max_blocks) blocks = max_blocks;
-    gather_rows_kernel<<<(unsigned)blocks, kGatherThreads, 0, stream>>>(
-        (const uint4*)X, (uint32_t)vec_per_row, keep_rows, M_keep_dev, M_keep_cap, (uint4*)X_keep);
-    return cudaGetLastError();
+    return launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(kGatherThreads), 0, stream,
+                      (const uint4*)X, (uint32_t)vec_per_row, keep_rows, M_keep_dev, M_keep_cap, (uint4*)X_keep);
 }
 
 cudaError_t launch_validate_keep_rows(const int32_t* keep_rows, const int32_t* M_keep_dev,
@@ -89,9 +92,8 @@ cudaError_t launch_validate_keep_rows(const int32_t* keep_rows, const int32_t* M
     int64_t blocks = (M_keep_cap + 255) / 256;
     if (blocks < 1) blocks = 1;
     if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
-    validate_keep_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(keep_rows, M_keep_dev, M_keep_cap, M,
-                                                                   status_word);
-    return cudaGetLastError();
+    return launch_pdl(validate_keep_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
+                      keep_rows, M_keep_dev, M_keep_cap, M, status_word);
 }
 
 }  // namespace sbp

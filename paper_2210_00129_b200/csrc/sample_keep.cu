@@ -56,6 +56,8 @@ sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint
                           uint32_t first_sample, int share_mask,
                           int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
     __shared__ SampShared sh;
+    pdl_launch_dependents();
+    pdl_wait();                 // earlier kernels of the stream may still be reading the index buffers
     const uint32_t b = blockIdx.x;
     const uint32_t gid = share_mask ? 0u : first_sample + b;
     const uint32_t groups = (N + 3u) >> 2;
@@ -173,6 +175,8 @@ sample_keep_grid_kernel(int family, uint32_t H, uint32_t W, uint32_t k0, uint32_
                         uint32_t first_sample, int share_mask,
                         int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
     __shared__ SampShared sh;
+    pdl_launch_dependents();
+    pdl_wait();
     const uint32_t b = blockIdx.x;
     const uint32_t N = H * W;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -229,16 +233,11 @@ cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, 
                                int32_t* keep_rows, int32_t* keep_offsets, cudaStream_t stream) {
     const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
     const dim3 grid((unsigned)B), block(kSampThreads);
-    if (mode == SBP_MASK_RANDOM) {
-        sample_keep_random_kernel<<<grid, block, 0, stream>>>((uint32_t)(H * W), (uint32_t)K, k0, k1, step,
-                                                              first_sample, share_mask ? 1 : 0,
-                                                              keep_rows, keep_offsets);
-    } else {
-        sample_keep_grid_kernel<<<grid, block, 0, stream>>>(grid_family, (uint32_t)H, (uint32_t)W, k0, k1, step,
-                                                            first_sample, share_mask ? 1 : 0,
-                                                            keep_rows, keep_offsets);
-    }
-    return cudaGetLastError();
+    if (mode == SBP_MASK_RANDOM)
+        return launch_pdl(sample_keep_random_kernel, grid, block, 0, stream, (uint32_t)(H * W), (uint32_t)K, k0, k1,
+                          step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
+    return launch_pdl(sample_keep_grid_kernel, grid, block, 0, stream, grid_family, (uint32_t)H, (uint32_t)W, k0, k1,
+                      step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
 }
 
 }  // namespace sbp

@@ -103,7 +103,7 @@ sbp_status sbp_forward_cache(sbp_dtype dt, const void* X, int64_t M, int64_t C, 
 size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                            int64_t C_out) {
     if (M <= 0 || M_keep_cap < 0 || C_in <= 0 || C_out <= 0) return 256;
-    const size_t db_part = align_up(db_workspace_bytes(M_keep_cap, C_out), 256);
+    const size_t db_part = align_up(db_workspace_bytes(dt, M_keep_cap, C_out, kDbMaxSplits), 256);
     size_t dw_part = simt_dw_workspace_bytes(M_keep_cap, C_in, C_out);
     if (dt == SBP_BF16 && tc_shapes_supported(M, M_keep_cap, C_in, C_out)) {
         const size_t t = tc_dw_workspace_bytes(M_keep_cap, C_in, C_out);
@@ -140,7 +140,7 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     const bool accumulate = (flags & SBP_FLAG_ACCUMULATE) != 0;
     float* ws_db = static_cast<float*>(workspace);
     float* ws_dw = need_ws ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
-                                                      align_up(db_workspace_bytes(M_keep_cap, C_out), 256))
+                                                      align_up(db_workspace_bytes(dt, M_keep_cap, C_out, kDbMaxSplits), 256))
                            : nullptr;
 
     if (flags & SBP_FLAG_VALIDATE) {
@@ -149,8 +149,8 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     }
     const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
     if (db != nullptr) {
-        if (launch_db(dt, dY, keep_rows, M_keep_dev, M_keep_cap, C_out, db, accumulate, ws_db, status_word,
-                      stream) != cudaSuccess)
+        if (launch_db(dt, dY, keep_rows, M_keep_dev, M_keep_cap, C_out, db, accumulate, ws_db, kDbMaxSplits,
+                      status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
     }
     if (dW != nullptr) {

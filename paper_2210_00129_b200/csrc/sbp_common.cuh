@@ -16,6 +16,34 @@ __device__ __forceinline__ void report_device_error(int32_t* status_word, int32_
     if (status_word != nullptr) atomicCAS(status_word, 0, code);
 }
 
+// Programmatic dependent launch: every kernel of the library lets its successor start launching
+// right away and itself waits for its predecessor's results before touching global memory, so
+// launch latency and block scheduling overlap with the tail of the previous kernel.
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Number of valid kept rows: the device-side count when given, else the host capacity.
 __device__ __forceinline__ int64_t load_m_keep(const int32_t* M_keep_dev, int64_t M_keep_cap) {
     if (M_keep_dev == nullptr) return M_keep_cap;
@@ -66,10 +94,12 @@ cudaError_t launch_validate_keep_rows(const int32_t* keep_rows, const int32_t* M
                                       cudaStream_t stream);
 
 // partial column sums of the kept rows of dY -> db (deterministic two-pass reduction)
-size_t db_workspace_bytes(int64_t M_keep_cap, int64_t C_out);
+// max_splits bounds the number of row splits (and so the scratch: splits * C_out floats)
+constexpr int kDbMaxSplits = 512;
+size_t db_workspace_bytes(sbp_dtype dt, int64_t M_keep_cap, int64_t C_out, int max_splits);
 cudaError_t launch_db(sbp_dtype dt, const void* dY, const int32_t* keep_rows, const int32_t* M_keep_dev,
                       int64_t M_keep_cap, int64_t C_out, float* db, bool accumulate, float* workspace,
-                      const int32_t* status_word, cudaStream_t stream);
+                      int max_splits, const int32_t* status_word, cudaStream_t stream);
 
 // out[i] = (accumulate ? out[i] : 0) + sum_s partials[s*n + i], summed in ascending s
 cudaError_t launch_reduce_partials(const float* partials, int splits, int64_t n, float* out,

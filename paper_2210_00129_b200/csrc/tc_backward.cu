@@ -128,6 +128,8 @@ tc_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __nv_bfloat16* __r
              __nv_bfloat16* __restrict__ dX, int32_t* status_word) {
     using Cfg = TcCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
+    pdl_launch_dependents();
+    pdl_wait();
     if (status_word != nullptr && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -261,6 +263,8 @@ tc_dw_kernel(const __grid_constant__ CUtensorMap map_x, const __nv_bfloat16* __r
              int accumulate, int32_t* status_word) {
     using Cfg = TcCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
+    pdl_launch_dependents();
+    pdl_wait();
     if (status_word != nullptr && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -455,20 +459,21 @@ sbp_status launch_tc_dx(const void* dY, const void* W, const int32_t* keep_rows,
     CUtensorMap map_w;
     if (!make_map(&map_w, W, C_in, C_out, (uint32_t)bn)) return SBP_ERR_CUDA;
     const dim3 grid((unsigned)((M_keep_cap + kBM - 1) / kBM), (unsigned)((C_in + bn - 1) / bn));
+    cudaError_t launch_err;
     if (bn == 256) {
         static cudaError_t once = allow_smem(tc_dx_kernel<256>, TcCfg<256>::kSmemBytes);
         if (once != cudaSuccess) return SBP_ERR_CUDA;
-        tc_dx_kernel<256><<<grid, kTcThreads, TcCfg<256>::kSmemBytes, stream>>>(
+        launch_err = launch_pdl(tc_dx_kernel<256>, grid, dim3(kTcThreads), TcCfg<256>::kSmemBytes, stream,
             map_w, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M, M_keep_cap, (int)C_in, (int)C_out,
             (__nv_bfloat16*)dX, status_word);
     } else {
         static cudaError_t once = allow_smem(tc_dx_kernel<128>, TcCfg<128>::kSmemBytes);
         if (once != cudaSuccess) return SBP_ERR_CUDA;
-        tc_dx_kernel<128><<<grid, kTcThreads, TcCfg<128>::kSmemBytes, stream>>>(
+        launch_err = launch_pdl(tc_dx_kernel<128>, grid, dim3(kTcThreads), TcCfg<128>::kSmemBytes, stream,
             map_w, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M, M_keep_cap, (int)C_in, (int)C_out,
             (__nv_bfloat16*)dX, status_word);
     }
-    return cudaGetLastError() == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+    return launch_err == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
 }
 
 sbp_status launch_tc_dw(const void* X_keep, const void* dY, const int32_t* keep_rows, const int32_t* M_keep_dev,
@@ -482,20 +487,21 @@ sbp_status launch_tc_dw(const void* X_keep, const void* dY, const int32_t* keep_
     float* out = p.splits > 1 ? workspace : dW;
     const int acc_in_kernel = (p.splits == 1 && accumulate) ? 1 : 0;
     const int64_t split_stride = C_in * C_out;
+    cudaError_t launch_err;
     if (p.bn == 256) {
         static cudaError_t once = allow_smem(tc_dw_kernel<256>, TcCfg<256>::kSmemBytes);
         if (once != cudaSuccess) return SBP_ERR_CUDA;
-        tc_dw_kernel<256><<<grid, kTcThreads, TcCfg<256>::kSmemBytes, stream>>>(
+        launch_err = launch_pdl(tc_dw_kernel<256>, grid, dim3(kTcThreads), TcCfg<256>::kSmemBytes, stream,
             map_x, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M_keep_cap, (int)C_in, (int)C_out, out,
             split_stride, acc_in_kernel, status_word);
     } else {
         static cudaError_t once = allow_smem(tc_dw_kernel<128>, TcCfg<128>::kSmemBytes);
         if (once != cudaSuccess) return SBP_ERR_CUDA;
-        tc_dw_kernel<128><<<grid, kTcThreads, TcCfg<128>::kSmemBytes, stream>>>(
+        launch_err = launch_pdl(tc_dw_kernel<128>, grid, dim3(kTcThreads), TcCfg<128>::kSmemBytes, stream,
             map_x, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M_keep_cap, (int)C_in, (int)C_out, out,
             split_stride, acc_in_kernel, status_word);
     }
-    if (cudaGetLastError() != cudaSuccess) return SBP_ERR_CUDA;
+    if (launch_err != cudaSuccess) return SBP_ERR_CUDA;
     if (p.splits > 1 &&
         launch_reduce_partials(workspace, p.splits, C_in * C_out, dW, accumulate, status_word, stream) != cudaSuccess)
         return SBP_ERR_CUDA;
