@@ -225,7 +225,7 @@ def run_cuda(args, w, name):
     sid = stream.cuda_stream
 
     def step(i, keep_ratio=r, events=None):
-        """One pass of the whole path; `events` (6 per step) bracket its five calls on the launch stream."""
+        """One pass of the whole path; `events` (5 per step) bracket its four calls on the launch stream."""
         s = sets[i % n_sets]
         cnt = s["offs"][B:B + 1]
         capk = B * sbp.sbp_keep_count(mode, H, W_, keep_ratio) if keep_ratio != r else cap_total
@@ -238,22 +238,19 @@ def run_cuda(args, w, name):
         sbp.sbp_linear_backward(code, None, s["dY"], None, s["rows"], cnt, M, capk, C_in, C_out, None, s["db"], None,
                                 0, ws, ws_bytes, status, stream=sid)
         rec(3)
-        sbp.sbp_linear_backward(code, s["Xk"], s["dY"], None, s["rows"], cnt, M, capk, C_in, C_out, s["dW"], None, None,
-                                0, ws, ws_bytes, status, stream=sid)
+        sbp.sbp_linear_backward(code, s["Xk"], s["dY"], s["W"], s["rows"], cnt, M, capk, C_in, C_out, s["dW"], None,
+                                s["dX"], 0, ws, ws_bytes, status, stream=sid)
         rec(4)
-        sbp.sbp_linear_backward(code, None, s["dY"], s["W"], s["rows"], cnt, M, capk, C_in, C_out, None, None, s["dX"],
-                                0, ws, ws_bytes, status, stream=sid)
-        rec(5)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    PHASES = ("sample_keep", "forward_cache", "db", "dW", "dX")
+    PHASES = ("sample_keep", "forward_cache", "db", "dW_dX")
 
     def timed(k_steps, keep_ratio=r):
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(k_steps)]
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(k_steps)]
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
@@ -280,7 +277,7 @@ def run_cuda(args, w, name):
         sampler.start()
         time.sleep(0.3)
     total_ms, phase_ms = timed(args.steps)
-    dx_ms = phase_ms["dX"]
+    gemm_ms = phase_ms["dW_dX"]
     if sampler:
         clocks = sampler.stop()
     assert int(status.item()) == 0, "device status word set during the timed steps"
@@ -293,8 +290,8 @@ def run_cuda(args, w, name):
     for i in range(3):
         step(i, 1.0)
     full_ms, full_phase = timed(bwd_steps, keep_ratio=1.0)
-    bwd_keep = phase_ms["db"] + phase_ms["dW"] + phase_ms["dX"]
-    bwd_full = full_phase["db"] + full_phase["dW"] + full_phase["dX"]
+    bwd_keep = phase_ms["db"] + phase_ms["dW_dX"]
+    bwd_full = full_phase["db"] + full_phase["dW_dX"]
     bwd_speedup = bwd_full / bwd_keep
     saved_frac = (M_keep * C_in * es + 4 * M_keep + 4 * (B + 1)) / (M * C_in * es)
 
@@ -334,20 +331,22 @@ def run_cuda(args, w, name):
     if rank == 0:
         peaks, peak_kind = load_peaks()
         tc_path = dtype == "bf16" and min(C_in, C_out) >= 128 and cap_total >= 64
-        dx_flops = 2.0 * M_keep * C_in * C_out
+        gemm_flops = 4.0 * M_keep * C_in * C_out          # both products of Eq. 5, one fused launch
         if tc_path:
             peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-            roofline = {"kernel": "tc_dx_kernel", "bound": "tensor", "achieved": dx_flops / (dx_ms * 1e-3) / 1e12,
+            roofline = {"kernel": "tc_backward_kernel (dW and dX tiles)", "bound": "tensor",
+                        "achieved": gemm_flops / (gemm_ms * 1e-3) / 1e12,
                         "peak": peak, "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step)",
                         "unit": "TFLOP/s", "traffic": None}
         else:
             # plain-FMA path: 128 fp32 FMA lanes x 148 SMs x 2 FLOP at the maximum SM clock
             peak = 148 * 128 * 2 * 1.965e9 / 1e12
-            roofline = {"kernel": "simt_dx_kernel", "bound": "alu", "achieved": dx_flops / (dx_ms * 1e-3) / 1e12,
+            roofline = {"kernel": "simt_dw_kernel + simt_dx_kernel", "bound": "alu",
+                        "achieved": gemm_flops / (gemm_ms * 1e-3) / 1e12,
                         "peak": peak, "peak_kind": "derived: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz", "unit": "TFLOP/s",
                         "traffic": None}
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        roofline["launch_ms"] = dx_ms
+        roofline["launch_ms"] = gemm_ms
 
         B_s = pick_oracle_sample(w)
         import oracle

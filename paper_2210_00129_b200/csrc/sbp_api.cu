@@ -153,25 +153,18 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
                       status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
     }
-    if (dW != nullptr) {
-        if (tc) {
-            const sbp_status s = launch_tc_dw(X_keep, dY, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW,
-                                              accumulate, ws_dw, status_word, stream);
-            if (s != SBP_OK) return s;
-        } else if (launch_simt_dw(dt, X_keep, dY, keep_rows, M_keep_dev, M_keep_cap, C_in, C_out, dW, accumulate,
-                                  ws_dw, status_word, stream) != cudaSuccess) {
+    if (tc) {
+        // both products in one persistent tensor-core kernel
+        const sbp_status s = launch_tc_backward(X_keep, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW,
+                                                accumulate, dX, ws_dw, status_word, stream);
+        if (s != SBP_OK) return s;
+    } else {
+        if (dW != nullptr && launch_simt_dw(dt, X_keep, dY, keep_rows, M_keep_dev, M_keep_cap, C_in, C_out, dW,
+                                            accumulate, ws_dw, status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
-        }
-    }
-    if (dX != nullptr) {
-        if (tc) {
-            const sbp_status s = launch_tc_dx(dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dX,
-                                              status_word, stream);
-            if (s != SBP_OK) return s;
-        } else if (launch_simt_dx(dt, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dX, status_word,
-                                  stream) != cudaSuccess) {
+        if (dX != nullptr && launch_simt_dx(dt, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dX,
+                                            status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
-        }
     }
     return SBP_OK;
 }
@@ -181,7 +174,8 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
     const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
     int n = (flags & SBP_FLAG_VALIDATE) ? 1 : 0;
     if (want_db) n += 2;                                   // strip partials + fixed-order reduce
-    if (want_dW) n += tc ? tc_dw_kernel_count(M_keep_cap, C_in, C_out) : simt_dw_kernel_count(M_keep_cap, C_in, C_out);
+    if (tc) return n + tc_backward_kernel_count(M_keep_cap, C_in, C_out, want_dW != 0, want_dX != 0);
+    if (want_dW) n += simt_dw_kernel_count(M_keep_cap, C_in, C_out);
     if (want_dX) n += 1;
     return n;
 }

@@ -119,13 +119,11 @@ cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const in
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
-int    tc_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
-sbp_status launch_tc_dw(const void* X_keep, const void* dY, const int32_t* keep_rows,
-                        const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
-                        int64_t C_out, float* dW, bool accumulate, float* workspace,
-                        int32_t* status_word, cudaStream_t stream);
-sbp_status launch_tc_dx(const void* dY, const void* W, const int32_t* keep_rows,
-                        const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
-                        int64_t C_out, void* dX, int32_t* status_word, cudaStream_t stream);
+int    tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx);
+// dW (nullable) and dX (nullable) of one layer in a single persistent kernel (+ the split reduce)
+sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
+                              const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
+                              int64_t C_out, float* dW, bool accumulate, void* dX, float* workspace,
+                              int32_t* status_word, cudaStream_t stream);
 
 }  // namespace sbp

@@ -1,22 +1,23 @@
-// bf16 tensor-core (tcgen05 / TMEM) kernels for the two products of the SBP linear backward (Eq. 5).
+// bf16 tensor-core (tcgen05 / TMEM) kernel for the two products of the SBP linear backward (Eq. 5).
 //
-//   dX kernel:  D[m, i] = sum_j dY[keep_rows[m], j] * W[i, j]            (both operands K-major)
-//               A = kept rows of dY, gathered straight from the full dY; B = W tile (TMA);
-//               the epilogue rounds to bf16, scatters each row to dX[keep_rows[m], :] and
-//               zero-fills the dropped rows between kept rows while the MMAs run.
-//   dW kernel:  D[i, j] = sum_m X_keep[m, i] * dY[keep_rows[m], j]       (both operands MN-major)
-//               A = X_keep tile (TMA), B = gathered dY rows; the reduction over kept rows is
-//               split across blockIdx.z, partials reduced in a fixed order.
+//   dX tiles:  D[m, i] = sum_j dY[keep_rows[m], j] * W[i, j]            (both operands K-major)
+//              A = kept rows of dY, gathered straight from the full dY; B = W tile (TMA);
+//              the epilogue rounds to bf16, scatters each row to dX[keep_rows[m], :] and
+//              zero-fills the dropped rows between kept rows.
+//   dW tiles:  D[i, j] = sum_m X_keep[m, i] * dY[keep_rows[m], j]       (both operands MN-major)
+//              A = X_keep tile (TMA), B = gathered dY rows; long reductions are cut into pieces
+//              whose partial results a second kernel adds in a fixed order.
 //
-// One CTA computes a 128 x BN fp32 accumulator tile held in tensor memory.  Warp roles:
-// warps 0-3 epilogue (TMEM lane quadrant = warp id), warp 4 TMA producer of the dense operand,
-// warp 5 MMA issuer and TMEM owner, warps 6-9 gather producers: they copy the indexed rows of dY
-// with coalesced 16-byte cp.async into the 128-byte-swizzled layout the MMA reads; each thread's
-// copies signal the stage's barrier when they land (cp.async.mbarrier.arrive), so the producers run
-// a full ring ahead of the consumer without ever waiting on their own copies.  (TMA tile::gather4
-// was measured at ~45 ns of issue time per instruction per SM whatever it fetches, far too slow
-// to feed a tile.)  Operand stages are 64 elements deep
-// in the reduction dimension and cycle through a full/empty mbarrier ring.  Every wait is bounded.
+// ONE persistent kernel runs both products: every CTA (one per SM) walks a static, cost-sorted
+// list of 128 x BN output tiles of either kind.  The operand ring (64-deep, 128-byte-swizzled
+// stages behind full/empty mbarriers) never drains between tiles, and the fp32 accumulator in
+// tensor memory is double-buffered, so the epilogue of one tile overlaps the MMAs of the next.
+// Warp roles: warps 0-3 epilogue (TMEM lane quadrant = warp id), warp 4 TMA producer of the dense
+// operand, warp 5 MMA issuer and TMEM owner, warps 6-9 gather producers, which copy the indexed
+// rows of dY with coalesced 16-byte cp.async into the swizzled layout the MMA reads; each thread's
+// copies signal the stage's barrier when they land (cp.async.mbarrier.arrive).  TMA tile::gather4
+// was measured at ~45 ns of issue time per instruction per SM whatever it fetches - far too slow
+// to feed a tile - and is not used.  Every wait is bounded and reports through the status word.
 #include "tc_ptx.cuh"
 
 namespace sbp {
@@ -25,31 +26,102 @@ namespace {
 constexpr int kTcThreads = 320;
 constexpr int kGatherWarp0 = 6;          // first of the four gather warps
 constexpr int kGatherThreads = 128;
-constexpr int kBM = 128;                 // accumulator rows per CTA (= TMEM lanes)
+constexpr int kBM = 128;                 // accumulator rows per tile (= TMEM lanes)
 constexpr int kBK = 64;                  // reduction depth per stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kUmmaK = 16;          // reduction depth of one tcgen05.mma for 16-bit operands
 constexpr uint32_t kRowBytes = 128;      // bytes per swizzled smem row
 constexpr uint32_t kAtomBytes = 1024;    // 8 rows x 128 B: one swizzle atom
 constexpr uint32_t kBlock64Bytes = 64 * kRowBytes;   // a 64-row slab (MN-major operands: one 64-wide block)
-
-template <int BN>
-struct TcCfg {
-    static constexpr uint32_t kABytes = kBM * kRowBytes;          // 16 KB
-    static constexpr uint32_t kBBytes = BN * kRowBytes;           // 16 / 32 KB
-    static constexpr uint32_t kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = (BN == 256) ? 4 : 6;
-    static constexpr uint32_t kCtlBytes = 256;
-    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kCtlBytes + 1024;   // + alignment slack
-};
+constexpr int kStages = 4;
+constexpr uint32_t kABytes = kBM * kRowBytes;        // 16 KB
+constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
+constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
+constexpr uint32_t kAccCols = 256;       // TMEM columns per accumulator buffer (two buffers = all 512)
+constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + 1024;   // ring + control block + alignment slack
 
 struct TcControl {
-    uint64_t full_bar[8];      // 1 arrival with the TMA byte count + one arrival per gather thread
-    uint64_t empty_bar[8];     // 1 arrival: tcgen05.commit of the MMAs that read the stage
-    uint64_t accum_bar;        // 1 arrival: all MMAs of the tile have finished
+    uint64_t full_bar[kStages];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
+    uint64_t empty_bar[kStages];   // 1 arrival: tcgen05.commit of the MMAs that read the stage
+    uint64_t acc_full[2];          // 1 arrival: all MMAs of the tile in this accumulator have finished
+    uint64_t acc_empty[2];         // 4 arrivals: each epilogue warp has read the accumulator out
     uint32_t tmem_slot;
     int abort_flag;
 };
 static_assert(sizeof(TcControl) <= 256, "control block");
+
+struct TcParams {
+    const __nv_bfloat16* dY;
+    const int32_t* keep_rows;
+    const int32_t* M_keep_dev;
+    int64_t M, M_keep_cap;
+    int C_in, C_out;
+    __nv_bfloat16* dX;             // nullptr: no dX tiles
+    float* dW_out;                 // nullptr: no dW tiles; dW itself or the partial buffer
+    int64_t dw_split_stride;       // elements between partial buffers
+    int dw_splits;
+    int dw_accumulate;             // add into dW_out (only with one split)
+    int32_t* status_word;
+};
+
+// ---- the static tile list -------------------------------------------------------------------
+struct Schedule {
+    uint32_t x_tiles, x_ntiles, x_kb;                 // dX: row tiles x column tiles, k-blocks per tile
+    uint32_t w_tiles, w_jtiles, w_kb_total, w_kb_per; // dW: (i tiles x j tiles x splits), k-blocks per piece
+    uint32_t splits;
+    bool w_first;                                     // the costlier kind is handed out first
+    uint32_t total;
+};
+struct Tile {
+    bool is_dw;
+    uint32_t row_tile, col_tile;      // dX: kept-row tile, C_in tile; dW: C_in tile, C_out tile
+    uint32_t split, kb_begin, num_kb;
+};
+
+template <int BNX, int BNW>
+__device__ __forceinline__ Schedule make_schedule(const TcParams& p, int64_t M_keep) {
+    Schedule s;
+    s.x_ntiles = (uint32_t)((p.C_in + BNX - 1) / BNX);
+    s.x_tiles = (p.dX != nullptr) ? (uint32_t)((M_keep + kBM - 1) / kBM) * s.x_ntiles : 0u;
+    s.x_kb = (uint32_t)((p.C_out + kBK - 1) / kBK);
+    s.splits = (uint32_t)p.dw_splits;
+    s.w_jtiles = (uint32_t)((p.C_out + BNW - 1) / BNW);
+    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_in + kBM - 1) / kBM) * s.w_jtiles * s.splits : 0u;
+    s.w_kb_total = (uint32_t)((M_keep + kBK - 1) / kBK);
+    s.w_kb_per = (s.w_kb_total + s.splits - 1) / s.splits;
+    s.w_first = s.w_kb_per >= s.x_kb;
+    s.total = s.x_tiles + s.w_tiles;
+    return s;
+}
+
+__device__ __forceinline__ Tile decode_tile(const Schedule& s, uint32_t q) {
+    Tile t;
+    const uint32_t first = s.w_first ? s.w_tiles : s.x_tiles;
+    t.is_dw = (q < first) == s.w_first;
+    const uint32_t idx = (q < first) ? q : q - first;
+    if (t.is_dw) {
+        t.split = idx % s.splits;
+        const uint32_t ij = idx / s.splits;
+        t.row_tile = ij / s.w_jtiles;
+        t.col_tile = ij % s.w_jtiles;
+        t.kb_begin = s.w_kb_per * t.split;
+        const uint32_t end = (t.kb_begin + s.w_kb_per < s.w_kb_total) ? t.kb_begin + s.w_kb_per : s.w_kb_total;
+        t.num_kb = (end > t.kb_begin) ? end - t.kb_begin : 0u;
+    } else {
+        t.split = 0;
+        t.row_tile = idx / s.x_ntiles;
+        t.col_tile = idx % s.x_ntiles;
+        t.kb_begin = 0;
+        t.num_kb = s.x_kb;
+    }
+    return t;
+}
+
+// CTA b takes list positions b, 2G-1-b, 2G+b, 4G-1-b, ...: with the list sorted by cost this
+// evens out the load without any run-time counter.
+__device__ __forceinline__ uint32_t list_position(uint32_t pass) {
+    const uint32_t G = gridDim.x, b = blockIdx.x;
+    return pass * G + ((pass & 1u) ? (G - 1u - b) : b);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -61,330 +133,300 @@ __device__ __forceinline__ uint32_t swizzled(uint32_t row, uint32_t chunk) {
     return row * kRowBytes + ((chunk ^ (row & 7u)) << 4);
 }
 
-template <int BN>
-__device__ __forceinline__ void init_pipeline(TcControl* ctl) {
+// ---------------------------------------------------------------------------------------------
+template <int BNX, int BNW>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                   const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
+    const uint32_t ring = (raw_addr + 1023u) & ~1023u;              // swizzle atoms need 1024-byte alignment
+    TcControl* ctl = reinterpret_cast<TcControl*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes);
+
+    // ---- set-up that needs nothing from earlier kernels: overlaps their tail ----
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TcCfg<BN>::kStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_bar[s]), 1 + kGatherThreads);
             ptx::mbar_init(ptx::smem_addr(&ctl->empty_bar[s]), 1);
         }
-        ptx::mbar_init(ptx::smem_addr(&ctl->accum_bar), 1);
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[a]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 4);
+        }
         ctl->abort_flag = 0;
         ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&map_w);
+        ptx::prefetch_tensormap(&map_x);
     }
-    if ((threadIdx.x >> 5) == 5) ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), BN);
+    if (warp == 5) ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
-}
-
-// TMA thread after a failed wait: let the copies it already issued land before shared memory goes away
-template <int STAGES>
-__device__ __forceinline__ void drain_tma(TcControl* ctl, uint32_t issued) {
-    for (uint32_t it = (issued > (uint32_t)STAGES ? issued - STAGES : 0u); it < issued; ++it) {
-        const uint32_t bar = ptx::smem_addr(&ctl->full_bar[it % STAGES]);
-        for (int spin = 0; spin < (1 << 14); ++spin)
-            if (ptx::mbar_try_wait(bar, (it / STAGES) & 1u)) break;
-    }
-}
-
-// The MMA issuer's loop is the same for both kernels up to the operand descriptors.
-template <int BN, bool MN_MAJOR>
-__device__ __forceinline__ void mma_loop(TcControl* ctl, uint32_t tiles, uint32_t tmem_base, uint32_t num_kb,
-                                         volatile int* abort_flag, int32_t* status_word) {
-    using Cfg = TcCfg<BN>;
-    constexpr uint32_t idesc = ptx::umma_idesc_bf16(kBM, BN, MN_MAJOR, MN_MAJOR);
-    // K-major: a 16-deep slice is 32 bytes along the swizzled row; 8-row groups sit 1024 B apart.
-    // MN-major: a 16-deep slice is 16 rows (two atoms); 64-wide blocks of the MN extent sit 8 KB apart.
-    constexpr uint32_t k_step = MN_MAJOR ? kUmmaK * kRowBytes : kUmmaK * 2;
-    constexpr uint32_t lbo = MN_MAJOR ? kBlock64Bytes : 16;
-    bool ok = true;
-    for (uint32_t it = 0; it < num_kb; ++it) {
-        const int s = it % Cfg::kStages;
-        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / Cfg::kStages) & 1u, abort_flag, status_word);
-        if (!ok) break;
-        ptx::tc_fence_after_sync();
-        ptx::fence_async_proxy();        // the gathered operand was written by cp.async (generic proxy)
-        const uint32_t a_addr = tiles + s * Cfg::kStageBytes, b_addr = a_addr + Cfg::kABytes;
-#pragma unroll
-        for (uint32_t k = 0; k < kBK / kUmmaK; ++k) {
-            const uint64_t da = ptx::umma_desc_sw128(a_addr + k * k_step, lbo, kAtomBytes);
-            const uint64_t db = ptx::umma_desc_sw128(b_addr + k * k_step, lbo, kAtomBytes);
-            ptx::umma_bf16(tmem_base, da, db, idesc, (it | k) != 0u);
-        }
-        ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));     // stage reusable once these MMAs retire
-    }
-    if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->accum_bar));
-}
-
-// --------------------------------------------------------------------------------------------
-// dX = scatter(dY_keep * W^T) with zero fill
-// --------------------------------------------------------------------------------------------
-template <int BN>
-__global__ void __launch_bounds__(kTcThreads, 1)
-tc_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __nv_bfloat16* __restrict__ dY,
-             const int32_t* __restrict__ keep_rows, const int32_t* __restrict__ M_keep_dev,
-             int64_t M, int64_t M_keep_cap, int C_in, int C_out,
-             __nv_bfloat16* __restrict__ dX, int32_t* status_word) {
-    using Cfg = TcCfg<BN>;
-    extern __shared__ uint8_t smem_raw[];
-    pdl_launch_dependents();
-    pdl_wait();
-    if (status_word != nullptr && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
-    const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * kBM;
-    const int n0 = blockIdx.y * BN;
-    const int strip_cols = (C_in - n0 < BN) ? C_in - n0 : BN;       // multiple of 8
-    const int strip_vecs = strip_cols >> 3;                          // 16-byte vectors per row of the strip
-
-    if (M_keep == 0) {                   // nothing kept: the first row tile clears its column strip
-        if (blockIdx.x == 0)
-            for (int64_t t = threadIdx.x; t < M * strip_vecs; t += kTcThreads)
-                ptx::st_global_v4(dX + (t / strip_vecs) * C_in + n0 + (t % strip_vecs) * 8, 0u, 0u, 0u, 0u);
-        return;
-    }
-    if (m0 >= M_keep) return;
-
-    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
-    const uint32_t tiles = (raw_addr + 1023u) & ~1023u;             // swizzle atoms need 1024-byte alignment
-    TcControl* ctl = reinterpret_cast<TcControl*>(smem_raw + (tiles - raw_addr) + Cfg::kStages * Cfg::kStageBytes);
-    const uint32_t num_kb = (uint32_t)((C_out + kBK - 1) / kBK);
-    init_pipeline<BN>(ctl);
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctl->tmem_slot);
     volatile int* abort_flag = &ctl->abort_flag;
+    int32_t* status_word = p.status_word;
 
-    if (warp == 4) {
-        // ---------------- TMA producer: the W tile of every stage ----------------
+    pdl_wait();                                                      // from here on global memory is read
+    const bool skip_all = status_word != nullptr && *reinterpret_cast<volatile int32_t*>(status_word) != 0;
+    const int64_t M_keep = load_m_keep(p.M_keep_dev, p.M_keep_cap);
+    const Schedule sched = make_schedule<BNX, BNW>(p, M_keep);
+    const int C_in = p.C_in, C_out = p.C_out;
+
+    if (skip_all) {
+        // an earlier check failed: leave every output untouched
+    } else if (warp == 4) {
+        // ---------------- TMA producer: the dense operand of every stage ----------------
         if (lane == 0) {
-            ptx::prefetch_tensormap(&map_w);
-            uint32_t it = 0;
-            for (; it < num_kb; ++it) {
-                const int s = it % Cfg::kStages;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / Cfg::kStages) & 1u) ^ 1u, abort_flag, status_word))
-                    break;
-                const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
-                ptx::mbar_arrive_expect_tx(full, Cfg::kBBytes);
-                ptx::tma_load_2d(tiles + s * Cfg::kStageBytes + Cfg::kABytes, &map_w, (int)(it * kBK), n0, full);
+            uint32_t it = 0;                                         // stage uses so far, over all tiles
+            bool ok = true;
+            for (uint32_t pass = 0; ok; ++pass) {
+                const uint32_t q = list_position(pass);
+                if (q >= sched.total) break;
+                const Tile t = decode_tile(sched, q);
+                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
+                    const int s = it % kStages;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                    if (!ok) break;
+                    const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
+                    const uint32_t a_dst = ring + s * kStageBytes;
+                    if (t.is_dw) {                                   // X_keep tile: two 64-wide blocks of 64 kept rows
+                        const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.row_tile * kBM);
+                        ptx::mbar_arrive_expect_tx(full, kABytes);
+                        ptx::tma_load_2d(a_dst, &map_x, i0, row0, full);
+                        ptx::tma_load_2d(a_dst + kBlock64Bytes, &map_x, i0 + 64, row0, full);
+                    } else {                                         // W tile: BNX rows x 64 columns
+                        ptx::mbar_arrive_expect_tx(full, BNX * kRowBytes);
+                        ptx::tma_load_2d(a_dst + kABytes, &map_w, (int)(k * kBK), (int)(t.col_tile * BNX), full);
+                    }
+                }
             }
-            if (it < num_kb) drain_tma<Cfg::kStages>(ctl, it);
+            if (!ok) {   // let the copies already issued land before shared memory goes away
+                for (uint32_t j = (it > (uint32_t)kStages ? it - kStages : 0u); j < it; ++j) {
+                    const uint32_t bar = ptx::smem_addr(&ctl->full_bar[j % kStages]);
+                    for (int spin = 0; spin < (1 << 14); ++spin)
+                        if (ptx::mbar_try_wait(bar, (j / kStages) & 1u)) break;
+                }
+            }
         }
         __syncwarp();
     } else if (warp == 5) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) mma_loop<BN, false>(ctl, tiles, tmem_base, num_kb, abort_flag, status_word);
+        if (lane == 0) {
+            uint32_t it = 0, used = 0;                               // stage uses, accumulator uses
+            bool ok = true;
+            for (uint32_t pass = 0; ok; ++pass) {
+                const uint32_t q = list_position(pass);
+                if (q >= sched.total) break;
+                const Tile t = decode_tile(sched, q);
+                if (t.num_kb == 0) continue;
+                const uint32_t acc = used & 1u;
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[acc]), ((used >> 1) & 1u) ^ 1u, abort_flag, status_word);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                // K-major (dX): a 16-deep slice is 32 bytes along the swizzled row, 8-row groups 1024 B apart.
+                // MN-major (dW): a 16-deep slice is 16 rows (two atoms); 64-wide blocks of the MN extent 8 KB apart.
+                const uint32_t idesc = t.is_dw ? ptx::umma_idesc_bf16(kBM, BNW, true, true)
+                                               : ptx::umma_idesc_bf16(kBM, BNX, false, false);
+                const uint32_t k_step = t.is_dw ? kUmmaK * kRowBytes : kUmmaK * 2;
+                const uint32_t lbo = t.is_dw ? kBlock64Bytes : 16;
+                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
+                    const int s = it % kStages;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / kStages) & 1u, abort_flag, status_word);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    ptx::fence_async_proxy();        // the gathered operand was written by cp.async (generic proxy)
+                    const uint32_t a_addr = ring + s * kStageBytes, b_addr = a_addr + kABytes;
+#pragma unroll
+                    for (uint32_t u = 0; u < kBK / kUmmaK; ++u) {
+                        const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, kAtomBytes);
+                        const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, kAtomBytes);
+                        ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
+                    }
+                    ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));      // stage reusable once these MMAs retire
+                }
+                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
+                ++used;
+            }
+        }
         __syncwarp();
     } else if (warp >= kGatherWarp0) {
-        // ---------------- gather producers: 128 kept rows x 128 bytes of dY per stage ----------------
-        // one instruction of a warp moves 4 rows x 128 B; a warp owns 32 rows of the tile
+        // ---------------- gather producers ----------------
         const int gw = warp - kGatherWarp0;
-        const uint32_t chunk = lane & 7;
-        const __nv_bfloat16* src[8];
-        uint32_t dst[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t row = gw * 32 + i * 4 + (lane >> 3);
-            int64_t m = m0 + row;
-            if (m >= M_keep) m = M_keep - 1;                          // padding rows of the last tile: never stored
-            src[i] = dY + (int64_t)__ldg(keep_rows + m) * C_out + chunk * 8;
-            dst[i] = swizzled(row, chunk);
-        }
-        for (uint32_t it = 0; it < num_kb; ++it) {
-            const int s = it % Cfg::kStages;
-            if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / Cfg::kStages) & 1u) ^ 1u, abort_flag, status_word))
-                break;
-            const uint32_t a_dst = tiles + s * Cfg::kStageBytes;
-            const int col = (int)(it * kBK + chunk * 8);
-            const uint32_t bytes = (col < C_out) ? 16u : 0u;      // columns past C_out read as zero
-            const int off = (col < C_out) ? (int)(it * kBK) : 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ptx::cp_async_16(a_dst + dst[i], src[i] + off, bytes);
-            // the stage's barrier gets this thread's arrival when the copies above have landed
-            ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
-        }
-        ptx::cp_async_wait_all();
-    } else {
-        // ---------------- epilogue warps: zero fill first, then scatter the accumulator rows ----------------
-        const int64_t m = m0 + warp * 32 + lane;
-        const bool valid = m < M_keep;
-        const int64_t cur = valid ? (int64_t)__ldg(keep_rows + m) : -1;
-        const int64_t prev = (valid && m > 0) ? (int64_t)__ldg(keep_rows + m - 1) : -1;
-        for (int t = 0; t < 32; ++t) {
-            if (!__shfl_sync(0xffffffffu, valid ? 1 : 0, t)) break;
-            const int64_t c = __shfl_sync(0xffffffffu, cur, t);
-            int64_t g = __shfl_sync(0xffffffffu, prev, t) + 1;
-            for (; g < c; ++g)
-                for (int v = lane; v < strip_vecs; v += 32)
-                    ptx::st_global_v4(dX + g * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
-            if (m0 + warp * 32 + t == M_keep - 1)                   // after the very last kept row
-                for (g = c + 1; g < M; ++g)
-                    for (int v = lane; v < strip_vecs; v += 32)
-                        ptx::st_global_v4(dX + g * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
-        }
+        uint32_t it = 0;
         bool ok = true;
-        if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->accum_bar), 0u, abort_flag, status_word);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (ok) {
-            ptx::tc_fence_after_sync();
-            __nv_bfloat16* out_row = dX + (valid ? cur : 0) * C_in + n0;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                float v[32];
-                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                ptx::tmem_ld_wait();
-                if (valid) {
+        for (uint32_t pass = 0; ok; ++pass) {
+            const uint32_t q = list_position(pass);
+            if (q >= sched.total) break;
+            const Tile t = decode_tile(sched, q);
+            if (!t.is_dw) {
+                // dX tile: 128 kept rows x 128 bytes per stage; one warp instruction moves 4 rows x 128 B
+                const uint32_t chunk = lane & 7;
+                const int64_t m0 = (int64_t)t.row_tile * kBM;
+                const __nv_bfloat16* src[8];
+                uint32_t dst[8];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (c0 + q * 8 < strip_cols)
-                            ptx::st_global_v4(out_row + c0 + q * 8,
-                                              pack_bf16(v[q * 8 + 0], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
-                                              pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t row = gw * 32 + i * 4 + (lane >> 3);
+                    int64_t m = m0 + row;
+                    if (m >= M_keep) m = M_keep - 1;                  // padding rows of the last tile: never stored
+                    src[i] = p.dY + (int64_t)__ldg(p.keep_rows + m) * C_out + chunk * 8;
+                    dst[i] = swizzled(row, chunk);
+                }
+                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
+                    const int s = it % kStages;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                    ok = __all_sync(0xffffffffu, ok);                 // the warp leaves the loop together
+                    if (!ok) break;
+                    const uint32_t a_dst = ring + s * kStageBytes;
+                    const int col = (int)(k * kBK + chunk * 8);
+                    const uint32_t bytes = (col < C_out) ? 16u : 0u;  // columns past C_out read as zero
+                    const int off = (col < C_out) ? (int)(k * kBK) : 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) ptx::cp_async_16(a_dst + dst[i], src[i] + off, bytes);
+                    // the stage's barrier gets this thread's arrival when the copies above have landed
+                    ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
+                }
+            } else {
+                // dW tile: 64 kept rows x BNW columns per stage; a warp owns 16 rows, one instruction moves 512 B
+                constexpr int kChunksPerRow = BNW / 8;               // 16-byte chunks of one row of the tile
+                constexpr int kRowsPerInstr = 32 / kChunksPerRow;    // 1 (BNW = 256) or 2 (BNW = 128)
+                constexpr int kInstr = 16 / kRowsPerInstr;
+                const uint32_t c = lane % kChunksPerRow;             // chunk within the row
+                const uint32_t sub = lane / kChunksPerRow;           // which of the rows of this instruction
+                const int col = (int)(t.col_tile * BNW) + (int)c * 8;
+                const bool col_ok = col < C_out;                     // columns past C_out read as zero
+                const __nv_bfloat16* col_ptr = p.dY + (col_ok ? col : 0);
+                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
+                    const int s = it % kStages;
+                    // row ids of this warp's 16 rows: lanes 0..15 fetch one each
+                    const int64_t mrow = (int64_t)(t.kb_begin + k) * kBK + gw * 16 + (lane & 15);
+                    const int my_row = (mrow < M_keep) ? __ldg(p.keep_rows + mrow) : -1;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    const uint32_t b_dst = ring + s * kStageBytes + kABytes;
+#pragma unroll
+                    for (int i = 0; i < kInstr; ++i) {
+                        const uint32_t r = gw * 16 + i * kRowsPerInstr + sub;         // row within the 64-row stage
+                        const int g = __shfl_sync(0xffffffffu, my_row, i * kRowsPerInstr + (int)sub);
+                        const bool live = g >= 0 && col_ok;                           // rows past M_keep read as zero
+                        ptx::cp_async_16(b_dst + (c >> 3) * kBlock64Bytes + swizzled(r, c & 7u),
+                                         col_ptr + (live ? (int64_t)g * C_out : 0), live ? 16u : 0u);
                     }
+                    ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
                 }
             }
         }
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 5) {
-        ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, BN);
-    }
-}
-
-// --------------------------------------------------------------------------------------------
-// dW = X_keep^T * dY_keep, split over the kept rows
-// --------------------------------------------------------------------------------------------
-template <int BN>
-__global__ void __launch_bounds__(kTcThreads, 1)
-tc_dw_kernel(const __grid_constant__ CUtensorMap map_x, const __nv_bfloat16* __restrict__ dY,
-             const int32_t* __restrict__ keep_rows, const int32_t* __restrict__ M_keep_dev,
-             int64_t M_keep_cap, int C_in, int C_out, float* __restrict__ out, int64_t split_stride,
-             int accumulate, int32_t* status_word) {
-    using Cfg = TcCfg<BN>;
-    extern __shared__ uint8_t smem_raw[];
-    pdl_launch_dependents();
-    pdl_wait();
-    if (status_word != nullptr && *reinterpret_cast<volatile int32_t*>(status_word) != 0) return;
-    const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int j0 = blockIdx.x * BN, i0 = blockIdx.y * kBM;
-    const uint32_t total_kb = (uint32_t)((M_keep + kBK - 1) / kBK);
-    const uint32_t kb_per = (total_kb + gridDim.z - 1) / gridDim.z;
-    const uint32_t kb_begin = kb_per * blockIdx.z;
-    const uint32_t kb_end = (kb_begin + kb_per < total_kb) ? kb_begin + kb_per : total_kb;
-    const uint32_t num_kb = (kb_end > kb_begin) ? kb_end - kb_begin : 0u;
-    float* dst_base = out + (int64_t)blockIdx.z * split_stride;
-
-    if (num_kb == 0) {                   // this split has no kept rows: its partial is zero
-        if (!accumulate)
-            for (int t = threadIdx.x; t < kBM * (BN / 4); t += kTcThreads) {
-                const int i = i0 + t / (BN / 4), j = j0 + (t % (BN / 4)) * 4;
-                if (i < C_in && j < C_out) ptx::st_global_v4(dst_base + (int64_t)i * C_out + j, 0u, 0u, 0u, 0u);
-            }
-        return;
-    }
-
-    const uint32_t raw_addr = ptx::smem_addr(smem_raw);
-    const uint32_t tiles = (raw_addr + 1023u) & ~1023u;
-    TcControl* ctl = reinterpret_cast<TcControl*>(smem_raw + (tiles - raw_addr) + Cfg::kStages * Cfg::kStageBytes);
-    init_pipeline<BN>(ctl);
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctl->tmem_slot);
-    volatile int* abort_flag = &ctl->abort_flag;
-
-    if (warp == 4) {
-        // ---------------- TMA producer: the X_keep tile (two 64-wide blocks) of every stage ----------------
-        if (lane == 0) {
-            ptx::prefetch_tensormap(&map_x);
-            uint32_t it = 0;
-            for (; it < num_kb; ++it) {
-                const int s = it % Cfg::kStages;
-                if (!ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / Cfg::kStages) & 1u) ^ 1u, abort_flag, status_word))
-                    break;
-                const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
-                const uint32_t a_dst = tiles + s * Cfg::kStageBytes;
-                const int row0 = (int)((kb_begin + it) * kBK);
-                ptx::mbar_arrive_expect_tx(full, Cfg::kABytes);
-                ptx::tma_load_2d(a_dst, &map_x, i0, row0, full);
-                ptx::tma_load_2d(a_dst + kBlock64Bytes, &map_x, i0 + 64, row0, full);
-            }
-            if (it < num_kb) drain_tma<Cfg::kStages>(ctl, it);
-        }
-        __syncwarp();
-    } else if (warp == 5) {
-        // ---------------- MMA issuer: both operands MN-major ----------------
-        if (lane == 0) mma_loop<BN, true>(ctl, tiles, tmem_base, num_kb, abort_flag, status_word);
-        __syncwarp();
-    } else if (warp >= kGatherWarp0) {
-        // ---------------- gather producers: 64 kept rows x BN columns of dY per stage ----------------
-        // a warp owns 16 rows of each stage; one instruction moves 512 contiguous bytes
-        constexpr int kChunksPerRow = BN / 8;                   // 16-byte chunks of one row of the tile
-        constexpr int kRowsPerInstr = 32 / kChunksPerRow;       // 1 (BN = 256) or 2 (BN = 128)
-        constexpr int kInstr = 16 / kRowsPerInstr;
-        const int gw = warp - kGatherWarp0;
-        const uint32_t c = lane % kChunksPerRow;                // chunk within the row
-        const uint32_t sub = lane / kChunksPerRow;              // which of the rows of this instruction
-        const int col = j0 + (int)c * 8;
-        const bool col_ok = col < C_out;                        // columns past C_out read as zero
-        const __nv_bfloat16* col_ptr = dY + (col_ok ? col : 0);
-        for (uint32_t it = 0; it < num_kb; ++it) {
-            const int s = it % Cfg::kStages;
-            // row ids of this warp's 16 rows: lanes 0..15 fetch one each
-            const int64_t mrow = (int64_t)(kb_begin + it) * kBK + gw * 16 + (lane & 15);
-            const int my_row = (mrow < M_keep) ? __ldg(keep_rows + mrow) : -1;
-            bool ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / Cfg::kStages) & 1u) ^ 1u, abort_flag, status_word);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const uint32_t b_dst = tiles + s * Cfg::kStageBytes + Cfg::kABytes;
-#pragma unroll
-            for (int i = 0; i < kInstr; ++i) {
-                const uint32_t r = gw * 16 + i * kRowsPerInstr + sub;             // row within the 64-row stage
-                const int g = __shfl_sync(0xffffffffu, my_row, i * kRowsPerInstr + (int)sub);
-                const bool live = g >= 0 && col_ok;                               // rows past M_keep read as zero
-                ptx::cp_async_16(b_dst + (c >> 3) * kBlock64Bytes + swizzled(r, c & 7u),
-                                 col_ptr + (live ? (int64_t)g * C_out : 0), live ? 16u : 0u);
-            }
-            ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
-        }
         ptx::cp_async_wait_all();
     } else {
-        // ---------------- epilogue: fp32 accumulator rows to dW (or to this split's partial) ----------------
+        // ---------------- epilogue warps ----------------
+        if (M_keep == 0 && p.dX != nullptr) {                        // nothing kept: dX is all zeros
+            const int64_t vecs = p.M * (int64_t)(C_in / 8);
+            for (int64_t v = (int64_t)blockIdx.x * 128 + threadIdx.x; v < vecs; v += (int64_t)gridDim.x * 128)
+                ptx::st_global_v4(p.dX + v * 8, 0u, 0u, 0u, 0u);
+        }
+        uint32_t used = 0;
         bool ok = true;
-        if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->accum_bar), 0u, abort_flag, status_word);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (ok) {
-            ptx::tc_fence_after_sync();
-            const int i = i0 + warp * 32 + lane;
-            float* out_row = dst_base + (int64_t)i * C_out + j0;
+        for (uint32_t pass = 0; ok; ++pass) {
+            const uint32_t q = list_position(pass);
+            if (q >= sched.total) break;
+            const Tile t = decode_tile(sched, q);
+            const uint32_t acc = used & 1u;
+            const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
+            if (!t.is_dw) {
+                // ---- dX tile: zero the dropped rows around this warp's kept rows, then scatter ----
+                const int n0 = (int)(t.col_tile * BNX);
+                const int strip_cols = (C_in - n0 < BNX) ? C_in - n0 : BNX;   // multiple of 8
+                const int strip_vecs = strip_cols >> 3;
+                const int64_t m0 = (int64_t)t.row_tile * kBM;
+                const int64_t m = m0 + warp * 32 + lane;
+                const bool valid = m < M_keep;
+                const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
+                const int64_t prev = (valid && m > 0) ? (int64_t)__ldg(p.keep_rows + m - 1) : -1;
+                for (int r = 0; r < 32; ++r) {
+                    if (!__shfl_sync(0xffffffffu, valid ? 1 : 0, r)) break;
+                    const int64_t c = __shfl_sync(0xffffffffu, cur, r);
+                    int64_t g = __shfl_sync(0xffffffffu, prev, r) + 1;
+                    for (; g < c; ++g)
+                        for (int v = lane; v < strip_vecs; v += 32)
+                            ptx::st_global_v4(p.dX + g * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
+                    if (m0 + warp * 32 + r == M_keep - 1)            // after the very last kept row
+                        for (g = c + 1; g < p.M; ++g)
+                            for (int v = lane; v < strip_vecs; v += 32)
+                                ptx::st_global_v4(p.dX + g * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
+                }
+                if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                __nv_bfloat16* out_row = p.dX + (valid ? cur : 0) * C_in + n0;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                float v[32];
-                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                ptx::tmem_ld_wait();
-                if (i < C_in) {
+                for (int c0 = 0; c0 < BNX; c0 += 32) {
+                    float v[32];
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
+                    ptx::tmem_ld_wait();
+                    if (valid) {
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (j0 + c0 + q * 4 < C_out) {
-                            float4 w = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
-                            float4* p = reinterpret_cast<float4*>(out_row + c0 + q * 4);
-                            if (accumulate) { const float4 o = *p; w.x += o.x; w.y += o.y; w.z += o.z; w.w += o.w; }
-                            *p = w;
+                        for (int qd = 0; qd < 4; ++qd) {
+                            if (c0 + qd * 8 < strip_cols)
+                                ptx::st_global_v4(out_row + c0 + qd * 8,
+                                                  pack_bf16(v[qd * 8 + 0], v[qd * 8 + 1]), pack_bf16(v[qd * 8 + 2], v[qd * 8 + 3]),
+                                                  pack_bf16(v[qd * 8 + 4], v[qd * 8 + 5]), pack_bf16(v[qd * 8 + 6], v[qd * 8 + 7]));
+                        }
+                    }
+                }
+            } else {
+                // ---- dW tile: fp32 accumulator rows to dW (or to this piece's partial buffer) ----
+                const int i = (int)(t.row_tile * kBM) + warp * 32 + lane;
+                const int j0 = (int)(t.col_tile * BNW);
+                float* out_row = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i * C_out + j0;
+                if (t.num_kb == 0) {                                 // a piece without kept rows contributes zero
+                    if (!p.dw_accumulate && i < C_in)
+                        for (int c0 = 0; c0 < BNW; c0 += 4)
+                            if (j0 + c0 < C_out) ptx::st_global_v4(out_row + c0, 0u, 0u, 0u, 0u);
+                    continue;
+                }
+                if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+#pragma unroll 1
+                for (int c0 = 0; c0 < BNW; c0 += 32) {
+                    float v[32];
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
+                    ptx::tmem_ld_wait();
+                    if (i < C_in) {
+#pragma unroll
+                        for (int qd = 0; qd < 8; ++qd) {
+                            if (j0 + c0 + qd * 4 < C_out) {
+                                float4 w = make_float4(v[qd * 4], v[qd * 4 + 1], v[qd * 4 + 2], v[qd * 4 + 3]);
+                                float4* dst = reinterpret_cast<float4*>(out_row + c0 + qd * 4);
+                                if (p.dw_accumulate) { const float4 o = *dst; w.x += o.x; w.y += o.y; w.z += o.z; w.w += o.w; }
+                                *dst = w;
+                            }
                         }
                     }
                 }
             }
+            // this warp is done with the accumulator: hand it back to the MMA issuer
+            ptx::tc_fence_before_sync();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
+            ++used;
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 5) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, BN);
+        ptx::tmem_dealloc(tmem_base, 2 * kAccCols);
     }
 }
 
 // --------------------------------------------------------------------------------------------
-// host side: tensor maps and launches
+// host side: tensor maps, the split plan and the launch
 // --------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -415,25 +457,44 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename K>
-cudaError_t allow_smem(K kernel, uint32_t bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+struct Plan {
+    int bnx, bnw;          // accumulator width of dX / dW tiles
+    int splits;            // pieces each dW tile's reduction over kept rows is cut into
+    int64_t tiles;         // upper bound of the tile count (from the capacity)
+};
+
+Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
+    Plan pl;
+    pl.bnx = (C_in >= 256) ? 256 : 128;
+    pl.bnw = (C_out >= 256) ? 256 : 128;
+    const int64_t x_tiles = want_dx ? ((M_keep_cap + kBM - 1) / kBM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
+    const int64_t x_kb = (C_out + kBK - 1) / kBK;
+    const int64_t w_tiles = want_dw ? ((C_in + kBM - 1) / kBM) * ((C_out + pl.bnw - 1) / pl.bnw) : 0;
+    const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
+    // Cut the dW reductions so that one piece is no longer than an even share of all the work
+    // (in k-block units; a BN=128 tile's unit is cheaper, which only makes the cut finer).
+    pl.splits = 1;
+    if (want_dw) {
+        const int64_t units = x_tiles * x_kb + w_tiles * w_kb;
+        int64_t share = (units + kNumSMs - 1) / kNumSMs;
+        if (share < 16) share = 16;
+        int64_t s = (w_kb + share - 1) / share;
+        if (s > 64) s = 64;
+        if (s > w_kb) s = w_kb;
+        if (s < 1) s = 1;
+        pl.splits = (int)s;
+    }
+    pl.tiles = x_tiles + w_tiles * pl.splits;
+    return pl;
 }
 
-struct DwPlan { int bn; int splits; };
-
-DwPlan plan_dw(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
-    DwPlan p;
-    p.bn = (C_out >= 256) ? 256 : 128;
-    const int64_t tiles = ((C_in + kBM - 1) / kBM) * ((C_out + p.bn - 1) / p.bn);
-    const int64_t kb = (M_keep_cap + kBK - 1) / kBK;
-    // fill the 148 SMs once: as many splits as fit in one wave, each at least 4 stages deep
-    int64_t s = kNumSMs / tiles;
-    if (s > kb / 4) s = kb / 4;
-    if (s > 32) s = 32;
-    if (s < 1) s = 1;
-    p.splits = (int)s;
-    return p;
+template <int BNX, int BNW>
+cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
+                         const TcParams& prm) {
+    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (once != cudaSuccess) return once;
+    return launch_pdl(tc_backward_kernel<BNX, BNW>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x, prm);
 }
 
 }  // namespace
@@ -444,66 +505,57 @@ bool tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_
 }
 
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
-    const DwPlan p = plan_dw(M_keep_cap, C_in, C_out);
-    return p.splits > 1 ? (size_t)p.splits * (size_t)C_in * (size_t)C_out * sizeof(float) : 0;
+    // the split count depends on which products a call asks for; size for the larger of the two cases
+    const int s1 = make_plan(M_keep_cap, C_in, C_out, true, true).splits;
+    const int s2 = make_plan(M_keep_cap, C_in, C_out, true, false).splits;
+    const int s = s1 > s2 ? s1 : s2;
+    return s > 1 ? (size_t)s * (size_t)C_in * (size_t)C_out * sizeof(float) : 0;
 }
 
-int tc_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
-    return plan_dw(M_keep_cap, C_in, C_out).splits > 1 ? 2 : 1;
+int tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
+    if (!want_dw && !want_dx) return 0;
+    return 1 + ((want_dw && make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx).splits > 1) ? 1 : 0);
 }
 
-sbp_status launch_tc_dx(const void* dY, const void* W, const int32_t* keep_rows, const int32_t* M_keep_dev,
-                        int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out, void* dX,
-                        int32_t* status_word, cudaStream_t stream) {
-    const int bn = (C_in >= 256) ? 256 : 128;
-    CUtensorMap map_w;
-    if (!make_map(&map_w, W, C_in, C_out, (uint32_t)bn)) return SBP_ERR_CUDA;
-    const dim3 grid((unsigned)((M_keep_cap + kBM - 1) / kBM), (unsigned)((C_in + bn - 1) / bn));
-    cudaError_t launch_err;
-    if (bn == 256) {
-        static cudaError_t once = allow_smem(tc_dx_kernel<256>, TcCfg<256>::kSmemBytes);
-        if (once != cudaSuccess) return SBP_ERR_CUDA;
-        launch_err = launch_pdl(tc_dx_kernel<256>, grid, dim3(kTcThreads), TcCfg<256>::kSmemBytes, stream,
-            map_w, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M, M_keep_cap, (int)C_in, (int)C_out,
-            (__nv_bfloat16*)dX, status_word);
-    } else {
-        static cudaError_t once = allow_smem(tc_dx_kernel<128>, TcCfg<128>::kSmemBytes);
-        if (once != cudaSuccess) return SBP_ERR_CUDA;
-        launch_err = launch_pdl(tc_dx_kernel<128>, grid, dim3(kTcThreads), TcCfg<128>::kSmemBytes, stream,
-            map_w, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M, M_keep_cap, (int)C_in, (int)C_out,
-            (__nv_bfloat16*)dX, status_word);
-    }
-    return launch_err == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
-}
-
-sbp_status launch_tc_dw(const void* X_keep, const void* dY, const int32_t* keep_rows, const int32_t* M_keep_dev,
-                        int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out, float* dW, bool accumulate,
-                        float* workspace, int32_t* status_word, cudaStream_t stream) {
-    (void)M;
-    const DwPlan p = plan_dw(M_keep_cap, C_in, C_out);
-    CUtensorMap map_x;
-    if (!make_map(&map_x, X_keep, M_keep_cap, C_in, 64)) return SBP_ERR_CUDA;
-    const dim3 grid((unsigned)((C_out + p.bn - 1) / p.bn), (unsigned)((C_in + kBM - 1) / kBM), (unsigned)p.splits);
-    float* out = p.splits > 1 ? workspace : dW;
-    const int acc_in_kernel = (p.splits == 1 && accumulate) ? 1 : 0;
-    const int64_t split_stride = C_in * C_out;
-    cudaError_t launch_err;
-    if (p.bn == 256) {
-        static cudaError_t once = allow_smem(tc_dw_kernel<256>, TcCfg<256>::kSmemBytes);
-        if (once != cudaSuccess) return SBP_ERR_CUDA;
-        launch_err = launch_pdl(tc_dw_kernel<256>, grid, dim3(kTcThreads), TcCfg<256>::kSmemBytes, stream,
-            map_x, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M_keep_cap, (int)C_in, (int)C_out, out,
-            split_stride, acc_in_kernel, status_word);
-    } else {
-        static cudaError_t once = allow_smem(tc_dw_kernel<128>, TcCfg<128>::kSmemBytes);
-        if (once != cudaSuccess) return SBP_ERR_CUDA;
-        launch_err = launch_pdl(tc_dw_kernel<128>, grid, dim3(kTcThreads), TcCfg<128>::kSmemBytes, stream,
-            map_x, (const __nv_bfloat16*)dY, keep_rows, M_keep_dev, M_keep_cap, (int)C_in, (int)C_out, out,
-            split_stride, acc_in_kernel, status_word);
-    }
-    if (launch_err != cudaSuccess) return SBP_ERR_CUDA;
-    if (p.splits > 1 &&
-        launch_reduce_partials(workspace, p.splits, C_in * C_out, dW, accumulate, status_word, stream) != cudaSuccess)
+sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
+                              const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
+                              float* dW, bool accumulate, void* dX, float* workspace, int32_t* status_word,
+                              cudaStream_t stream) {
+    const bool want_dw = dW != nullptr, want_dx = dX != nullptr;
+    if (!want_dw && !want_dx) return SBP_OK;
+    const Plan pl = make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx);
+    CUtensorMap map_w, map_x;
+    // a product that is not requested still gets a valid map (of the other matrix): it is never used
+    const void* w_base = want_dx ? W : X_keep;
+    const void* x_base = want_dw ? X_keep : W;
+    if (!make_map(&map_w, w_base, want_dx ? C_in : M_keep_cap, want_dx ? C_out : C_in, want_dx ? (uint32_t)pl.bnx : 64u) ||
+        !make_map(&map_x, x_base, want_dw ? M_keep_cap : C_in, want_dw ? C_in : C_out, want_dw ? 64u : (uint32_t)pl.bnx))
+        return SBP_ERR_CUDA;
+    TcParams prm;
+    prm.dY = static_cast<const __nv_bfloat16*>(dY);
+    prm.keep_rows = keep_rows;
+    prm.M_keep_dev = M_keep_dev;
+    prm.M = M;
+    prm.M_keep_cap = M_keep_cap;
+    prm.C_in = (int)C_in;
+    prm.C_out = (int)C_out;
+    prm.dX = static_cast<__nv_bfloat16*>(dX);
+    prm.dW_out = want_dw ? (pl.splits > 1 ? workspace : dW) : nullptr;
+    prm.dw_split_stride = C_in * C_out;
+    prm.dw_splits = pl.splits;
+    prm.dw_accumulate = (pl.splits == 1 && accumulate) ? 1 : 0;
+    prm.status_word = status_word;
+    int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
+    if (ctas < 1) ctas = 1;
+    const dim3 grid((unsigned)ctas);
+    cudaError_t e;
+    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, prm);
+    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, prm);
+    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, prm);
+    else e = launch_fused<128, 128>(grid, stream, map_w, map_x, prm);
+    if (e != cudaSuccess) return SBP_ERR_CUDA;
+    if (want_dw && pl.splits > 1 &&
+        launch_reduce_partials(workspace, pl.splits, C_in * C_out, dW, accumulate, status_word, stream) != cudaSuccess)
         return SBP_ERR_CUDA;
     return SBP_OK;
 }
