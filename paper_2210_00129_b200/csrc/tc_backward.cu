@@ -4,16 +4,17 @@
 //              A = kept rows of dY, gathered straight from the full dY; B = W tile (TMA);
 //              the epilogue rounds to bf16, scatters each row to dX[keep_rows[m], :] and
 //              zero-fills the dropped rows between kept rows.
-//   dW tiles:  D[i, j] = sum_m X_keep[m, i] * dY[keep_rows[m], j]       (both operands MN-major)
-//              A = X_keep tile (TMA), B = gathered dY rows; long reductions are cut into pieces
-//              whose partial results a second kernel adds in a fixed order.
+//   dW tiles:  D[j, i] = sum_m dY[keep_rows[m], j] * X_keep[m, i]       (both operands MN-major)
+//              computed transposed so that the gathered operand is again the 128-row side:
+//              A = gathered dY rows, B = X_keep tile (TMA); the epilogue writes dW[i, j];
+//              long reductions are cut into pieces whose partials a second kernel adds in order.
 //
 // ONE persistent kernel runs both products: every CTA (one per SM) walks a static, cost-sorted
 // list of 128 x BN output tiles of either kind.  The operand ring (64-deep, 128-byte-swizzled
 // stages behind full/empty mbarriers) never drains between tiles, and the fp32 accumulator in
 // tensor memory is double-buffered, so the epilogue of one tile overlaps the MMAs of the next.
 // Warp roles: warps 0-3 epilogue (TMEM lane quadrant = warp id), warp 4 TMA producer of the dense
-// operand, warp 5 MMA issuer and TMEM owner, warps 6-9 gather producers, which copy the indexed
+// operand, warp 5 MMA issuer and TMEM owner, warps 6-7 gather producers, which copy the indexed
 // rows of dY with coalesced 16-byte cp.async into the swizzled layout the MMA reads; each thread's
 // copies signal the stage's barrier when they land (cp.async.mbarrier.arrive).  TMA tile::gather4
 // was measured at ~45 ns of issue time per instruction per SM whatever it fetches - far too slow
@@ -23,9 +24,10 @@
 namespace sbp {
 namespace {
 
-constexpr int kTcThreads = 320;
-constexpr int kGatherWarp0 = 6;          // first of the four gather warps
-constexpr int kGatherThreads = 128;
+constexpr int kGatherWarp0 = 6;          // first gather warp
+constexpr int kGatherWarps = 2;          // every gather thread adds an arrival per stage: keep them few
+constexpr int kGatherThreads = 32 * kGatherWarps;
+constexpr int kTcThreads = 32 * kGatherWarp0 + kGatherThreads;
 constexpr int kBM = 128;                 // accumulator rows per tile (= TMEM lanes)
 constexpr int kBK = 64;                  // reduction depth per stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kUmmaK = 16;          // reduction depth of one tcgen05.mma for 16-bit operands
@@ -66,14 +68,14 @@ struct TcParams {
 // ---- the static tile list -------------------------------------------------------------------
 struct Schedule {
     uint32_t x_tiles, x_ntiles, x_kb;                 // dX: row tiles x column tiles, k-blocks per tile
-    uint32_t w_tiles, w_jtiles, w_kb_total, w_kb_per; // dW: (i tiles x j tiles x splits), k-blocks per piece
+    uint32_t w_tiles, w_ctiles, w_kb_total, w_kb_per; // dW: (C_out tiles x C_in tiles x splits), k-blocks per piece
     uint32_t splits;
     bool w_first;                                     // the costlier kind is handed out first
     uint32_t total;
 };
 struct Tile {
     bool is_dw;
-    uint32_t row_tile, col_tile;      // dX: kept-row tile, C_in tile; dW: C_in tile, C_out tile
+    uint32_t row_tile, col_tile;      // dX: kept-row tile, C_in tile; dW: C_out tile (128), C_in tile (BNW)
     uint32_t split, kb_begin, num_kb;
 };
 
@@ -84,8 +86,8 @@ __device__ __forceinline__ Schedule make_schedule(const TcParams& p, int64_t M_k
     s.x_tiles = (p.dX != nullptr) ? (uint32_t)((M_keep + kBM - 1) / kBM) * s.x_ntiles : 0u;
     s.x_kb = (uint32_t)((p.C_out + kBK - 1) / kBK);
     s.splits = (uint32_t)p.dw_splits;
-    s.w_jtiles = (uint32_t)((p.C_out + BNW - 1) / BNW);
-    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_in + kBM - 1) / kBM) * s.w_jtiles * s.splits : 0u;
+    s.w_ctiles = (uint32_t)((p.C_in + BNW - 1) / BNW);
+    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_out + kBM - 1) / kBM) * s.w_ctiles * s.splits : 0u;
     s.w_kb_total = (uint32_t)((M_keep + kBK - 1) / kBK);
     s.w_kb_per = (s.w_kb_total + s.splits - 1) / s.splits;
     s.w_first = s.w_kb_per >= s.x_kb;
@@ -101,8 +103,8 @@ __device__ __forceinline__ Tile decode_tile(const Schedule& s, uint32_t q) {
     if (t.is_dw) {
         t.split = idx % s.splits;
         const uint32_t ij = idx / s.splits;
-        t.row_tile = ij / s.w_jtiles;
-        t.col_tile = ij % s.w_jtiles;
+        t.row_tile = ij / s.w_ctiles;
+        t.col_tile = ij % s.w_ctiles;
         t.kb_begin = s.w_kb_per * t.split;
         const uint32_t end = (t.kb_begin + s.w_kb_per < s.w_kb_total) ? t.kb_begin + s.w_kb_per : s.w_kb_total;
         t.num_kb = (end > t.kb_begin) ? end - t.kb_begin : 0u;
@@ -191,11 +193,12 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     if (!ok) break;
                     const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
                     const uint32_t a_dst = ring + s * kStageBytes;
-                    if (t.is_dw) {                                   // X_keep tile: two 64-wide blocks of 64 kept rows
-                        const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.row_tile * kBM);
-                        ptx::mbar_arrive_expect_tx(full, kABytes);
-                        ptx::tma_load_2d(a_dst, &map_x, i0, row0, full);
-                        ptx::tma_load_2d(a_dst + kBlock64Bytes, &map_x, i0 + 64, row0, full);
+                    if (t.is_dw) {                                   // X_keep tile: BNW/64 blocks of 64 columns x 64 kept rows
+                        const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.col_tile * BNW);
+                        ptx::mbar_arrive_expect_tx(full, BNW * kRowBytes);
+#pragma unroll
+                        for (int b = 0; b < BNW / 64; ++b)
+                            ptx::tma_load_2d(a_dst + kABytes + b * kBlock64Bytes, &map_x, i0 + b * 64, row0, full);
                     } else {                                         // W tile: BNX rows x 64 columns
                         ptx::mbar_arrive_expect_tx(full, BNX * kRowBytes);
                         ptx::tma_load_2d(a_dst + kABytes, &map_w, (int)(k * kBK), (int)(t.col_tile * BNX), full);
@@ -263,17 +266,15 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             const Tile t = decode_tile(sched, q);
             if (!t.is_dw) {
                 // dX tile: 128 kept rows x 128 bytes per stage; one warp instruction moves 4 rows x 128 B
-                const uint32_t chunk = lane & 7;
+                constexpr int kInstr = 32 / kGatherWarps;
+                const uint32_t chunk = lane & 7, sub = lane >> 3;
                 const int64_t m0 = (int64_t)t.row_tile * kBM;
-                const __nv_bfloat16* src[8];
-                uint32_t dst[8];
+                const __nv_bfloat16* src[kInstr];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint32_t row = gw * 32 + i * 4 + (lane >> 3);
-                    int64_t m = m0 + row;
+                for (int i = 0; i < kInstr; ++i) {
+                    int64_t m = m0 + (gw * kInstr + i) * 4 + sub;
                     if (m >= M_keep) m = M_keep - 1;                  // padding rows of the last tile: never stored
                     src[i] = p.dY + (int64_t)__ldg(p.keep_rows + m) * C_out + chunk * 8;
-                    dst[i] = swizzled(row, chunk);
                 }
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
                     const int s = it % kStages;
@@ -285,38 +286,59 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     const uint32_t bytes = (col < C_out) ? 16u : 0u;  // columns past C_out read as zero
                     const int off = (col < C_out) ? (int)(k * kBK) : 0;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) ptx::cp_async_16(a_dst + dst[i], src[i] + off, bytes);
+                    for (int i = 0; i < kInstr; ++i)
+                        ptx::cp_async_16(a_dst + swizzled((gw * kInstr + i) * 4 + sub, chunk), src[i] + off, bytes);
                     // the stage's barrier gets this thread's arrival when the copies above have landed
                     ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
                 }
             } else {
-                // dW tile: 64 kept rows x BNW columns per stage; a warp owns 16 rows, one instruction moves 512 B
-                constexpr int kChunksPerRow = BNW / 8;               // 16-byte chunks of one row of the tile
-                constexpr int kRowsPerInstr = 32 / kChunksPerRow;    // 1 (BNW = 256) or 2 (BNW = 128)
-                constexpr int kInstr = 16 / kRowsPerInstr;
-                const uint32_t c = lane % kChunksPerRow;             // chunk within the row
-                const uint32_t sub = lane / kChunksPerRow;           // which of the rows of this instruction
-                const int col = (int)(t.col_tile * BNW) + (int)c * 8;
+                // dW tile: 64 kept rows x 128 columns (256 B) of dY per stage; one warp instruction moves 2 rows
+                constexpr int kRows = 64 / kGatherWarps;             // rows of a stage this warp copies
+                constexpr int kIdxPerLane = (kRows + 31) / 32;       // row ids each lane holds per stage
+                constexpr int kInstr = kRows / 2;
+                constexpr int kAhead = 4;                            // row ids are fetched this many stages early
+                const uint32_t c = lane & 15;                        // 16-byte chunk within the 256-byte row piece
+                const uint32_t sub = lane >> 4;                      // which of the two rows of this instruction
+                const int col = (int)(t.row_tile * kBM) + (int)c * 8;
                 const bool col_ok = col < C_out;                     // columns past C_out read as zero
                 const __nv_bfloat16* col_ptr = p.dY + (col_ok ? col : 0);
-                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
-                    const int s = it % kStages;
-                    // row ids of this warp's 16 rows: lanes 0..15 fetch one each
-                    const int64_t mrow = (int64_t)(t.kb_begin + k) * kBK + gw * 16 + (lane & 15);
-                    const int my_row = (mrow < M_keep) ? __ldg(p.keep_rows + mrow) : -1;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    const uint32_t b_dst = ring + s * kStageBytes + kABytes;
+                int nxt[kAhead][kIdxPerLane];
+                auto fetch_ids = [&](uint32_t k_first) {
 #pragma unroll
-                    for (int i = 0; i < kInstr; ++i) {
-                        const uint32_t r = gw * 16 + i * kRowsPerInstr + sub;         // row within the 64-row stage
-                        const int g = __shfl_sync(0xffffffffu, my_row, i * kRowsPerInstr + (int)sub);
-                        const bool live = g >= 0 && col_ok;                           // rows past M_keep read as zero
-                        ptx::cp_async_16(b_dst + (c >> 3) * kBlock64Bytes + swizzled(r, c & 7u),
-                                         col_ptr + (live ? (int64_t)g * C_out : 0), live ? 16u : 0u);
+                    for (int u = 0; u < kAhead; ++u)
+#pragma unroll
+                        for (int h = 0; h < kIdxPerLane; ++h) {
+                            const int64_t mrow = (int64_t)(t.kb_begin + k_first + u) * kBK + gw * kRows + h * 32 + (lane % kRows);
+                            nxt[u][h] = (k_first + u < t.num_kb && mrow < M_keep) ? __ldg(p.keep_rows + mrow) : -1;
+                        }
+                };
+                fetch_ids(0);
+                for (uint32_t k0 = 0; k0 < t.num_kb && ok; k0 += kAhead) {
+                    int cur[kAhead][kIdxPerLane];
+#pragma unroll
+                    for (int u = 0; u < kAhead; ++u)
+#pragma unroll
+                        for (int h = 0; h < kIdxPerLane; ++h) cur[u][h] = nxt[u][h];
+                    fetch_ids(k0 + kAhead);
+#pragma unroll
+                    for (int u = 0; u < kAhead; ++u) {
+                        if (k0 + u >= t.num_kb) break;
+                        const int s = it % kStages;
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        const uint32_t a_dst = ring + s * kStageBytes;
+#pragma unroll
+                        for (int i = 0; i < kInstr; ++i) {
+                            const int rl = i * 2 + (int)sub;                                  // row within this warp's share
+                            const int g = __shfl_sync(0xffffffffu, cur[u][rl >> 5], rl & 31);
+                            const bool live = g >= 0 && col_ok;                               // rows past M_keep read as zero
+                            ptx::cp_async_16(a_dst + (c >> 3) * kBlock64Bytes + swizzled(gw * kRows + rl, c & 7u),
+                                             col_ptr + (live ? (int64_t)g * C_out : 0), live ? 16u : 0u);
+                        }
+                        ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
+                        ++it;
                     }
-                    ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
                 }
             }
         }
@@ -379,14 +401,14 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
                 }
             } else {
-                // ---- dW tile: fp32 accumulator rows to dW (or to this piece's partial buffer) ----
-                const int i = (int)(t.row_tile * kBM) + warp * 32 + lane;
-                const int j0 = (int)(t.col_tile * BNW);
-                float* out_row = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i * C_out + j0;
+                // ---- dW tile: accumulator row = output column j, accumulator column = output row i ----
+                // a warp-wide store of one accumulator column covers 32 consecutive j: 128 contiguous bytes
+                const int j = (int)(t.row_tile * kBM) + warp * 32 + lane;
+                const int i0 = (int)(t.col_tile * BNW);
+                float* out_col = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i0 * C_out + j;
                 if (t.num_kb == 0) {                                 // a piece without kept rows contributes zero
-                    if (!p.dw_accumulate && i < C_in)
-                        for (int c0 = 0; c0 < BNW; c0 += 4)
-                            if (j0 + c0 < C_out) ptx::st_global_v4(out_row + c0, 0u, 0u, 0u, 0u);
+                    if (!p.dw_accumulate && j < C_out)
+                        for (int c0 = 0; c0 < BNW && i0 + c0 < C_in; ++c0) out_col[(int64_t)c0 * C_out] = 0.f;
                     continue;
                 }
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
@@ -398,14 +420,12 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     float v[32];
                     ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
                     ptx::tmem_ld_wait();
-                    if (i < C_in) {
+                    if (j < C_out) {
 #pragma unroll
-                        for (int qd = 0; qd < 8; ++qd) {
-                            if (j0 + c0 + qd * 4 < C_out) {
-                                float4 w = make_float4(v[qd * 4], v[qd * 4 + 1], v[qd * 4 + 2], v[qd * 4 + 3]);
-                                float4* dst = reinterpret_cast<float4*>(out_row + c0 + qd * 4);
-                                if (p.dw_accumulate) { const float4 o = *dst; w.x += o.x; w.y += o.y; w.z += o.z; w.w += o.w; }
-                                *dst = w;
+                        for (int r = 0; r < 32; ++r) {
+                            if (i0 + c0 + r < C_in) {
+                                float* dst = out_col + (int64_t)(c0 + r) * C_out;
+                                *dst = p.dw_accumulate ? *dst + v[r] : v[r];
                             }
                         }
                     }
@@ -466,10 +486,10 @@ struct Plan {
 Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
     Plan pl;
     pl.bnx = (C_in >= 256) ? 256 : 128;
-    pl.bnw = (C_out >= 256) ? 256 : 128;
+    pl.bnw = (C_in >= 256) ? 256 : 128;
     const int64_t x_tiles = want_dx ? ((M_keep_cap + kBM - 1) / kBM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
     const int64_t x_kb = (C_out + kBK - 1) / kBK;
-    const int64_t w_tiles = want_dw ? ((C_in + kBM - 1) / kBM) * ((C_out + pl.bnw - 1) / pl.bnw) : 0;
+    const int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
     const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
     // Cut the dW reductions so that one piece is no longer than an even share of all the work
     // (in k-block units; a BN=128 tile's unit is cheaper, which only makes the cut finer).
