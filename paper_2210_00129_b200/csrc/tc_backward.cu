@@ -368,37 +368,66 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const bool valid = m < M_keep;
                 const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
                 const int64_t prev = (valid && m > 0) ? (int64_t)__ldg(p.keep_rows + m - 1) : -1;
-                for (int r = 0; r < 32; ++r) {
-                    if (!__shfl_sync(0xffffffffu, valid ? 1 : 0, r)) break;
-                    const int64_t c = __shfl_sync(0xffffffffu, cur, r);
-                    int64_t g = __shfl_sync(0xffffffffu, prev, r) + 1;
-                    for (; g < c; ++g)
-                        for (int v = lane; v < strip_vecs; v += 32)
-                            ptx::st_global_v4(p.dX + g * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
-                    if (m0 + warp * 32 + r == M_keep - 1)            // after the very last kept row
-                        for (g = c + 1; g < p.M; ++g)
-                            for (int v = lane; v < strip_vecs; v += 32)
-                                ptx::st_global_v4(p.dX + g * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
+                // Rows this warp owns: from just after the kept row preceding its first one up to its
+                // last kept row (to the end of dX if it holds the very last kept row).  They are walked
+                // in windows of 32; a warp-wide OR marks the kept rows of a window, the rest get zeros.
+                const int nvalid = __popc(__ballot_sync(0xffffffffu, valid));
+                if (nvalid > 0) {
+                    const int64_t lo = __shfl_sync(0xffffffffu, prev, 0) + 1;
+                    const int64_t last_cur = __shfl_sync(0xffffffffu, cur, nvalid - 1);
+                    const int64_t hi = (m0 + warp * 32 + nvalid == M_keep) ? p.M : last_cur;
+                    for (int64_t base = lo; base < hi; base += 32) {
+                        const int64_t d = cur - base;
+                        uint32_t todo = ~__reduce_or_sync(0xffffffffu, (valid && d >= 0 && d < 32) ? (1u << d) : 0u);
+                        if (hi - base < 32) todo &= (1u << (hi - base)) - 1u;
+                        if (strip_vecs <= 16) {                      // narrow strip: two rows per store instruction
+                            while (todo) {
+                                const int b0 = __ffs(todo) - 1;
+                                todo &= todo - 1u;
+                                const int b1 = todo ? __ffs(todo) - 1 : -1;
+                                if (todo) todo &= todo - 1u;
+                                const int b = (lane < 16) ? b0 : b1;
+                                const int v = lane & 15;
+                                if (b >= 0 && v < strip_vecs)
+                                    ptx::st_global_v4(p.dX + (base + b) * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
+                            }
+                        } else {
+                            while (todo) {
+                                const int b = __ffs(todo) - 1;
+                                todo &= todo - 1u;
+                                if (lane < strip_vecs)
+                                    ptx::st_global_v4(p.dX + (base + b) * C_in + n0 + lane * 8, 0u, 0u, 0u, 0u);
+                            }
+                        }
+                    }
                 }
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 __nv_bfloat16* out_row = p.dX + (valid ? cur : 0) * C_in + n0;
-#pragma unroll 1
-                for (int c0 = 0; c0 < BNX; c0 += 32) {
-                    float v[32];
-                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
-                    ptx::tmem_ld_wait();
-                    if (valid) {
+                auto store_chunk = [&](const float (&v)[32], int c0) {   // 32 accumulator columns -> 64 bytes of one row
+                    if (!valid) return;
 #pragma unroll
-                        for (int qd = 0; qd < 4; ++qd) {
-                            if (c0 + qd * 8 < strip_cols)
-                                ptx::st_global_v4(out_row + c0 + qd * 8,
-                                                  pack_bf16(v[qd * 8 + 0], v[qd * 8 + 1]), pack_bf16(v[qd * 8 + 2], v[qd * 8 + 3]),
-                                                  pack_bf16(v[qd * 8 + 4], v[qd * 8 + 5]), pack_bf16(v[qd * 8 + 6], v[qd * 8 + 7]));
-                        }
+                    for (int qd = 0; qd < 4; ++qd) {
+                        if (c0 + qd * 8 < strip_cols)
+                            ptx::st_global_v4(out_row + c0 + qd * 8,
+                                              pack_bf16(v[qd * 8 + 0], v[qd * 8 + 1]), pack_bf16(v[qd * 8 + 2], v[qd * 8 + 3]),
+                                              pack_bf16(v[qd * 8 + 4], v[qd * 8 + 5]), pack_bf16(v[qd * 8 + 6], v[qd * 8 + 7]));
                     }
+                };
+                // two register buffers: the next TMEM read is in flight while the current chunk is stored
+                float va[32], vb[32];
+                ptx::tmem_ld_32x32(taddr, va);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int c0 = 0; c0 < BNX; c0 += 64) {
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), vb);
+                    store_chunk(va, c0);
+                    ptx::tmem_ld_wait();
+                    if (c0 + 64 < BNX) ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
+                    store_chunk(vb, c0 + 32);
+                    ptx::tmem_ld_wait();
                 }
             } else {
                 // ---- dW tile: accumulator row = output column j, accumulator column = output row i ----
@@ -415,20 +444,27 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-#pragma unroll 1
-                for (int c0 = 0; c0 < BNW; c0 += 32) {
-                    float v[32];
-                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, v);
-                    ptx::tmem_ld_wait();
-                    if (j < C_out) {
+                auto store_cols = [&](const float (&v)[32], int c0) {    // 32 accumulator columns = 32 rows of dW
+                    if (j >= C_out) return;
 #pragma unroll
-                        for (int r = 0; r < 32; ++r) {
-                            if (i0 + c0 + r < C_in) {
-                                float* dst = out_col + (int64_t)(c0 + r) * C_out;
-                                *dst = p.dw_accumulate ? *dst + v[r] : v[r];
-                            }
+                    for (int r = 0; r < 32; ++r) {
+                        if (i0 + c0 + r < C_in) {
+                            float* dst = out_col + (int64_t)(c0 + r) * C_out;
+                            *dst = p.dw_accumulate ? *dst + v[r] : v[r];
                         }
                     }
+                };
+                float va[32], vb[32];
+                ptx::tmem_ld_32x32(taddr, va);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int c0 = 0; c0 < BNW; c0 += 64) {
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), vb);
+                    store_cols(va, c0);
+                    ptx::tmem_ld_wait();
+                    if (c0 + 64 < BNW) ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
+                    store_cols(vb, c0 + 32);
+                    ptx::tmem_ld_wait();
                 }
             }
             // this warp is done with the accumulator: hand it back to the MMA issuer
