@@ -21,6 +21,14 @@ inline bool ratio_ok(double r) { return r > 0.0 && r <= 1.0; }   // false for Na
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// scratch for the bias sums: the stand-alone kernel's row splits, or one partial row per SM when the
+// sums ride along in the tensor-core kernel
+inline size_t db_scratch_bytes(sbp_dtype dt, int64_t M_keep_cap, int64_t C_out) {
+    const size_t a = db_workspace_bytes(dt, M_keep_cap, C_out, kDbMaxSplits);
+    const size_t b = (size_t)kNumSMs * (size_t)C_out * sizeof(float);
+    return align_up(a > b ? a : b, 256);
+}
+
 inline bool use_tensor_cores(sbp_dtype dt, uint32_t flags, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
     return dt == SBP_BF16 && !(flags & SBP_FLAG_PLAIN_FMA) && tc_shapes_supported(M, M_keep_cap, C_in, C_out);
 }
@@ -103,7 +111,7 @@ sbp_status sbp_forward_cache(sbp_dtype dt, const void* X, int64_t M, int64_t C, 
 size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                            int64_t C_out) {
     if (M <= 0 || M_keep_cap < 0 || C_in <= 0 || C_out <= 0) return 256;
-    const size_t db_part = align_up(db_workspace_bytes(dt, M_keep_cap, C_out, kDbMaxSplits), 256);
+    const size_t db_part = db_scratch_bytes(dt, M_keep_cap, C_out);
     size_t dw_part = simt_dw_workspace_bytes(M_keep_cap, C_in, C_out);
     if (dt == SBP_BF16 && tc_shapes_supported(M, M_keep_cap, C_in, C_out)) {
         const size_t t = tc_dw_workspace_bytes(M_keep_cap, C_in, C_out);
@@ -140,7 +148,7 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     const bool accumulate = (flags & SBP_FLAG_ACCUMULATE) != 0;
     float* ws_db = static_cast<float*>(workspace);
     float* ws_dw = need_ws ? reinterpret_cast<float*>(static_cast<char*>(workspace) +
-                                                      align_up(db_workspace_bytes(dt, M_keep_cap, C_out, kDbMaxSplits), 256))
+                                                      db_scratch_bytes(dt, M_keep_cap, C_out))
                            : nullptr;
 
     if (flags & SBP_FLAG_VALIDATE) {
@@ -148,15 +156,18 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
             return SBP_ERR_CUDA;
     }
     const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
-    if (db != nullptr) {
+    // with the tensor-core kernel running, the bias sums ride along in it; otherwise they get their own kernel
+    const bool db_rides = tc && db != nullptr && (dW != nullptr || dX != nullptr);
+    if (db != nullptr && !db_rides) {
         if (launch_db(dt, dY, keep_rows, M_keep_dev, M_keep_cap, C_out, db, accumulate, ws_db, kDbMaxSplits,
                       status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
     }
     if (tc) {
-        // both products in one persistent tensor-core kernel
+        // both products (and the bias sums) in one persistent tensor-core kernel
         const sbp_status s = launch_tc_backward(X_keep, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW,
-                                                accumulate, dX, ws_dw, status_word, stream);
+                                                accumulate, dX, db_rides ? db : nullptr, ws_dw, ws_db, status_word,
+                                                stream);
         if (s != SBP_OK) return s;
     } else {
         if (dW != nullptr && launch_simt_dw(dt, X_keep, dY, keep_rows, M_keep_dev, M_keep_cap, C_in, C_out, dW,
@@ -173,8 +184,9 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
                                      int want_dW, int want_db, int want_dX, uint32_t flags) {
     const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
     int n = (flags & SBP_FLAG_VALIDATE) ? 1 : 0;
-    if (want_db) n += 2;                                   // strip partials + fixed-order reduce
-    if (tc) return n + tc_backward_kernel_count(M_keep_cap, C_in, C_out, want_dW != 0, want_dX != 0);
+    const bool db_rides = tc && want_db && (want_dW || want_dX);
+    if (want_db && !db_rides) n += 2;                      // strip partials + fixed-order reduce
+    if (tc) return n + tc_backward_kernel_count(M_keep_cap, C_in, C_out, want_dW != 0, want_dX != 0, db_rides);
     if (want_dW) n += simt_dw_kernel_count(M_keep_cap, C_in, C_out);
     if (want_dX) n += 1;
     return n;

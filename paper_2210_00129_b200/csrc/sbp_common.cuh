@@ -119,11 +119,13 @@ cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const in
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
-int    tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx);
-// dW (nullable) and dX (nullable) of one layer in a single persistent kernel (+ the split reduce)
+int    tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx,
+                                bool want_db);
+// dW (nullable) and dX (nullable) of one layer in a single persistent kernel (+ the split reduce); when db is
+// given its column sums ride along in the same kernel (db_workspace: kNumSMs * C_out floats) + one reduce
 sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
                               const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
-                              int64_t C_out, float* dW, bool accumulate, void* dX, float* workspace,
-                              int32_t* status_word, cudaStream_t stream);
+                              int64_t C_out, float* dW, bool accumulate, void* dX, float* db, float* workspace,
+                              float* db_workspace, int32_t* status_word, cudaStream_t stream);
 
 }  // namespace sbp

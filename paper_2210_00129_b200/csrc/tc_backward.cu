@@ -19,6 +19,9 @@
 // copies signal the stage's barrier when they land (cp.async.mbarrier.arrive).  TMA tile::gather4
 // was measured at ~45 ns of issue time per instruction per SM whatever it fetches - far too slow
 // to feed a tile - and is not used.  Every wait is bounded and reports through the status word.
+// Four more warps compute the bias gradient on the side: each CTA sums its share of the kept rows
+// of dY column-wise while the tensor pipe works (the kernel is latency-bound, not bandwidth-bound,
+// so the extra reads are free) and leaves one partial row per CTA for a fixed-order reduce.
 #include "tc_ptx.cuh"
 
 namespace sbp {
@@ -27,7 +30,9 @@ namespace {
 constexpr int kGatherWarp0 = 6;          // first gather warp
 constexpr int kGatherWarps = 2;          // every gather thread adds an arrival per stage: keep them few
 constexpr int kGatherThreads = 32 * kGatherWarps;
-constexpr int kTcThreads = 32 * kGatherWarp0 + kGatherThreads;
+constexpr int kBiasWarp0 = kGatherWarp0 + kGatherWarps;   // four bias warps ride along after the gather warps
+constexpr int kBiasThreads = 128;
+constexpr int kTcThreads = 32 * kBiasWarp0 + kBiasThreads;
 constexpr int kBM = 128;                 // accumulator rows per tile (= TMEM lanes)
 constexpr int kBK = 64;                  // reduction depth per stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kUmmaK = 16;          // reduction depth of one tcgen05.mma for 16-bit operands
@@ -39,7 +44,8 @@ constexpr uint32_t kABytes = kBM * kRowBytes;        // 16 KB
 constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
 constexpr uint32_t kAccCols = 256;       // TMEM columns per accumulator buffer (two buffers = all 512)
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + 1024;   // ring + control block + alignment slack
+constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float);   // cross-row-group sums of the bias warps
+constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kBiasSmemBytes + 1024;   // ring + control + bias + slack
 
 struct TcControl {
     uint64_t full_bar[kStages];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
@@ -62,6 +68,7 @@ struct TcParams {
     int64_t dw_split_stride;       // elements between partial buffers
     int dw_splits;
     int dw_accumulate;             // add into dW_out (only with one split)
+    float* db_partial;             // nullptr: no bias sums; else [gridDim.x, C_out] per-CTA column sums of kept dY rows
     int32_t* status_word;
 };
 
@@ -255,7 +262,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp >= kGatherWarp0) {
+    } else if (warp >= kGatherWarp0 && warp < kBiasWarp0) {
         // ---------------- gather producers ----------------
         const int gw = warp - kGatherWarp0;
         uint32_t it = 0;
@@ -343,6 +350,65 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         ptx::cp_async_wait_all();
+    } else if (warp >= kBiasWarp0) {
+        // ---------------- bias warps: db partial of this CTA's share of the kept rows ----------------
+        if (p.db_partial != nullptr) {
+            float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256);
+            const int t = threadIdx.x - kBiasWarp0 * 32;
+            const int V = C_out >> 3;                                  // 16-byte column vectors per row
+            int VT = 16;                                               // vectors covered per pass (power of two <= 128)
+            while (VT < V && VT < kBiasThreads) VT <<= 1;
+            const int RG = kBiasThreads / VT;                          // row groups working on the same columns
+            const int cvt = t % VT, rg = t / VT;
+            const int64_t rows_per = (M_keep + gridDim.x - 1) / gridDim.x;
+            const int64_t m_begin = rows_per * blockIdx.x;
+            const int64_t m_end = (m_begin + rows_per < M_keep) ? m_begin + rows_per : M_keep;
+            const uint4* dY4 = reinterpret_cast<const uint4*>(p.dY);
+            float* out = p.db_partial + (int64_t)blockIdx.x * C_out;
+            for (int cv0 = 0; cv0 < V; cv0 += VT) {
+                const int cv = cv0 + cvt;
+                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                if (cv < V) {
+                    for (int64_t m = m_begin + rg; m < m_end; m += (int64_t)RG * 8) {
+                        int64_t row[8];
+                        uint4 v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int64_t mm = m + (int64_t)u * RG;
+                            row[u] = (mm < m_end) ? (int64_t)__ldg(p.keep_rows + mm) : -1;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            v[u] = (row[u] >= 0) ? __ldg(dY4 + row[u] * V + cv) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                acc[2 * e] += __uint_as_float(w[e] << 16);
+                                acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                            }
+                        }
+                    }
+                }
+                // add the row groups in a fixed order
+#pragma unroll
+                for (int e = 0; e < 8; ++e) red[t * 8 + e] = acc[e];
+                asm volatile("bar.sync 1, %0;" ::"n"(kBiasThreads) : "memory");
+                if (rg == 0 && cv < V) {
+                    float sum[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) sum[e] = 0.f;
+                    for (int g = 0; g < RG; ++g)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) sum[e] += red[(g * VT + cvt) * 8 + e];
+                    float4* o = reinterpret_cast<float4*>(out + (int64_t)cv * 8);
+                    o[0] = make_float4(sum[0], sum[1], sum[2], sum[3]);
+                    o[1] = make_float4(sum[4], sum[5], sum[6], sum[7]);
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kBiasThreads) : "memory");
+            }
+        }
     } else {
         // ---------------- epilogue warps ----------------
         if (M_keep == 0 && p.dX != nullptr) {                        // nothing kept: dX is all zeros
@@ -568,15 +634,16 @@ size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
     return s > 1 ? (size_t)s * (size_t)C_in * (size_t)C_out * sizeof(float) : 0;
 }
 
-int tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
+int tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx,
+                             bool want_db) {
     if (!want_dw && !want_dx) return 0;
-    return 1 + ((want_dw && make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx).splits > 1) ? 1 : 0);
+    return 1 + ((want_dw && make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx).splits > 1) ? 1 : 0) + (want_db ? 1 : 0);
 }
 
 sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
                               const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
-                              float* dW, bool accumulate, void* dX, float* workspace, int32_t* status_word,
-                              cudaStream_t stream) {
+                              float* dW, bool accumulate, void* dX, float* db, float* workspace, float* db_workspace,
+                              int32_t* status_word, cudaStream_t stream) {
     const bool want_dw = dW != nullptr, want_dx = dX != nullptr;
     if (!want_dw && !want_dx) return SBP_OK;
     const Plan pl = make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx);
@@ -600,6 +667,7 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     prm.dw_split_stride = C_in * C_out;
     prm.dw_splits = pl.splits;
     prm.dw_accumulate = (pl.splits == 1 && accumulate) ? 1 : 0;
+    prm.db_partial = (db != nullptr) ? db_workspace : nullptr;
     prm.status_word = status_word;
     int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
     if (ctas < 1) ctas = 1;
@@ -612,6 +680,9 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     if (e != cudaSuccess) return SBP_ERR_CUDA;
     if (want_dw && pl.splits > 1 &&
         launch_reduce_partials(workspace, pl.splits, C_in * C_out, dW, accumulate, status_word, stream) != cudaSuccess)
+        return SBP_ERR_CUDA;
+    if (db != nullptr &&
+        launch_reduce_partials(db_workspace, (int)ctas, C_out, db, accumulate, status_word, stream) != cudaSuccess)
         return SBP_ERR_CUDA;
     return SBP_OK;
 }
