@@ -34,6 +34,9 @@ from paper_2210_00129_b200 import synth  # noqa: E402
 
 METRIC = "sbp_backward_tflops_kept_rows"
 UNIT = "TFLOP/s"
+# dram__bytes_read + dram__bytes_write of one launch of the dominant kernel, from the ncu capture summarised in
+# profiles/ (None = the kernel changed since, or the workload was never captured)
+NCU_TRAFFIC_BYTES = {"vit_b16_fc1": 60.2e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 WORKLOADS = {
@@ -356,7 +359,7 @@ def run_cuda(args, w, name):
                         "bound": "tensor",
                         "achieved": gemm_flops / (gemm_ms * 1e-3) / 1e12,
                         "peak": peak, "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step)",
-                        "unit": "TFLOP/s", "traffic": None}
+                        "unit": "TFLOP/s", "traffic": NCU_TRAFFIC_BYTES.get(name)}
         else:
             # plain-FMA path: 128 fp32 FMA lanes x 148 SMs x 2 FLOP at the maximum SM clock
             peak = 148 * 128 * 2 * 1.965e9 / 1e12
