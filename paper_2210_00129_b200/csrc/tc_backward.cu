@@ -9,13 +9,10 @@
 //              A = gathered dY rows, B = X_keep tile (TMA); the epilogue writes dW[i, j];
 //              long reductions are cut into pieces whose partials a second kernel adds in order.
 //
-// ONE persistent kernel runs both products.  CTAs work in pairs (a cluster of two SMs, tcgen05
-// cta_group::2): a pair walks a static, cost-sorted list of 256 x BN output tiles of either kind;
-// each CTA gathers its own 128 rows of A and loads half of B, the leader's MMA thread issues one
-// M = 256 instruction that reads both halves, and each CTA keeps its 128 accumulator rows in its own
-// tensor memory.  Sharing B halves the operand bytes per SM (32 KB per 64-deep k-block), so the ring
-// holds six stages: the kernel is bound by bytes in flight, not bandwidth.  The ring never drains
-// between tiles and the accumulator is double-buffered, so epilogues overlap the next tile's MMAs.
+// ONE persistent kernel runs both products: every CTA (one per SM) walks a static, cost-sorted
+// list of 128 x BN output tiles of either kind.  The operand ring (64-deep, 128-byte-swizzled
+// stages behind full/empty mbarriers) never drains between tiles, and the fp32 accumulator in
+// tensor memory is double-buffered, so the epilogue of one tile overlaps the MMAs of the next.
 // Warp roles: warps 0-3 epilogue (TMEM lane quadrant = warp id), warp 4 TMA producer of the dense
 // operand, warp 5 MMA issuer and TMEM owner, warps 6-7 gather producers, which copy the indexed
 // rows of dY with coalesced 16-byte cp.async into the swizzled layout the MMA reads; each thread's
@@ -36,27 +33,25 @@ constexpr int kGatherThreads = 32 * kGatherWarps;
 constexpr int kBiasWarp0 = kGatherWarp0 + kGatherWarps;   // four bias warps ride along after the gather warps
 constexpr int kBiasThreads = 128;
 constexpr int kTcThreads = 32 * kBiasWarp0 + kBiasThreads;
-constexpr int kBM = 128;                 // accumulator rows per CTA (= TMEM lanes)
-constexpr int kPairM = 2 * kBM;          // rows of a pair's tile
+constexpr int kBM = 128;                 // accumulator rows per tile (= TMEM lanes)
 constexpr int kBK = 64;                  // reduction depth per stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kUmmaK = 16;          // reduction depth of one tcgen05.mma for 16-bit operands
 constexpr uint32_t kRowBytes = 128;      // bytes per swizzled smem row
 constexpr uint32_t kAtomBytes = 1024;    // 8 rows x 128 B: one swizzle atom
 constexpr uint32_t kBlock64Bytes = 64 * kRowBytes;   // a 64-row slab (MN-major operands: one 64-wide block)
-constexpr int kStages = 6;
-constexpr uint32_t kABytes = kBM * kRowBytes;        // 16 KB: this CTA's 128 rows of A
-constexpr uint32_t kBBytesMax = 128 * kRowBytes;     // 16 KB: this CTA's half of B
+constexpr int kStages = 4;
+constexpr uint32_t kABytes = kBM * kRowBytes;        // 16 KB
+constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
 constexpr uint32_t kAccCols = 256;       // TMEM columns per accumulator buffer (two buffers = all 512)
 constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float);   // cross-row-group sums of the bias warps
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kBiasSmemBytes + 1024;   // ring + control + bias + slack
 
 struct TcControl {
-    uint64_t full_bar[kStages];    // this CTA's stage: 1 arrival with the TMA byte count + one per gather thread
-    uint64_t peer_full[kStages];   // leader only: 1 arrival from the peer CTA once its stage is full
-    uint64_t empty_bar[kStages];   // 1 arrival: the pair commit of the MMAs that read the stage (sent to both CTAs)
-    uint64_t acc_full[2];          // 1 arrival: all MMAs of the tile in this accumulator are done (sent to both CTAs)
-    uint64_t acc_empty[2];         // leader only: 8 arrivals, one per epilogue warp of the pair
+    uint64_t full_bar[kStages];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
+    uint64_t empty_bar[kStages];   // 1 arrival: tcgen05.commit of the MMAs that read the stage
+    uint64_t acc_full[2];          // 1 arrival: all MMAs of the tile in this accumulator have finished
+    uint64_t acc_empty[2];         // 4 arrivals: each epilogue warp has read the accumulator out
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -95,11 +90,11 @@ template <int BNX, int BNW>
 __device__ __forceinline__ Schedule make_schedule(const TcParams& p, int64_t M_keep) {
     Schedule s;
     s.x_ntiles = (uint32_t)((p.C_in + BNX - 1) / BNX);
-    s.x_tiles = (p.dX != nullptr) ? (uint32_t)((M_keep + kPairM - 1) / kPairM) * s.x_ntiles : 0u;
+    s.x_tiles = (p.dX != nullptr) ? (uint32_t)((M_keep + kBM - 1) / kBM) * s.x_ntiles : 0u;
     s.x_kb = (uint32_t)((p.C_out + kBK - 1) / kBK);
     s.splits = (uint32_t)p.dw_splits;
     s.w_ctiles = (uint32_t)((p.C_in + BNW - 1) / BNW);
-    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_out + kPairM - 1) / kPairM) * s.w_ctiles * s.splits : 0u;
+    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_out + kBM - 1) / kBM) * s.w_ctiles * s.splits : 0u;
     s.w_kb_total = (uint32_t)((M_keep + kBK - 1) / kBK);
     s.w_kb_per = (s.w_kb_total + s.splits - 1) / s.splits;
     s.w_first = s.w_kb_per >= s.x_kb;
@@ -130,10 +125,10 @@ __device__ __forceinline__ Tile decode_tile(const Schedule& s, uint32_t q) {
     return t;
 }
 
-// Pair b of G takes list positions b, 2G-1-b, 2G+b, 4G-1-b, ...: with the list sorted by cost this
+// CTA b takes list positions b, 2G-1-b, 2G+b, 4G-1-b, ...: with the list sorted by cost this
 // evens out the load without any run-time counter.
 __device__ __forceinline__ uint32_t list_position(uint32_t pass) {
-    const uint32_t G = gridDim.x >> 1, b = blockIdx.x >> 1;
+    const uint32_t G = gridDim.x, b = blockIdx.x;
     return pass * G + ((pass & 1u) ? (G - 1u - b) : b);
 }
 
@@ -157,29 +152,26 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t ring = (raw_addr + 1023u) & ~1023u;              // swizzle atoms need 1024-byte alignment
     TcControl* ctl = reinterpret_cast<TcControl*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes);
-    const uint32_t rank = ptx::cluster_ctarank();                   // 0 = leader of the pair, 1 = peer
 
     // ---- set-up that needs nothing from earlier kernels: overlaps their tail ----
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_bar[s]), 1 + kGatherThreads);
-            ptx::mbar_init(ptx::smem_addr(&ctl->peer_full[s]), 1);
             ptx::mbar_init(ptx::smem_addr(&ctl->empty_bar[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[a]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 8);
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 4);
         }
         ctl->abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&map_w);
         ptx::prefetch_tensormap(&map_x);
     }
-    if (warp == 5) ptx::tmem_alloc_pair(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
+    if (warp == 5) ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_sync_all();                                         // both CTAs' barriers exist before any remote arrival
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctl->tmem_slot);
     volatile int* abort_flag = &ctl->abort_flag;
@@ -208,17 +200,15 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     if (!ok) break;
                     const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
                     const uint32_t a_dst = ring + s * kStageBytes;
-                    if (t.is_dw) {                                   // this CTA's half of the X_keep tile: 64-column blocks x 64 kept rows
-                        const int row0 = (int)((t.kb_begin + k) * kBK);
-                        const int i0 = (int)(t.col_tile * BNW) + (int)rank * (BNW / 2);
-                        ptx::mbar_arrive_expect_tx(full, (BNW / 2) * kRowBytes);
+                    if (t.is_dw) {                                   // X_keep tile: BNW/64 blocks of 64 columns x 64 kept rows
+                        const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.col_tile * BNW);
+                        ptx::mbar_arrive_expect_tx(full, BNW * kRowBytes);
 #pragma unroll
-                        for (int b = 0; b < BNW / 128; ++b)
+                        for (int b = 0; b < BNW / 64; ++b)
                             ptx::tma_load_2d(a_dst + kABytes + b * kBlock64Bytes, &map_x, i0 + b * 64, row0, full);
-                    } else {                                         // this CTA's half of the W tile: BNX/2 rows x 64 columns
-                        ptx::mbar_arrive_expect_tx(full, (BNX / 2) * kRowBytes);
-                        ptx::tma_load_2d(a_dst + kABytes, &map_w, (int)(k * kBK),
-                                         (int)(t.col_tile * BNX) + (int)rank * (BNX / 2), full);
+                    } else {                                         // W tile: BNX rows x 64 columns
+                        ptx::mbar_arrive_expect_tx(full, BNX * kRowBytes);
+                        ptx::tma_load_2d(a_dst + kABytes, &map_w, (int)(k * kBK), (int)(t.col_tile * BNX), full);
                     }
                 }
             }
@@ -232,8 +222,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         }
         __syncwarp();
     } else if (warp == 5) {
-        // ---------------- leader: MMA issuer; peer: tells the leader when its half of a stage is full ----------------
-        if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
             uint32_t it = 0, used = 0;                               // stage uses, accumulator uses
             bool ok = true;
             for (uint32_t pass = 0; ok; ++pass) {
@@ -242,20 +232,19 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const Tile t = decode_tile(sched, q);
                 if (t.num_kb == 0) continue;
                 const uint32_t acc = used & 1u;
-                ok = ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->acc_empty[acc]), ((used >> 1) & 1u) ^ 1u, abort_flag, status_word);
+                ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[acc]), ((used >> 1) & 1u) ^ 1u, abort_flag, status_word);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * kAccCols;
                 // K-major (dX): a 16-deep slice is 32 bytes along the swizzled row, 8-row groups 1024 B apart.
                 // MN-major (dW): a 16-deep slice is 16 rows (two atoms); 64-wide blocks of the MN extent 8 KB apart.
-                const uint32_t idesc = t.is_dw ? ptx::umma_idesc_bf16(kPairM, BNW, true, true)
-                                               : ptx::umma_idesc_bf16(kPairM, BNX, false, false);
+                const uint32_t idesc = t.is_dw ? ptx::umma_idesc_bf16(kBM, BNW, true, true)
+                                               : ptx::umma_idesc_bf16(kBM, BNX, false, false);
                 const uint32_t k_step = t.is_dw ? kUmmaK * kRowBytes : kUmmaK * 2;
                 const uint32_t lbo = t.is_dw ? kBlock64Bytes : 16;
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
                     const int s = it % kStages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / kStages) & 1u, abort_flag, status_word) &&
-                         ptx::mbar_wait_cluster(ptx::smem_addr(&ctl->peer_full[s]), (it / kStages) & 1u, abort_flag, status_word);
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / kStages) & 1u, abort_flag, status_word);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     ptx::fence_async_proxy();        // the gathered operand was written by cp.async (generic proxy)
@@ -264,28 +253,12 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     for (uint32_t u = 0; u < kBK / kUmmaK; ++u) {
                         const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, kAtomBytes);
                         const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, kAtomBytes);
-                        ptx::umma_bf16_pair(d_tmem, da, db, idesc, (k | u) != 0u);
+                        ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
                     }
-                    ptx::umma_commit_pair(ptx::smem_addr(&ctl->empty_bar[s]), 3);   // both CTAs may refill the stage
+                    ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));      // stage reusable once these MMAs retire
                 }
-                if (ok) ptx::umma_commit_pair(ptx::smem_addr(&ctl->acc_full[acc]), 3);
+                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
                 ++used;
-            }
-        } else if (lane == 0) {
-            const uint32_t leader_peer_full = ptx::map_to_cta(ptx::smem_addr(&ctl->peer_full[0]), 0);
-            uint32_t it = 0;
-            bool ok = true;
-            for (uint32_t pass = 0; ok; ++pass) {
-                const uint32_t q = list_position(pass);
-                if (q >= sched.total) break;
-                const Tile t = decode_tile(sched, q);
-                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
-                    const int s = it % kStages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / kStages) & 1u, abort_flag, status_word);
-                    if (!ok) break;
-                    ptx::fence_async_proxy();        // this CTA's cp.async writes, before the tensor core reads them
-                    ptx::mbar_arrive_remote(leader_peer_full + (uint32_t)s * 8u);
-                }
             }
         }
         __syncwarp();
@@ -302,7 +275,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 // dX tile: 128 kept rows x 128 bytes per stage; one warp instruction moves 4 rows x 128 B
                 constexpr int kInstr = 32 / kGatherWarps;
                 const uint32_t chunk = lane & 7, sub = lane >> 3;
-                const int64_t m0 = (int64_t)t.row_tile * kPairM + rank * kBM;
+                const int64_t m0 = (int64_t)t.row_tile * kBM;
                 const __nv_bfloat16* src[kInstr];
 #pragma unroll
                 for (int i = 0; i < kInstr; ++i) {
@@ -333,7 +306,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 constexpr int kAhead = 4;                            // row ids are fetched this many stages early
                 const uint32_t c = lane & 15;                        // 16-byte chunk within the 256-byte row piece
                 const uint32_t sub = lane >> 4;                      // which of the two rows of this instruction
-                const int col = (int)(t.row_tile * kPairM + rank * kBM) + (int)c * 8;
+                const int col = (int)(t.row_tile * kBM) + (int)c * 8;
                 const bool col_ok = col < C_out;                     // columns past C_out read as zero
                 const __nv_bfloat16* col_ptr = p.dY + (col_ok ? col : 0);
                 int nxt[kAhead][kIdxPerLane];
@@ -456,7 +429,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const int n0 = (int)(t.col_tile * BNX);
                 const int strip_cols = (C_in - n0 < BNX) ? C_in - n0 : BNX;   // multiple of 8
                 const int strip_vecs = strip_cols >> 3;
-                const int64_t m0 = (int64_t)t.row_tile * kPairM + rank * kBM;
+                const int64_t m0 = (int64_t)t.row_tile * kBM;
                 const int64_t m = m0 + warp * 32 + lane;
                 const bool valid = m < M_keep;
                 const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
@@ -525,7 +498,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             } else {
                 // ---- dW tile: accumulator row = output column j, accumulator column = output row i ----
                 // a warp-wide store of one accumulator column covers 32 consecutive j: 128 contiguous bytes
-                const int j = (int)(t.row_tile * kPairM + rank * kBM) + warp * 32 + lane;
+                const int j = (int)(t.row_tile * kBM) + warp * 32 + lane;
                 const int i0 = (int)(t.col_tile * BNW);
                 float* out_col = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i0 * C_out + j;
                 if (t.num_kb == 0) {                                 // a piece without kept rows contributes zero
@@ -562,19 +535,15 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
             // this warp is done with the accumulator: hand it back to the MMA issuer
             ptx::tc_fence_before_sync();
-            if (lane == 0) {
-                if (rank == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
-                else ptx::mbar_arrive_remote(ptx::map_to_cta(ptx::smem_addr(&ctl->acc_empty[acc]), 0));
-            }
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
             ++used;
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_sync_all();        // nobody of the pair still signals the other's barriers or reads its operands
     if (warp == 5) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc_pair(tmem_base, 2 * kAccCols);
+        ptx::tmem_dealloc(tmem_base, 2 * kAccCols);
     }
 }
 
@@ -613,23 +582,23 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, ui
 struct Plan {
     int bnx, bnw;          // accumulator width of dX / dW tiles
     int splits;            // pieces each dW tile's reduction over kept rows is cut into
-    int64_t tiles;         // upper bound of the pair-tile count (from the capacity)
+    int64_t tiles;         // upper bound of the tile count (from the capacity)
 };
 
 Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
     Plan pl;
     pl.bnx = (C_in >= 256) ? 256 : 128;
     pl.bnw = (C_in >= 256) ? 256 : 128;
-    const int64_t x_tiles = want_dx ? ((M_keep_cap + kPairM - 1) / kPairM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
+    const int64_t x_tiles = want_dx ? ((M_keep_cap + kBM - 1) / kBM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
     const int64_t x_kb = (C_out + kBK - 1) / kBK;
-    const int64_t w_tiles = want_dw ? ((C_out + kPairM - 1) / kPairM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
+    const int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
     const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
     // Cut the dW reductions so that one piece is no longer than an even share of all the work
     // (in k-block units; a BN=128 tile's unit is cheaper, which only makes the cut finer).
     pl.splits = 1;
     if (want_dw) {
         const int64_t units = x_tiles * x_kb + w_tiles * w_kb;
-        int64_t share = (units + kNumSMs / 2 - 1) / (kNumSMs / 2);      // per CTA pair
+        int64_t share = (units + kNumSMs - 1) / kNumSMs;
         if (share < 16) share = 16;
         int64_t s = (w_kb + share - 1) / share;
         if (s > 64) s = 64;
@@ -641,40 +610,13 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     return pl;
 }
 
-// How many CTA pairs the device can keep resident at once (a pair needs two SMs of one cluster-capable group).
 template <int BNX, int BNW>
-int max_resident_pairs() {
-    static int pairs = [] {
-        if (cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSmemBytes) != cudaSuccess)
-            return 0;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kNumSMs);
-        cfg.blockDim = dim3(kTcThreads);
-        cfg.dynamicSmemBytes = kSmemBytes;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, tc_backward_kernel<BNX, BNW>, &cfg) != cudaSuccess) return 0;
-        return n < kNumSMs / 2 ? n : kNumSMs / 2;
-    }();
-    return pairs;
-}
-
-template <int BNX, int BNW>
-cudaError_t launch_fused(int64_t pair_tiles, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
-                         const TcParams& prm, int* ctas_out) {
-    int pairs = max_resident_pairs<BNX, BNW>();
-    if (pairs < 1) return cudaErrorLaunchOutOfResources;
-    if (pair_tiles < pairs) pairs = (int)(pair_tiles < 1 ? 1 : pair_tiles);
-    *ctas_out = 2 * pairs;
-    return launch_pdl_cluster(tc_backward_kernel<BNX, BNW>, dim3(2 * pairs), dim3(kTcThreads), kSmemBytes, 2, stream,
-                              map_w, map_x, prm);
+cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
+                         const TcParams& prm) {
+    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (once != cudaSuccess) return once;
+    return launch_pdl(tc_backward_kernel<BNX, BNW>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x, prm);
 }
 
 }  // namespace
@@ -709,10 +651,8 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     // a product that is not requested still gets a valid map (of the other matrix): it is never used
     const void* w_base = want_dx ? W : X_keep;
     const void* x_base = want_dw ? X_keep : W;
-    // W is loaded in boxes of bnx/2 rows (each CTA of a pair fetches half of the tile), X_keep in 64 x 64 boxes
-    const uint32_t w_box = (uint32_t)pl.bnx / 2;
-    if (!make_map(&map_w, w_base, want_dx ? C_in : M_keep_cap, want_dx ? C_out : C_in, want_dx ? w_box : 64u) ||
-        !make_map(&map_x, x_base, want_dw ? M_keep_cap : C_in, want_dw ? C_in : C_out, want_dw ? 64u : w_box))
+    if (!make_map(&map_w, w_base, want_dx ? C_in : M_keep_cap, want_dx ? C_out : C_in, want_dx ? (uint32_t)pl.bnx : 64u) ||
+        !make_map(&map_x, x_base, want_dw ? M_keep_cap : C_in, want_dw ? C_in : C_out, want_dw ? 64u : (uint32_t)pl.bnx))
         return SBP_ERR_CUDA;
     TcParams prm;
     prm.dY = static_cast<const __nv_bfloat16*>(dY);
@@ -729,18 +669,20 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     prm.dw_accumulate = (pl.splits == 1 && accumulate) ? 1 : 0;
     prm.db_partial = (db != nullptr) ? db_workspace : nullptr;
     prm.status_word = status_word;
-    int ctas = 0;
+    int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
+    if (ctas < 1) ctas = 1;
+    const dim3 grid((unsigned)ctas);
     cudaError_t e;
-    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(pl.tiles, stream, map_w, map_x, prm, &ctas);
-    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(pl.tiles, stream, map_w, map_x, prm, &ctas);
-    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(pl.tiles, stream, map_w, map_x, prm, &ctas);
-    else e = launch_fused<128, 128>(pl.tiles, stream, map_w, map_x, prm, &ctas);
+    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, prm);
+    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, prm);
+    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, prm);
+    else e = launch_fused<128, 128>(grid, stream, map_w, map_x, prm);
     if (e != cudaSuccess) return SBP_ERR_CUDA;
     if (want_dw && pl.splits > 1 &&
         launch_reduce_partials(workspace, pl.splits, C_in * C_out, dW, accumulate, status_word, stream) != cudaSuccess)
         return SBP_ERR_CUDA;
     if (db != nullptr &&
-        launch_reduce_partials(db_workspace, ctas, C_out, db, accumulate, status_word, stream) != cudaSuccess)
+        launch_reduce_partials(db_workspace, (int)ctas, C_out, db, accumulate, status_word, stream) != cudaSuccess)
         return SBP_ERR_CUDA;
     return SBP_OK;
 }
