@@ -143,6 +143,137 @@ sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint
     }
 }
 
+// ---- large maps: one sample spread over a cluster of C thread blocks ----
+// Each block owns a contiguous slice of the positions.  The per-pass digit histograms stay in the
+// blocks' shared memory and are summed through distributed shared memory, so every block derives
+// the same threshold; slice counts exchanged the same way give each block its output offset.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_load(const uint32_t* local_ptr, uint32_t rank) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(local_ptr);
+    uint32_t ra, v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+template <int C>
+__global__ void __launch_bounds__(kSampThreads)
+sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint32_t step,
+                                  uint32_t first_sample, int share_mask,
+                                  int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
+    __shared__ SampShared sh;
+    __shared__ uint32_t slice_counts[2];          // positions of this slice below / equal to the threshold
+    pdl_launch_dependents();
+    pdl_wait();
+    const uint32_t rank = cluster_rank();
+    const uint32_t b = blockIdx.x / C;
+    const uint32_t gid = share_mask ? 0u : first_sample + b;
+    const uint32_t groups = (N + 3u) >> 2;
+    const uint32_t per = (groups + C - 1) / C;
+    const uint32_t g_begin = rank * per;
+    const uint32_t g_end = (g_begin + per < groups) ? g_begin + per : groups;
+    const int64_t row_base = (int64_t)b * N;
+    int32_t* out = keep_rows + (int64_t)b * K;
+    if (rank == 0 && threadIdx.x == 0) {
+        keep_offsets[b + 1] = (int32_t)((b + 1) * (int64_t)K);
+        if (b == 0) keep_offsets[0] = 0;
+    }
+
+    uint32_t prefix = 0, known = 0, remaining = K;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += kSampThreads) sh.hist[i] = 0;
+        __syncthreads();
+        for (uint32_t q = g_begin + threadIdx.x; q < g_end; q += kSampThreads) {
+            const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t n = 4u * q + e;
+                if (n < N && (pw.w[e] & known) == prefix) atomicAdd(&sh.hist[(pw.w[e] >> shift) & 0xffu], 1u);
+            }
+        }
+        cluster_sync();                                   // every slice's histogram is complete
+        uint32_t cnt = 0;
+        if (threadIdx.x < 256)
+            for (uint32_t r = 0; r < (uint32_t)C; ++r) cnt += cluster_load(&sh.hist[threadIdx.x], r);
+        const uint2 sc = block_excl_scan(cnt, sh.warp_sums_a);
+        if (threadIdx.x < 256 && sc.x < remaining && remaining <= sc.x + cnt) {
+            sh.sel_digit = threadIdx.x;
+            sh.sel_below = sc.x;
+        }
+        __syncthreads();
+        prefix |= sh.sel_digit << shift;
+        known |= 0xffu << shift;
+        remaining -= sh.sel_below;
+        cluster_sync();                                   // nobody still reads a histogram that is about to be cleared
+    }
+    const uint32_t threshold = prefix;
+
+    // slice counts -> rank of this slice's first tie and its first output slot
+    uint32_t lt = 0, eq = 0;
+    for (uint32_t q = g_begin + threadIdx.x; q < g_end; q += kSampThreads) {
+        const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (4u * q + e < N) {
+                lt += pw.w[e] < threshold;
+                eq += pw.w[e] == threshold;
+            }
+        }
+    }
+    const uint32_t lt_total = block_excl_scan(lt, sh.warp_sums_a).y;
+    const uint32_t eq_total = block_excl_scan(eq, sh.warp_sums_b).y;
+    if (threadIdx.x == 0) { slice_counts[0] = lt_total; slice_counts[1] = eq_total; }
+    cluster_sync();
+    uint32_t eq_seen = 0, written = 0;
+    for (uint32_t r = 0; r < rank; ++r) {
+        const uint32_t lt_r = cluster_load(&slice_counts[0], r), eq_r = cluster_load(&slice_counts[1], r);
+        const uint32_t room = remaining > eq_seen ? remaining - eq_seen : 0u;
+        written += lt_r + (eq_r < room ? eq_r : room);
+        eq_seen += eq_r;
+    }
+
+    // ordered compaction of this slice
+    for (uint32_t q0 = g_begin; q0 < g_end; q0 += kSampThreads) {
+        const uint32_t q = q0 + threadIdx.x;
+        uint32_t lt_mask = 0, eq_mask = 0;
+        if (q < g_end) {
+            const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (4u * q + e < N) {
+                    if (pw.w[e] < threshold) lt_mask |= 1u << e;
+                    else if (pw.w[e] == threshold) eq_mask |= 1u << e;
+                }
+            }
+        }
+        uint32_t keep_mask = lt_mask;
+        const uint2 se = block_excl_scan(__popc(eq_mask), sh.warp_sums_a);
+        uint32_t tie_rank = eq_seen + se.x;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (eq_mask & (1u << e)) {
+                if (tie_rank < remaining) keep_mask |= 1u << e;
+                ++tie_rank;
+            }
+        }
+        eq_seen += se.y;
+        const uint2 sk = block_excl_scan(__popc(keep_mask), sh.warp_sums_b);
+        uint32_t pos = written + sk.x;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (keep_mask & (1u << e)) out[pos++] = (int32_t)(row_base + 4u * q + e);
+        written += sk.y;
+    }
+    cluster_sync();                                       // the slice counts stay readable until every block is done
+}
+
 // ---- grid-wise masks: 2x2-periodic lattice with a per-sample phase ----
 __device__ __forceinline__ uint32_t grid_phase(int family, uint32_t gid, uint32_t step, uint32_t k0, uint32_t k1) {
     if (family == 4) return 0u;
@@ -233,9 +364,27 @@ cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, 
                                int32_t* keep_rows, int32_t* keep_offsets, cudaStream_t stream) {
     const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
     const dim3 grid((unsigned)B), block(kSampThreads);
-    if (mode == SBP_MASK_RANDOM)
+    if (mode == SBP_MASK_RANDOM) {
+        const int64_t N = H * W;
+        // large maps with few samples: spread each sample over a cluster so that more SMs take part
+        int cluster = 1;
+        if (K < N && N > 8192 && B * 8 <= 4 * kNumSMs) cluster = N > 32768 ? 8 : (N > 16384 ? 4 : 2);
+        const dim3 cgrid((unsigned)(B * cluster));
+        switch (cluster) {
+            case 8:
+                return launch_pdl_cluster(sample_keep_random_cluster_kernel<8>, cgrid, block, 0, 8, stream, (uint32_t)N,
+                                          (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
+            case 4:
+                return launch_pdl_cluster(sample_keep_random_cluster_kernel<4>, cgrid, block, 0, 4, stream, (uint32_t)N,
+                                          (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
+            case 2:
+                return launch_pdl_cluster(sample_keep_random_cluster_kernel<2>, cgrid, block, 0, 2, stream, (uint32_t)N,
+                                          (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
+            default: break;
+        }
         return launch_pdl(sample_keep_random_kernel, grid, block, 0, stream, (uint32_t)(H * W), (uint32_t)K, k0, k1,
                           step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
+    }
     return launch_pdl(sample_keep_grid_kernel, grid, block, 0, stream, grid_family, (uint32_t)H, (uint32_t)W, k0, k1,
                       step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
 }

@@ -29,6 +29,9 @@ def relerr(got, want):
     (0, 4, 14, 14, 1.0, 1, 1, 0, 0),
     (0, 3, 56, 56, 0.5, 2, 0, 0, 0),                     # several sweeps of the block
     (0, 2, 200, 334, 0.5, 0, 0, 0, 0),                   # detection-resolution map
+    (0, 3, 100, 100, 0.5, 4, 1, 0, 0),                   # one sample over a cluster of 2 blocks
+    (0, 2, 128, 160, 0.25, 5, 2, 9, 0),                  # ... of 4 blocks
+    (0, 1, 181, 181, 0.75, 6, 0, 0, sbp.SBP_FLAG_SHARE_MASK),   # ... of 8 blocks, ragged slices
     (0, 7, 1, 1, 0.5, 3, 0, 0, 0),
     (0, 3, 3, 3, 0.01, 3, 0, 0, 0),
     (0, 6, 9, 11, 0.5, 4, 2, 5, sbp.SBP_FLAG_SHARE_MASK),
