@@ -44,7 +44,9 @@ constexpr uint32_t kABytes = kBM * kRowBytes;        // 16 KB
 constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
 constexpr uint32_t kAccCols = 256;       // TMEM columns per accumulator buffer (two buffers = all 512)
-constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float);   // cross-row-group sums of the bias warps
+constexpr int kBiasChunk = 64;           // kept rows whose ids the bias warps stage at a time
+constexpr int kBiasDepth = 16;           // 16-byte loads each bias thread keeps in flight
+constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float) + kBiasChunk * sizeof(int);   // cross-row-group sums + staged row ids
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kBiasSmemBytes + 1024;   // ring + control + bias + slack
 
 struct TcControl {
@@ -365,31 +367,35 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             const int64_t m_end = (m_begin + rows_per < M_keep) ? m_begin + rows_per : M_keep;
             const uint4* dY4 = reinterpret_cast<const uint4*>(p.dY);
             float* out = p.db_partial + (int64_t)blockIdx.x * C_out;
+            int* ids = reinterpret_cast<int*>(red + kBiasThreads * 8);  // row ids of the current chunk of kept rows
             for (int cv0 = 0; cv0 < V; cv0 += VT) {
                 const int cv = cv0 + cvt;
                 float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                if (cv < V) {
-                    for (int64_t m = m_begin + rg; m < m_end; m += (int64_t)RG * 8) {
-                        int64_t row[8];
-                        uint4 v[8];
+                for (int64_t mc = m_begin; mc < m_end; mc += kBiasChunk) {
+                    // stage the chunk's row ids once, so that the dY loads below depend on no other load
+                    if (t < kBiasChunk) ids[t] = (mc + t < m_end) ? __ldg(p.keep_rows + mc + t) : -1;
+                    asm volatile("bar.sync 1, %0;" ::"n"(kBiasThreads) : "memory");
+                    if (cv < V) {
+                        for (int r0 = rg; r0 < kBiasChunk; r0 += RG * kBiasDepth) {
+                            uint4 v[kBiasDepth];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const int64_t mm = m + (int64_t)u * RG;
-                            row[u] = (mm < m_end) ? (int64_t)__ldg(p.keep_rows + mm) : -1;
-                        }
+                            for (int u = 0; u < kBiasDepth; ++u) {
+                                const int r = r0 + u * RG;
+                                const int row = (r < kBiasChunk) ? ids[r] : -1;
+                                v[u] = (row >= 0) ? __ldg(dY4 + (int64_t)row * V + cv) : make_uint4(0u, 0u, 0u, 0u);
+                            }
 #pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            v[u] = (row[u] >= 0) ? __ldg(dY4 + row[u] * V + cv) : make_uint4(0u, 0u, 0u, 0u);
+                            for (int u = 0; u < kBiasDepth; ++u) {
+                                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                acc[2 * e] += __uint_as_float(w[e] << 16);
-                                acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                                for (int e = 0; e < 4; ++e) {
+                                    acc[2 * e] += __uint_as_float(w[e] << 16);
+                                    acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                                }
                             }
                         }
                     }
+                    asm volatile("bar.sync 1, %0;" ::"n"(kBiasThreads) : "memory");
                 }
                 // add the row groups in a fixed order
 #pragma unroll
@@ -510,14 +516,20 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
+                // The two cases are separate loops of explicit stores on purpose: written as one conditional
+                // expression the compiler reads the old value in both cases, and a plain write then waits
+                // for a load of memory it is about to overwrite.
+                const bool add_in = p.dw_accumulate != 0;
                 auto store_cols = [&](const float (&v)[32], int c0) {    // 32 accumulator columns = 32 rows of dW
                     if (j >= C_out) return;
+                    if (add_in) {
 #pragma unroll
-                    for (int r = 0; r < 32; ++r) {
-                        if (i0 + c0 + r < C_in) {
-                            float* dst = out_col + (int64_t)(c0 + r) * C_out;
-                            *dst = p.dw_accumulate ? *dst + v[r] : v[r];
-                        }
+                        for (int r = 0; r < 32; ++r)
+                            if (i0 + c0 + r < C_in) out_col[(int64_t)(c0 + r) * C_out] += v[r];
+                    } else {
+#pragma unroll
+                        for (int r = 0; r < 32; ++r)
+                            if (i0 + c0 + r < C_in) ptx::st_global_f32(out_col + (int64_t)(c0 + r) * C_out, v[r]);
                     }
                 };
                 float va[32], vb[32];
