@@ -103,50 +103,94 @@ db_partial_kernel(const uint4* __restrict__ dY, uint32_t col_vecs, const int32_t
     }
 }
 
-// few partials: one thread per float4 of the output, partials added in ascending order
-__global__ void __launch_bounds__(256)
-reduce_partials_flat_kernel(const float4* __restrict__ partials, int splits, int64_t n_vec, float4* __restrict__ out,
-                            int accumulate, const int32_t* __restrict__ status_word) {
-    pdl_launch_dependents();
-    pdl_wait();
-    if (status_word != nullptr && *status_word != 0) return;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
-        float4 s = accumulate ? out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int k = 0; k < splits; ++k) {
-            const float4 p = __ldg(partials + (int64_t)k * n_vec + i);
-            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
-        }
-        out[i] = s;
-    }
-}
+// ---- deterministic reduction of [splits, n] partial results ------------------------------------
+// One launch serves up to two reductions (the split partials of dW and the per-block partials of
+// db of one backward call): the first a.blocks blocks work on job a, the rest on job b.
+struct ReduceJob {
+    const float4* partials;
+    float4* out;
+    int64_t n_vec;        // float4 elements per partial
+    int splits;
+    int accumulate;
+    int deep;             // 0: one thread per float4, partials added in ascending order
+                          // 1: 8 float4 columns x 32 row lanes per block; lane y adds partials y, y+32, ...
+                          //    in ascending order, the 32 lane sums are then added in lane order
+    int blocks;
+};
 
-// many partials: 32 float4 columns x 8 interleaved partial lanes per block; each lane adds its
-// partials in ascending order, the eight lane sums are then added in lane order
-__global__ void __launch_bounds__(256)
-reduce_partials_deep_kernel(const float4* __restrict__ partials, int splits, int64_t n_vec, float4* __restrict__ out,
-                            int accumulate, const int32_t* __restrict__ status_word) {
-    __shared__ float4 red[8][32];
-    pdl_launch_dependents();
-    pdl_wait();
-    if (status_word != nullptr && *status_word != 0) return;
-    const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
-    const int64_t i = (int64_t)blockIdx.x * 32 + x;
+__device__ __forceinline__ void add4(float4& s, const float4& p) { s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w; }
+
+__device__ __forceinline__ void run_reduce_job(const ReduceJob& jb, int block, float4 (*red)[8]) {
+    if (!jb.deep) {
+        const int64_t stride = (int64_t)jb.blocks * blockDim.x;
+        for (int64_t i = (int64_t)block * blockDim.x + threadIdx.x; i < jb.n_vec; i += stride) {
+            float4 s = jb.accumulate ? jb.out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k0 = 0; k0 < jb.splits; k0 += 4) {           // four independent loads in flight
+                float4 p[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    p[u] = (k0 + u < jb.splits) ? __ldg(jb.partials + (int64_t)(k0 + u) * jb.n_vec + i)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (k0 + u < jb.splits) add4(s, p[u]);
+            }
+            jb.out[i] = s;
+        }
+        return;
+    }
+    const int x = threadIdx.x & 7, y = threadIdx.x >> 3;
+    const int64_t i = (int64_t)block * 8 + x;
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (i < n_vec) {
-        for (int k = y; k < splits; k += 8) {
-            const float4 p = __ldg(partials + (int64_t)k * n_vec + i);
-            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+    if (i < jb.n_vec) {
+        for (int k0 = y; k0 < jb.splits; k0 += 32 * 4) {
+            float4 p[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                p[u] = (k0 + 32 * u < jb.splits) ? __ldg(jb.partials + (int64_t)(k0 + 32 * u) * jb.n_vec + i)
+                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (k0 + 32 * u < jb.splits) add4(s, p[u]);
         }
     }
     red[y][x] = s;
     __syncthreads();
-    if (y == 0 && i < n_vec) {
-        float4 t = accumulate ? out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    if (y == 0 && i < jb.n_vec) {
+        float4 t = jb.accumulate ? jb.out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int w = 0; w < 8; ++w) { t.x += red[w][x].x; t.y += red[w][x].y; t.z += red[w][x].z; t.w += red[w][x].w; }
-        out[i] = t;
+        for (int w = 0; w < 32; ++w) add4(t, red[w][x]);
+        jb.out[i] = t;
     }
+}
+
+__global__ void __launch_bounds__(256)
+reduce_partials_kernel(const ReduceJob a, const ReduceJob b, const int32_t* __restrict__ status_word) {
+    __shared__ float4 red[32][8];
+    pdl_launch_dependents();
+    pdl_wait();
+    if (status_word != nullptr && *status_word != 0) return;
+    if ((int)blockIdx.x < a.blocks) run_reduce_job(a, (int)blockIdx.x, red);
+    else run_reduce_job(b, (int)blockIdx.x - a.blocks, red);
+}
+
+ReduceJob make_reduce_job(const float* partials, int splits, int64_t n, float* out, bool accumulate) {
+    ReduceJob jb;
+    jb.partials = reinterpret_cast<const float4*>(partials);
+    jb.out = reinterpret_cast<float4*>(out);
+    jb.n_vec = n / 4;             // n is a multiple of 4 for every caller
+    jb.splits = splits;
+    jb.accumulate = accumulate ? 1 : 0;
+    jb.deep = splits > 8 ? 1 : 0;
+    int64_t blocks;
+    if (jb.deep) {
+        blocks = (jb.n_vec + 7) / 8;
+    } else {
+        blocks = (jb.n_vec + 255) / 256;
+        if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
+    }
+    jb.blocks = (int)(blocks < 1 ? 1 : blocks);
+    return jb;
 }
 
 }  // namespace
@@ -176,17 +220,19 @@ cudaError_t launch_db(sbp_dtype dt, const void* dY, const int32_t* keep_rows, co
 
 cudaError_t launch_reduce_partials(const float* partials, int splits, int64_t n, float* out,
                                    bool accumulate, const int32_t* status_word, cudaStream_t stream) {
-    const int64_t n_vec = n / 4;   // n is a multiple of 4 for every caller
-    if (splits > 8) {
-        const int64_t blocks = (n_vec + 31) / 32;
-        return launch_pdl(reduce_partials_deep_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
-                          (const float4*)partials, splits, n_vec, (float4*)out, accumulate ? 1 : 0, status_word);
-    }
-    int64_t blocks = (n_vec + 255) / 256;
-    if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
-    if (blocks < 1) blocks = 1;
-    return launch_pdl(reduce_partials_flat_kernel, dim3((unsigned)blocks), dim3(256), 0, stream,
-                      (const float4*)partials, splits, n_vec, (float4*)out, accumulate ? 1 : 0, status_word);
+    const ReduceJob a = make_reduce_job(partials, splits, n, out, accumulate);
+    ReduceJob none = a;
+    none.blocks = 0;
+    return launch_pdl(reduce_partials_kernel, dim3((unsigned)a.blocks), dim3(256), 0, stream, a, none, status_word);
+}
+
+cudaError_t launch_reduce_partials_pair(const float* partials_a, int splits_a, int64_t n_a, float* out_a,
+                                        const float* partials_b, int splits_b, int64_t n_b, float* out_b,
+                                        bool accumulate, const int32_t* status_word, cudaStream_t stream) {
+    const ReduceJob a = make_reduce_job(partials_a, splits_a, n_a, out_a, accumulate);
+    const ReduceJob b = make_reduce_job(partials_b, splits_b, n_b, out_b, accumulate);
+    return launch_pdl(reduce_partials_kernel, dim3((unsigned)(a.blocks + b.blocks)), dim3(256), 0, stream, a, b,
+                      status_word);
 }
 
 }  // namespace sbp

@@ -125,6 +125,11 @@ cudaError_t launch_db(sbp_dtype dt, const void* dY, const int32_t* keep_rows, co
 cudaError_t launch_reduce_partials(const float* partials, int splits, int64_t n, float* out,
                                    bool accumulate, const int32_t* status_word, cudaStream_t stream);
 
+// two such reductions in one launch (both with the same accumulate setting)
+cudaError_t launch_reduce_partials_pair(const float* partials_a, int splits_a, int64_t n_a, float* out_a,
+                                        const float* partials_b, int splits_b, int64_t n_b, float* out_b,
+                                        bool accumulate, const int32_t* status_word, cudaStream_t stream);
+
 // plain-FMA (CUDA-core) products for fp32 and for bf16 shapes the tensor-core kernels do not take
 size_t simt_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 int    simt_dw_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out);

@@ -649,7 +649,8 @@ size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
 int tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx,
                              bool want_db) {
     if (!want_dw && !want_dx) return 0;
-    return 1 + ((want_dw && make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx).splits > 1) ? 1 : 0) + (want_db ? 1 : 0);
+    const bool reduce_dw = want_dw && make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx).splits > 1;
+    return 1 + ((reduce_dw || want_db) ? 1 : 0);       // the two reductions share one launch
 }
 
 sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
@@ -690,12 +691,16 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, prm);
     else e = launch_fused<128, 128>(grid, stream, map_w, map_x, prm);
     if (e != cudaSuccess) return SBP_ERR_CUDA;
-    if (want_dw && pl.splits > 1 &&
-        launch_reduce_partials(workspace, pl.splits, C_in * C_out, dW, accumulate, status_word, stream) != cudaSuccess)
-        return SBP_ERR_CUDA;
-    if (db != nullptr &&
-        launch_reduce_partials(db_workspace, (int)ctas, C_out, db, accumulate, status_word, stream) != cudaSuccess)
-        return SBP_ERR_CUDA;
+    const bool reduce_dw = want_dw && pl.splits > 1, reduce_db = db != nullptr;
+    cudaError_t r = cudaSuccess;
+    if (reduce_dw && reduce_db)
+        r = launch_reduce_partials_pair(workspace, pl.splits, C_in * C_out, dW, db_workspace, (int)ctas, C_out, db,
+                                        accumulate, status_word, stream);
+    else if (reduce_dw)
+        r = launch_reduce_partials(workspace, pl.splits, C_in * C_out, dW, accumulate, status_word, stream);
+    else if (reduce_db)
+        r = launch_reduce_partials(db_workspace, (int)ctas, C_out, db, accumulate, status_word, stream);
+    if (r != cudaSuccess) return SBP_ERR_CUDA;
     return SBP_OK;
 }
 
