@@ -22,6 +22,8 @@
 // Four more warps compute the bias gradient on the side: each CTA sums its share of the kept rows
 // of dY column-wise while the tensor pipe works (the kernel is latency-bound, not bandwidth-bound,
 // so the extra reads are free) and leaves one partial row per CTA for a fixed-order reduce.
+#include <mutex>
+
 #include "tc_ptx.cuh"
 
 namespace sbp {
@@ -47,7 +49,13 @@ constexpr uint32_t kAccCols = 256;       // TMEM columns per accumulator buffer 
 constexpr int kBiasChunk = 64;           // kept rows whose ids the bias warps stage at a time
 constexpr int kBiasDepth = 16;           // 16-byte loads each bias thread keeps in flight
 constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float) + kBiasChunk * sizeof(int);   // cross-row-group sums + staged row ids
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kBiasSmemBytes + 1024;   // ring + control + bias + slack
+constexpr int kEpiChunk = 16;            // accumulator columns (= rows of dW) per TMA store of the dW epilogue
+constexpr int kEpiBufs = 3;              // staging buffers the dW epilogue rotates through
+constexpr uint32_t kEpiBufBytes = kEpiChunk * kBM * sizeof(float);   // 8 KB: 16 rows of dW x 128 columns
+constexpr int kEpiBarrier = 2;           // named barrier of the four epilogue warps
+constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kBiasSmemBytes + kEpiBufs * kEpiBufBytes + 1024;   // ring + control + bias + staging + slack
+static_assert((256 + kBiasSmemBytes) % 128 == 0, "staging buffers start on a 128-byte boundary");
+static_assert(kSmemBytes <= 227 * 1024, "shared memory per block");
 
 struct TcControl {
     uint64_t full_bar[kStages];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
@@ -70,6 +78,7 @@ struct TcParams {
     int64_t dw_split_stride;       // elements between partial buffers
     int dw_splits;
     int dw_accumulate;             // add into dW_out (only with one split)
+    int dw_tma;                    // dW tiles leave through TMA stores (dW_out is 16-byte aligned)
     float* db_partial;             // nullptr: no bias sums; else [gridDim.x, C_out] per-CTA column sums of kept dY rows
     int32_t* status_word;
 };
@@ -148,7 +157,7 @@ __device__ __forceinline__ uint32_t swizzled(uint32_t row, uint32_t chunk) {
 template <int BNX, int BNW>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                   const TcParams p) {
+                   const __grid_constant__ CUtensorMap map_dw, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -422,7 +431,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             for (int64_t v = (int64_t)blockIdx.x * 128 + threadIdx.x; v < vecs; v += (int64_t)gridDim.x * 128)
                 ptx::st_global_v4(p.dX + v * 8, 0u, 0u, 0u, 0u);
         }
-        uint32_t used = 0;
+        uint32_t used = 0, staged = 0;                               // accumulator uses, staging-buffer uses
         bool ok = true;
         for (uint32_t pass = 0; ok; ++pass) {
             const uint32_t q = list_position(pass);
@@ -474,7 +483,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
                 }
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);            // the four epilogue warps go on, or give up, together
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 __nv_bfloat16* out_row = p.dX + (valid ? cur : 0) * C_in + n0;
@@ -513,7 +522,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     continue;
                 }
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);            // the four epilogue warps go on, or give up, together
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 // The two cases are separate loops of explicit stores on purpose: written as one conditional
@@ -532,17 +541,45 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             if (i0 + c0 + r < C_in) ptx::st_global_f32(out_col + (int64_t)(c0 + r) * C_out, v[r]);
                     }
                 };
-                float va[32], vb[32];
-                ptx::tmem_ld_32x32(taddr, va);
-                ptx::tmem_ld_wait();
+                if (p.dw_tma) {
+                    // 16 rows of dW x 128 columns at a time: registers -> staging buffer -> one TMA store (or
+                    // reduce-add), which clips at the edges of dW.  A buffer is rewritten three chunks later;
+                    // the issuing thread has by then waited for all but the newest store to have read theirs.
+                    const int j0 = (int)(t.row_tile * kBM);
+                    const int live = (C_in - i0 < BNW) ? C_in - i0 : BNW;
+                    const int chunks = (live + kEpiChunk - 1) / kEpiChunk;
+                    const uint32_t stage_off = (ring - raw_addr) + kStages * kStageBytes + 256 + kBiasSmemBytes;
+#pragma unroll 1
+                    for (int c = 0; c < chunks; ++c, ++staged) {
+                        float v[kEpiChunk];
+                        ptx::tmem_ld_32x16(taddr + (uint32_t)(c * kEpiChunk), v);
+                        ptx::tmem_ld_wait();
+                        const uint32_t buf_off = stage_off + (staged % kEpiBufs) * kEpiBufBytes;
+                        float* buf = reinterpret_cast<float*>(smem_raw + buf_off) + warp * 32 + lane;
 #pragma unroll
-                for (int c0 = 0; c0 < BNW; c0 += 64) {
-                    ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), vb);
-                    store_cols(va, c0);
+                        for (int r = 0; r < kEpiChunk; ++r) buf[r * kBM] = v[r];
+                        ptx::fence_async_proxy();
+                        if (threadIdx.x == 0) ptx::bulk_wait_read<1>();
+                        ptx::bar_named<kEpiBarrier, 128>();
+                        if (threadIdx.x == 0) {
+                            if (add_in) ptx::tma_reduce_add_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
+                            else ptx::tma_store_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
+                            ptx::bulk_commit();
+                        }
+                    }
+                } else {
+                    float va[32], vb[32];
+                    ptx::tmem_ld_32x32(taddr, va);
                     ptx::tmem_ld_wait();
-                    if (c0 + 64 < BNW) ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
-                    store_cols(vb, c0 + 32);
-                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int c0 = 0; c0 < BNW; c0 += 64) {
+                        ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), vb);
+                        store_cols(va, c0);
+                        ptx::tmem_ld_wait();
+                        if (c0 + 64 < BNW) ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
+                        store_cols(vb, c0 + 32);
+                        ptx::tmem_ld_wait();
+                    }
                 }
             }
             // this warp is done with the accumulator: hand it back to the MMA issuer
@@ -551,6 +588,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             ++used;
         }
     }
+    if (threadIdx.x == 0) ptx::bulk_wait_all();                      // the TMA stores of the dW epilogue have landed
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 5) {
@@ -591,11 +629,64 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 [splits, C_in, C_out] output of the dW tiles, box = 1 x 16 rows x 128 columns, no swizzle
+bool make_map_dw(CUtensorMap* map, const float* base, int64_t splits, int64_t C_in, int64_t C_out) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)C_out, (cuuint64_t)C_in, (cuuint64_t)splits};
+    const cuuint64_t strides[2] = {(cuuint64_t)C_out * 4, (cuuint64_t)C_in * (cuuint64_t)C_out * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)kBM, (cuuint32_t)kEpiChunk, 1};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, elem_strides,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct Plan {
     int bnx, bnw;          // accumulator width of dX / dW tiles
     int splits;            // pieces each dW tile's reduction over kept rows is cut into
     int64_t tiles;         // upper bound of the tile count (from the capacity)
 };
+
+// Estimated run time of the tile list for a given split count, in units of one dX k-block: the
+// longest per-block total under the kernel's own static assignment (block b takes list positions
+// b, 2G-1-b, 2G+b, ...), the epilogue of that block's last tile, and the reduce launch that
+// splitting costs.  The weights are measured ratios on ViT-B shapes; they only rank candidates.
+double estimate_cost(int64_t x_tiles, int64_t x_kb, int64_t w_tiles, int64_t w_kb, int64_t splits, int64_t dw_elems) {
+    constexpr double kDwKb = 1.12;        // a dW k-block (two gathered MN-major operands) relative to a dX one
+    constexpr double kTileSwitch = 0.5;   // per tile: pipeline hand-over
+    constexpr double kTailDx = 9.0, kTailDw = 6.0;   // exposed epilogue of the last tile
+    const int64_t kb_per = (w_kb + splits - 1) / splits;
+    const int64_t w_pieces = w_tiles * splits;
+    const int64_t total = x_tiles + w_pieces;
+    if (total == 0) return 0.0;
+    const int64_t G = total < kNumSMs ? total : kNumSMs;
+    const bool w_first = kb_per >= x_kb;
+    const int64_t first = w_first ? w_pieces : x_tiles;
+    double worst = 0.0;
+    for (int64_t b = 0; b < G; ++b) {
+        double sum = 0.0, tail = 0.0;
+        for (int64_t pass = 0;; ++pass) {
+            const int64_t q = pass * G + ((pass & 1) ? (G - 1 - b) : b);
+            if (q >= total) break;
+            const bool is_dw = (q < first) == w_first;
+            if (is_dw) {
+                const int64_t split = (q < first ? q : q - first) % splits;
+                int64_t n = w_kb - kb_per * split;
+                if (n > kb_per) n = kb_per;
+                if (n < 0) n = 0;
+                sum += kDwKb * (double)n + kTileSwitch;
+                tail = kTailDw;
+            } else {
+                sum += (double)x_kb + kTileSwitch;
+                tail = kTailDx;
+            }
+        }
+        if (sum + tail > worst) worst = sum + tail;
+    }
+    if (splits > 1) worst += 7.0 + (double)(splits + 1) * (double)dw_elems * 4.0 / 1.7e6;   // launch + traffic of the reduce
+    return worst;
+}
 
 Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
     Plan pl;
@@ -605,18 +696,37 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     const int64_t x_kb = (C_out + kBK - 1) / kBK;
     const int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
     const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
-    // Cut the dW reductions so that one piece is no longer than an even share of all the work
-    // (in k-block units; a BN=128 tile's unit is cheaper, which only makes the cut finer).
     pl.splits = 1;
     if (want_dw) {
-        const int64_t units = x_tiles * x_kb + w_tiles * w_kb;
-        int64_t share = (units + kNumSMs - 1) / kNumSMs;
-        if (share < 16) share = 16;
-        int64_t s = (w_kb + share - 1) / share;
-        if (s > 64) s = 64;
-        if (s > w_kb) s = w_kb;
-        if (s < 1) s = 1;
-        pl.splits = (int)s;
+        // the same answer for the same shape: remember the last few shapes instead of searching on every call
+        struct Memo { int64_t cap, ci, co; int flags, splits; };
+        static Memo memo[8];
+        static int memo_next = 0;
+        static std::mutex memo_mutex;
+        const int flags = want_dx ? 1 : 0;
+        bool known = false;
+        {
+            std::lock_guard<std::mutex> lock(memo_mutex);
+            for (const Memo& m : memo)
+                if (m.splits > 0 && m.cap == M_keep_cap && m.ci == C_in && m.co == C_out && m.flags == flags) {
+                    pl.splits = m.splits;
+                    known = true;
+                }
+        }
+        if (!known) {
+            int64_t max_s = w_kb < 64 ? w_kb : 64;
+            if (max_s < 1) max_s = 1;
+            // the search walks every tile: with very many tiles any cut balances, so bound the work
+            while (max_s > 1 && (x_tiles + w_tiles * max_s) * max_s > (1 << 22)) max_s /= 2;
+            double best = 0.0;
+            for (int64_t sp = 1; sp <= max_s; ++sp) {
+                const double c = estimate_cost(x_tiles, x_kb, w_tiles, w_kb, sp, C_in * C_out);
+                if (sp == 1 || c < best * 0.995) { best = c; pl.splits = (int)sp; }
+            }
+            std::lock_guard<std::mutex> lock(memo_mutex);
+            memo[memo_next] = Memo{M_keep_cap, C_in, C_out, flags, pl.splits};
+            memo_next = (memo_next + 1) % 8;
+        }
     }
     pl.tiles = x_tiles + w_tiles * pl.splits;
     return pl;
@@ -624,11 +734,11 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
 
 template <int BNX, int BNW>
 cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
-                         const TcParams& prm) {
+                         const CUtensorMap& map_dw, const TcParams& prm) {
     static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW>,
                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (once != cudaSuccess) return once;
-    return launch_pdl(tc_backward_kernel<BNX, BNW>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x, prm);
+    return launch_pdl(tc_backward_kernel<BNX, BNW>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x, map_dw, prm);
 }
 
 }  // namespace
@@ -660,7 +770,7 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     const bool want_dw = dW != nullptr, want_dx = dX != nullptr;
     if (!want_dw && !want_dx) return SBP_OK;
     const Plan pl = make_plan(M_keep_cap, C_in, C_out, want_dw, want_dx);
-    CUtensorMap map_w, map_x;
+    CUtensorMap map_w, map_x, map_dw;
     // a product that is not requested still gets a valid map (of the other matrix): it is never used
     const void* w_base = want_dx ? W : X_keep;
     const void* x_base = want_dw ? X_keep : W;
@@ -680,16 +790,23 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     prm.dw_split_stride = C_in * C_out;
     prm.dw_splits = pl.splits;
     prm.dw_accumulate = (pl.splits == 1 && accumulate) ? 1 : 0;
+    // TMA stores need a 16-byte aligned base; any other dW pointer takes the plain-store epilogue
+    prm.dw_tma = (want_dw && reinterpret_cast<uintptr_t>(prm.dW_out) % 16 == 0) ? 1 : 0;
+    if (prm.dw_tma) {
+        if (!make_map_dw(&map_dw, prm.dW_out, pl.splits, C_in, C_out)) return SBP_ERR_CUDA;
+    } else {
+        map_dw = map_x;                                              // never used
+    }
     prm.db_partial = (db != nullptr) ? db_workspace : nullptr;
     prm.status_word = status_word;
     int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
     if (ctas < 1) ctas = 1;
     const dim3 grid((unsigned)ctas);
     cudaError_t e;
-    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, prm);
-    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, prm);
-    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, prm);
-    else e = launch_fused<128, 128>(grid, stream, map_w, map_x, prm);
+    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, map_dw, prm);
+    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, map_dw, prm);
+    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, map_dw, prm);
+    else e = launch_fused<128, 128>(grid, stream, map_w, map_x, map_dw, prm);
     if (e != cudaSuccess) return SBP_ERR_CUDA;
     const bool reduce_dw = want_dw && pl.splits > 1, reduce_db = db != nullptr;
     cudaError_t r = cudaSuccess;
