@@ -153,6 +153,53 @@ __device__ __forceinline__ uint32_t swizzled(uint32_t row, uint32_t chunk) {
     return row * kRowBytes + ((chunk ^ (row & 7u)) << 4);
 }
 
+// Zero the dropped rows of dX that belong to quarter `wq` (32 kept rows) of a dX tile, in the tile's
+// column strip: from just after the kept row preceding the quarter's first one up to its last kept
+// row (to the end of dX if it holds the very last kept row).  The rows are walked in windows of 32; a
+// warp-wide OR marks the kept rows of a window, the rest get zeros.  One warp, no other data needed:
+// the side warps run this for every dX tile of the block while the tensor pipe works.
+template <int BNX>
+__device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile& t, int64_t M_keep, int wq, int lane) {
+    const int C_in = p.C_in;
+    const int n0 = (int)(t.col_tile * BNX);
+    const int strip_cols = (C_in - n0 < BNX) ? C_in - n0 : BNX;   // multiple of 8
+    const int strip_vecs = strip_cols >> 3;
+    const int64_t m0 = (int64_t)t.row_tile * kBM;
+    const int64_t m = m0 + wq * 32 + lane;
+    const bool valid = m < M_keep;
+    const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
+    const int64_t prev = (valid && m > 0) ? (int64_t)__ldg(p.keep_rows + m - 1) : -1;
+    const int nvalid = __popc(__ballot_sync(0xffffffffu, valid));
+    if (nvalid == 0) return;
+    const int64_t lo = __shfl_sync(0xffffffffu, prev, 0) + 1;
+    const int64_t last_cur = __shfl_sync(0xffffffffu, cur, nvalid - 1);
+    const int64_t hi = (m0 + wq * 32 + nvalid == M_keep) ? p.M : last_cur;
+    for (int64_t base = lo; base < hi; base += 32) {
+        const int64_t d = cur - base;
+        uint32_t todo = ~__reduce_or_sync(0xffffffffu, (valid && d >= 0 && d < 32) ? (1u << d) : 0u);
+        if (hi - base < 32) todo &= (1u << (hi - base)) - 1u;
+        if (strip_vecs <= 16) {                      // narrow strip: two rows per store instruction
+            while (todo) {
+                const int b0 = __ffs(todo) - 1;
+                todo &= todo - 1u;
+                const int b1 = todo ? __ffs(todo) - 1 : -1;
+                if (todo) todo &= todo - 1u;
+                const int b = (lane < 16) ? b0 : b1;
+                const int v = lane & 15;
+                if (b >= 0 && v < strip_vecs)
+                    ptx::st_global_v4(p.dX + (base + b) * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
+            }
+        } else {
+            while (todo) {
+                const int b = __ffs(todo) - 1;
+                todo &= todo - 1u;
+                if (lane < strip_vecs)
+                    ptx::st_global_v4(p.dX + (base + b) * C_in + n0 + lane * 8, 0u, 0u, 0u, 0u);
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 template <int BNX, int BNW>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -362,7 +409,16 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         }
         ptx::cp_async_wait_all();
     } else if (warp >= kBiasWarp0) {
-        // ---------------- bias warps: db partial of this CTA's share of the kept rows ----------------
+        // ---------------- side warps: zeros for the dropped rows of dX, then the bias sums ----------------
+        if (p.dX != nullptr && M_keep > 0) {
+            for (uint32_t pass = 0;; ++pass) {
+                const uint32_t q = list_position(pass);
+                if (q >= sched.total) break;
+                const Tile t = decode_tile(sched, q);
+                if (!t.is_dw) zero_dropped_rows<BNX>(p, t, M_keep, warp - kBiasWarp0, lane);
+            }
+        }
+        // db partial of this CTA's share of the kept rows
         if (p.db_partial != nullptr) {
             float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256);
             const int t = threadIdx.x - kBiasWarp0 * 32;
@@ -440,75 +496,52 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             const uint32_t acc = used & 1u;
             const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
             if (!t.is_dw) {
-                // ---- dX tile: zero the dropped rows around this warp's kept rows, then scatter ----
+                // ---- dX tile: scatter the kept rows (the dropped rows are zeroed by the side warps) ----
                 const int n0 = (int)(t.col_tile * BNX);
                 const int strip_cols = (C_in - n0 < BNX) ? C_in - n0 : BNX;   // multiple of 8
-                const int strip_vecs = strip_cols >> 3;
                 const int64_t m0 = (int64_t)t.row_tile * kBM;
                 const int64_t m = m0 + warp * 32 + lane;
                 const bool valid = m < M_keep;
                 const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
-                const int64_t prev = (valid && m > 0) ? (int64_t)__ldg(p.keep_rows + m - 1) : -1;
-                // Rows this warp owns: from just after the kept row preceding its first one up to its
-                // last kept row (to the end of dX if it holds the very last kept row).  They are walked
-                // in windows of 32; a warp-wide OR marks the kept rows of a window, the rest get zeros.
-                const int nvalid = __popc(__ballot_sync(0xffffffffu, valid));
-                if (nvalid > 0) {
-                    const int64_t lo = __shfl_sync(0xffffffffu, prev, 0) + 1;
-                    const int64_t last_cur = __shfl_sync(0xffffffffu, cur, nvalid - 1);
-                    const int64_t hi = (m0 + warp * 32 + nvalid == M_keep) ? p.M : last_cur;
-                    for (int64_t base = lo; base < hi; base += 32) {
-                        const int64_t d = cur - base;
-                        uint32_t todo = ~__reduce_or_sync(0xffffffffu, (valid && d >= 0 && d < 32) ? (1u << d) : 0u);
-                        if (hi - base < 32) todo &= (1u << (hi - base)) - 1u;
-                        if (strip_vecs <= 16) {                      // narrow strip: two rows per store instruction
-                            while (todo) {
-                                const int b0 = __ffs(todo) - 1;
-                                todo &= todo - 1u;
-                                const int b1 = todo ? __ffs(todo) - 1 : -1;
-                                if (todo) todo &= todo - 1u;
-                                const int b = (lane < 16) ? b0 : b1;
-                                const int v = lane & 15;
-                                if (b >= 0 && v < strip_vecs)
-                                    ptx::st_global_v4(p.dX + (base + b) * C_in + n0 + v * 8, 0u, 0u, 0u, 0u);
-                            }
-                        } else {
-                            while (todo) {
-                                const int b = __ffs(todo) - 1;
-                                todo &= todo - 1u;
-                                if (lane < strip_vecs)
-                                    ptx::st_global_v4(p.dX + (base + b) * C_in + n0 + lane * 8, 0u, 0u, 0u, 0u);
-                            }
-                        }
-                    }
-                }
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
+                if (threadIdx.x == 0) ptx::bulk_wait_read<0>();       // the staging memory is no longer read by TMA stores of a dW tile
                 ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);            // the four epilogue warps go on, or give up, together
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                __nv_bfloat16* out_row = p.dX + (valid ? cur : 0) * C_in + n0;
-                auto store_chunk = [&](const float (&v)[32], int c0) {   // 32 accumulator columns -> 64 bytes of one row
-                    if (!valid) return;
-#pragma unroll
-                    for (int qd = 0; qd < 4; ++qd) {
-                        if (c0 + qd * 8 < strip_cols)
-                            ptx::st_global_v4(out_row + c0 + qd * 8,
-                                              pack_bf16(v[qd * 8 + 0], v[qd * 8 + 1]), pack_bf16(v[qd * 8 + 2], v[qd * 8 + 3]),
-                                              pack_bf16(v[qd * 8 + 4], v[qd * 8 + 5]), pack_bf16(v[qd * 8 + 6], v[qd * 8 + 7]));
-                    }
-                };
-                // two register buffers: the next TMEM read is in flight while the current chunk is stored
+                // Each lane holds one row of the accumulator, but a store instruction that writes 32
+                // different rows costs 32 memory transactions.  So the warp transposes 64 columns at a
+                // time through its own 4 KB of (swizzled) shared memory and writes four rows x 128
+                // contiguous bytes per instruction.
+                uint8_t* wbuf = smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256 + kBiasSmemBytes + warp * 4096;
+                const int cur32 = valid ? (int)cur : -1;
+                const int sub = lane >> 3, ch = lane & 7;
                 float va[32], vb[32];
                 ptx::tmem_ld_32x32(taddr, va);
-                ptx::tmem_ld_wait();
+                ptx::tmem_ld_32x32(taddr + 32u, vb);
+#pragma unroll 1
+                for (int c0 = 0; c0 < strip_cols; c0 += 64) {
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                for (int c0 = 0; c0 < BNX; c0 += 64) {
-                    ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), vb);
-                    store_chunk(va, c0);
-                    ptx::tmem_ld_wait();
-                    if (c0 + 64 < BNX) ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
-                    store_chunk(vb, c0 + 32);
-                    ptx::tmem_ld_wait();
+                    for (int q = 0; q < 8; ++q) {
+                        const float* f = (q < 4) ? &va[q * 8] : &vb[(q - 4) * 8];
+                        *reinterpret_cast<uint4*>(wbuf + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                            make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                    }
+                    __syncwarp();
+                    if (c0 + 64 < strip_cols) {                      // the next 64 columns are read while these are stored
+                        ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
+                        ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 96), vb);
+                    }
+                    const bool col_ok = c0 + ch * 8 < strip_cols;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = i * 4 + sub;
+                        const int g = __shfl_sync(0xffffffffu, cur32, r);
+                        const uint4 pk = *reinterpret_cast<const uint4*>(wbuf + r * 128 + ((ch ^ (r & 7)) << 4));
+                        if (g >= 0 && col_ok)
+                            ptx::st_global_v4(p.dX + (int64_t)g * C_in + n0 + c0 + ch * 8, pk.x, pk.y, pk.z, pk.w);
+                    }
+                    __syncwarp();
                 }
             } else {
                 // ---- dW tile: accumulator row = output column j, accumulator column = output row i ----
