@@ -112,16 +112,16 @@ struct ReduceJob {
     int64_t n_vec;        // float4 elements per partial
     int splits;
     int accumulate;
-    int deep;             // 0: one thread per float4, partials added in ascending order
-                          // 1: 8 float4 columns x 32 row lanes per block; lane y adds partials y, y+32, ...
-                          //    in ascending order, the 32 lane sums are then added in lane order
+    int lanes;            // 1: one thread per float4, partials added in ascending order
+                          // Y = 4 or 32: 256/Y float4 columns x Y row lanes per block; lane y adds partials
+                          //    y, y+Y, ... in ascending order, the Y lane sums are then added in lane order
     int blocks;
 };
 
 __device__ __forceinline__ void add4(float4& s, const float4& p) { s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w; }
 
-__device__ __forceinline__ void run_reduce_job(const ReduceJob& jb, int block, float4 (*red)[8]) {
-    if (!jb.deep) {
+__device__ __forceinline__ void run_reduce_job(const ReduceJob& jb, int block, float4* red) {
+    if (jb.lanes == 1) {
         const int64_t stride = (int64_t)jb.blocks * blockDim.x;
         for (int64_t i = (int64_t)block * blockDim.x + threadIdx.x; i < jb.n_vec; i += stride) {
             float4 s = jb.accumulate ? jb.out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -139,34 +139,34 @@ __device__ __forceinline__ void run_reduce_job(const ReduceJob& jb, int block, f
         }
         return;
     }
-    const int x = threadIdx.x & 7, y = threadIdx.x >> 3;
-    const int64_t i = (int64_t)block * 8 + x;
+    const int Y = jb.lanes, X = 256 / Y;
+    const int x = threadIdx.x % X, y = threadIdx.x / X;
+    const int64_t i = (int64_t)block * X + x;
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i < jb.n_vec) {
-        for (int k0 = y; k0 < jb.splits; k0 += 32 * 4) {
+        for (int k0 = y; k0 < jb.splits; k0 += Y * 4) {
             float4 p[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                p[u] = (k0 + 32 * u < jb.splits) ? __ldg(jb.partials + (int64_t)(k0 + 32 * u) * jb.n_vec + i)
-                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                p[u] = (k0 + Y * u < jb.splits) ? __ldg(jb.partials + (int64_t)(k0 + Y * u) * jb.n_vec + i)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (k0 + 32 * u < jb.splits) add4(s, p[u]);
+                if (k0 + Y * u < jb.splits) add4(s, p[u]);
         }
     }
-    red[y][x] = s;
+    red[y * X + x] = s;
     __syncthreads();
     if (y == 0 && i < jb.n_vec) {
         float4 t = jb.accumulate ? jb.out[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int w = 0; w < 32; ++w) add4(t, red[w][x]);
+        for (int w = 0; w < Y; ++w) add4(t, red[w * X + x]);
         jb.out[i] = t;
     }
 }
 
 __global__ void __launch_bounds__(256)
 reduce_partials_kernel(const ReduceJob a, const ReduceJob b, const int32_t* __restrict__ status_word) {
-    __shared__ float4 red[32][8];
+    __shared__ float4 red[256];
     pdl_launch_dependents();
     pdl_wait();
     if (status_word != nullptr && *status_word != 0) return;
@@ -181,10 +181,13 @@ ReduceJob make_reduce_job(const float* partials, int splits, int64_t n, float* o
     jb.n_vec = n / 4;             // n is a multiple of 4 for every caller
     jb.splits = splits;
     jb.accumulate = accumulate ? 1 : 0;
-    jb.deep = splits > 8 ? 1 : 0;
+    // few partials: one thread per element; many partials of a short vector (db): 32 lanes per column;
+    // many partials of a long one (dW): 4 lanes per column
+    jb.lanes = splits <= 8 ? 1 : (jb.n_vec <= 8192 ? 32 : 4);
     int64_t blocks;
-    if (jb.deep) {
-        blocks = (jb.n_vec + 7) / 8;
+    if (jb.lanes > 1) {
+        const int64_t cols = 256 / jb.lanes;
+        blocks = (jb.n_vec + cols - 1) / cols;
     } else {
         blocks = (jb.n_vec + 255) / 256;
         if (blocks > kNumSMs * 8) blocks = kNumSMs * 8;
