@@ -235,7 +235,7 @@ def run_cuda(args, w, name):
         s["p"]["cnt"] = s["offs"].data_ptr() + 4 * B
     cap_full = B * sbp.sbp_keep_count(mode, H, W_, 1.0)
 
-    def step(i, keep_ratio=r, events=None, all_events=False):
+    def step(i, keep_ratio=r, events=None, all_events=False, sid=sid):
         """One pass of the whole path: draw the keep set, cache the kept rows, run the backward.
 
         `events` = (before, after) the backward call on the launch stream (the call whose first kernel is the
@@ -293,6 +293,37 @@ def run_cuda(args, w, name):
         step(i)
     barrier()
     assert int(status.item()) == 0, "device status word set during warm-up"
+
+    # One captured step per buffer set (sampler, cache, backward through the same C-ABI calls): replaying them
+    # keeps the host out of the timed region.  The step counter of a captured step is fixed, so the masks repeat
+    # every n_sets steps; every replay still draws, gathers and multiplies from scratch.
+    graphs = []
+    if args.launch == "graph":
+        cap_stream = torch.cuda.Stream()
+        cap_stream.wait_stream(stream)
+        for k in range(n_sets):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap_stream):
+                step(k, sid=cap_stream.cuda_stream)
+            graphs.append(g)
+        for g in graphs:
+            g.replay()
+        barrier()
+
+    def timed_graphs(k_steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(k_steps):
+            graphs[i % n_sets].replay()
+        e1.record(stream)
+        barrier()
+        total_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        return total_ms
     M_keep = int(sets[0]["offs"][B].item())
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -302,7 +333,10 @@ def run_cuda(args, w, name):
     # The headline region carries no events between its calls (an event record between two kernels
     # keeps the second from starting its launch early); the same K steps are then repeated with the
     # backward call bracketed, which gives the launch duration the roofline figure uses.
-    total_ms, _, _ = timed(args.steps, inner_events=False)
+    if args.launch == "graph":
+        total_ms = timed_graphs(args.steps)
+    else:
+        total_ms, _, _ = timed(args.steps, inner_events=False)
     _, gemm_ms, _ = timed(args.steps)
     if sampler:
         clocks = sampler.stop()
@@ -388,7 +422,9 @@ def run_cuda(args, w, name):
             "config": {"workload": name, "B_per_gpu": B, "H": H, "W": W_, "C_in": C_in, "C_out": C_out, "keep_ratio": r,
                        "mask": "grid" if mode else "random", "M": M, "M_keep": M_keep,
                        "l2": f"inputs larger than L2: {n_sets} rotating buffer sets of {set_bytes / 1e6:.0f} MB",
-                       "parallelism": f"dp{world} (batch sharded by sample id, no collective)"},
+                       "parallelism": f"dp{world} (batch sharded by sample id, no collective)",
+                       "launch": ("CUDA graph replay, one captured step (3 C-ABI calls) per buffer set" if args.launch == "graph"
+                                  else "direct C-ABI calls")},
             "roofline": roofline,
             "cpu_baseline": {"value": cpu_flops / cpu_s / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
                              "kind": "oracle", "seconds": cpu_s,
@@ -415,6 +451,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="vit_b16_fc1", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--launch", default="graph", choices=["graph", "calls"],
+                    help="timed steps: replay of captured steps (default) or direct C-ABI calls from Python")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     if args.impl == "reference":
