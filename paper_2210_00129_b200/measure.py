@@ -174,6 +174,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--group", default="all", choices=["vit", "convnext", "detection", "sampler", "all"])
     ap.add_argument("--iters", type=int, default=24)
+    ap.add_argument("--compact", action="store_true", help="one table row per layer: us (t_min / t) per call")
     args = ap.parse_args()
     sbp.load_library()
     pk, kind = peaks()
@@ -181,14 +182,23 @@ def main():
     print(f"peaks ({kind}): bf16 {pk['bf16_tflops_sustained']:.0f} TFLOP/s sustained, HBM {pk['hbm_gbs']:.0f} GB/s; "
           f"{args.iters} graph-replayed launches per figure, rotating buffer sets larger than L2\n")
     if args.group != "sampler":
-        print("| layer | M_keep | call | us | t_min us | t_min/t | bound | achieved |")
-        print("|---|---|---|---|---|---|---|---|")
+        if args.compact:
+            print("us (t_min / t) per call; bound of the whole backward in the last column\n")
+            print("| layer | M_keep | sample | cache | db | dW | dX | backward (dW+db+dX) | TFLOP/s | bound |")
+            print("|---|---|---|---|---|---|---|---|---|---|")
+        else:
+            print("| layer | M_keep | call | us | t_min us | t_min/t | bound | achieved |")
+            print("|---|---|---|---|---|---|---|---|")
         full = {}
         res = []
         for spec in layers(args.group):
             m = measure_layer(bench, spec, pk)
             res.append((spec, m))
-            for k in ("sample", "cache", "db", "dW", "dX", "bwd"):
+            if args.compact:
+                cells = " | ".join(f"{m['t'][k]:.1f} ({m['tmin'][k] / m['t'][k]:.2f})" for k in ("cache", "db", "dW", "dX", "bwd"))
+                print(f"| {m['name']} | {m['M_keep']} | {m['t']['sample']:.1f} | {cells} | "
+                      f"{2 * m['flop'] / m['t']['bwd'] / 1e6:.0f} | {m['bound']['bwd']} |")
+            for k in (() if args.compact else ("sample", "cache", "db", "dW", "dX", "bwd")):
                 us = m["t"][k]
                 if k in ("dW", "dX", "bwd"):
                     ach = f"{(2 if k == 'bwd' else 1) * m['flop'] / us / 1e6:.0f} TFLOP/s"
