@@ -47,7 +47,9 @@ constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
 constexpr uint32_t kAccCols = 256;       // TMEM columns per accumulator buffer (two buffers = all 512)
 constexpr int kBiasChunk = 64;           // kept rows whose ids the bias warps stage at a time
-constexpr int kBiasDepth = 16;           // 16-byte loads each bias thread keeps in flight
+// 16-byte loads each side-warp thread keeps in flight for the bias sums: a template parameter of the kernel,
+// 8 or 16.  The deep queue finishes long row lists in time; with short lists it only takes memory
+// bandwidth from the operand copies (ViT-B fc1: 5 us per call), so the host picks per shape.
 constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float) + kBiasChunk * sizeof(int);   // cross-row-group sums + staged row ids
 constexpr int kEpiChunk = 16;            // accumulator columns (= rows of dW) per TMA store of the dW epilogue
 constexpr int kEpiBufs = 3;              // staging buffers the dW epilogue rotates through
@@ -201,7 +203,7 @@ __device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile&
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int BNX, int BNW>
+template <int BNX, int BNW, int kBiasDepth>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                    const __grid_constant__ CUtensorMap map_dw, const TcParams p) {
@@ -765,13 +767,21 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     return pl;
 }
 
-template <int BNX, int BNW>
-cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
-                         const CUtensorMap& map_dw, const TcParams& prm) {
-    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW>,
+template <int BNX, int BNW, int DEPTH>
+cudaError_t launch_fused_depth(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
+                               const CUtensorMap& map_dw, const TcParams& prm) {
+    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW, DEPTH>,
                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (once != cudaSuccess) return once;
-    return launch_pdl(tc_backward_kernel<BNX, BNW>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x, map_dw, prm);
+    return launch_pdl(tc_backward_kernel<BNX, BNW, DEPTH>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x,
+                      map_dw, prm);
+}
+
+template <int BNX, int BNW>
+cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
+                         const CUtensorMap& map_dw, const TcParams& prm, bool deep_side_queue) {
+    return deep_side_queue ? launch_fused_depth<BNX, BNW, 16>(grid, stream, map_w, map_x, map_dw, prm)
+                           : launch_fused_depth<BNX, BNW, 8>(grid, stream, map_w, map_x, map_dw, prm);
 }
 
 }  // namespace
@@ -835,11 +845,24 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
     if (ctas < 1) ctas = 1;
     const dim3 grid((unsigned)ctas);
+    // Bias sums on the side: 16-byte loads per side-warp thread against the time the main loop leaves them
+    // (about 1.3 us per batch of loads in flight, 0.45 us per k-block).  The shallow queue is enough when it
+    // ends well within the main loop.
+    bool deep_side = true;
+    if (db != nullptr) {
+        const int64_t x_tiles = want_dx ? ((M_keep_cap + kBM - 1) / kBM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
+        const int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
+        const double kb_total = (double)x_tiles * (double)((C_out + kBK - 1) / kBK) +
+                                (double)w_tiles * (double)((M_keep_cap + kBK - 1) / kBK);
+        const double loop_us = kb_total / (double)ctas * 0.45;
+        const double loads = (double)((M_keep_cap + ctas - 1) / ctas) * (double)(C_out / 8) / (double)kBiasThreads;
+        deep_side = loads / 8.0 * 1.3 > 0.6 * loop_us;
+    }
     cudaError_t e;
-    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, map_dw, prm);
-    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, map_dw, prm);
-    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, map_dw, prm);
-    else e = launch_fused<128, 128>(grid, stream, map_w, map_x, map_dw, prm);
+    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
+    else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
+    else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
+    else e = launch_fused<128, 128>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
     if (e != cudaSuccess) return SBP_ERR_CUDA;
     const bool reduce_dw = want_dw && pl.splits > 1, reduce_db = db != nullptr;
     cudaError_t r = cudaSuccess;
