@@ -21,7 +21,6 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 __global__ void __launch_bounds__(kGatherThreads)
 gather_rows_kernel(const uint4* __restrict__ X, uint32_t vec_per_row, const int32_t* __restrict__ keep_rows,
                    const int32_t* __restrict__ M_keep_dev, int64_t M_keep_cap, uint4* __restrict__ X_keep) {
-    pdl_launch_dependents();
     pdl_wait();
     const int64_t M_keep = load_m_keep(M_keep_dev, M_keep_cap);
     const int64_t total = M_keep_cap * (int64_t)vec_per_row;
@@ -50,6 +49,9 @@ gather_rows_kernel(const uint4* __restrict__ X, uint32_t vec_per_row, const int3
             if (i < total) X_keep[i] = v[u];
         }
     }
+    // Only now may the next kernel's blocks take their places: the usual successor (the backward kernel) needs
+    // a whole SM per block, and resident early it would push this kernel's remaining blocks off the SMs.
+    pdl_launch_dependents();
 }
 
 __global__ void validate_keep_rows_kernel(const int32_t* __restrict__ keep_rows,
