@@ -58,7 +58,9 @@ enum {
     SBP_FLAG_SHARE_MASK = 1,  /* every sample of the call uses sample 0's mask (one mask per iteration, Supp. A.4) */
     SBP_FLAG_ACCUMULATE = 2,  /* dW += and db += instead of overwrite (gradient accumulation) */
     SBP_FLAG_VALIDATE = 4,    /* check keep_rows on the device before use; result in the status word */
-    SBP_FLAG_PLAIN_FMA = 8    /* bf16 only: use the CUDA-core FMA kernels instead of the tensor-core ones */
+    SBP_FLAG_PLAIN_FMA = 8,   /* bf16 only: use the CUDA-core FMA kernels instead of the tensor-core ones */
+    SBP_FLAG_DY_COMPACT = 16, /* dY holds only the kept rows, packed: [M_keep_cap, C_out] (chained layers, Sec. 3.3.1) */
+    SBP_FLAG_DX_COMPACT = 32  /* dX receives only the kept rows, packed: [M_keep_cap, C_in]; no zero rows are written */
 };
 
 const char* sbp_status_string(sbp_status s);
@@ -137,6 +139,16 @@ size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_ke
  * W [C_in, C_out], keep_rows strictly ascending ids in [0, M).  M_keep is
  * *M_keep_dev if non-NULL, else M_keep_cap.  Any of dW, db, dX may be NULL to skip
  * that product.
+ *
+ * Chained layers (Sec. 3.3.1, Eq. 9: with the same keep set on consecutive point-wise
+ * layers the kept and dropped sets pass through unchanged, so the gradient between
+ * them is non-zero only in the kept rows).  Such a block can keep that gradient
+ * packed: SBP_FLAG_DX_COMPACT makes this call write dX[m, :] = dY_row(m) * W^T into a
+ * [M_keep_cap, C_in] tensor (rows in [M_keep, M_keep_cap) are zeroed, no other zeros
+ * are written), and SBP_FLAG_DY_COMPACT makes it read row m of a [M_keep_cap, C_out]
+ * dY instead of row keep_rows[m] of the full one.  The layer at the block's boundary
+ * uses neither flag on its side facing the rest of the network.  With both flags
+ * keep_rows is not used and may be NULL.
  *
  * SBP_BF16: inputs bf16, products accumulated in fp32 on the tensor cores, dX
  * rounded to bf16 (nearest even).  SBP_F32: plain fp32 FMA arithmetic.

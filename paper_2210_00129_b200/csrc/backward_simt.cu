@@ -73,7 +73,7 @@ simt_dw_kernel(const T* __restrict__ X_keep, const T* __restrict__ dY, const int
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
         if (m < m_end) {
             if (i0 + lc < C_in) a = load4<T>(X_keep + m * C_in + i0 + lc);
-            if (j0 + lc < C_out) b = load4<T>(dY + (int64_t)__ldg(keep_rows + m) * C_out + j0 + lc);
+            if (j0 + lc < C_out) b = load4<T>(dY + (int64_t)mapped_row(keep_rows, m) * C_out + j0 + lc);
         }
         *reinterpret_cast<float4*>(&As[lk][lc]) = a;
         *reinterpret_cast<float4*>(&Bs[lk][lc]) = b;
@@ -105,13 +105,15 @@ simt_dw_kernel(const T* __restrict__ X_keep, const T* __restrict__ dY, const int
 
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads)
-simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t* __restrict__ keep_rows,
-               const int32_t* __restrict__ M_keep_dev, int64_t M, int64_t M_keep_cap, int C_in, int C_out,
+simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t* __restrict__ dy_rows,
+               const int32_t* __restrict__ dx_rows, const int32_t* __restrict__ M_keep_dev, int64_t M, int64_t M_keep_cap, int C_in, int C_out,
                T* __restrict__ dX, const int32_t* __restrict__ status_word) {
     __shared__ __align__(16) float As[kTileK][kTile + 4];
     __shared__ __align__(16) float Bs[kTileK][kTile + 4];
-    // rows[0] = kept row before the tile (or -1), rows[1 + t] = rows of the tile, M past the last kept row
+    // rows[0] = output row before the tile (or -1), rows[1 + t] = output rows of the tile, M past the last kept
+    // row; src[t] = rows of dY the tile reads
     __shared__ int64_t rows[kTile + 2];
+    __shared__ int64_t src[kTile];
     pdl_launch_dependents();
     pdl_wait();
     if (status_word != nullptr && *status_word != 0) return;
@@ -133,7 +135,8 @@ simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t*
     const int tile_rows = (int)((M_keep - m0 < kTile) ? M_keep - m0 : kTile);
     for (int t = threadIdx.x; t <= kTile + 1; t += kSimtThreads) {
         const int64_t m = m0 + t - 1;
-        rows[t] = (m < 0) ? -1 : (m < M_keep ? (int64_t)__ldg(keep_rows + m) : M);
+        rows[t] = (m < 0) ? -1 : (m < M_keep ? (int64_t)mapped_row(dx_rows, m) : M);
+        if (t >= 1 && t <= kTile) src[t - 1] = (m < M_keep) ? (int64_t)mapped_row(dy_rows, m) : -1;
     }
     __syncthreads();
 
@@ -150,7 +153,7 @@ simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t*
 
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int lr = threadIdx.x >> 2, lc = (threadIdx.x & 3) * 4;    // loader: tile row, 4 of the 16 k columns
-    const int64_t a_row = (lr < tile_rows) ? rows[1 + lr] : -1;
+    const int64_t a_row = (lr < tile_rows) ? src[lr] : -1;
     float acc[4][4] = {};
     for (int j0 = 0; j0 < C_out; j0 += kTileK) {
         float4 a = zero4, b = zero4;
@@ -214,7 +217,7 @@ cudaError_t launch_simt_dw(sbp_dtype dt, const void* X_keep, const void* dY, con
     return launch_reduce_partials(workspace, splits, C_in * C_out, dW, accumulate, status_word, stream);
 }
 
-cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const int32_t* keep_rows,
+cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const int32_t* dy_rows, const int32_t* dx_rows,
                            const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
                            int64_t C_out, void* dX, const int32_t* status_word, cudaStream_t stream) {
     int64_t row_tiles = (M_keep_cap + kTile - 1) / kTile;
@@ -222,10 +225,10 @@ cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const in
     const dim3 grid((unsigned)row_tiles, (unsigned)((C_in + kTile - 1) / kTile));
     if (dt == SBP_BF16)
         return launch_pdl(simt_dx_kernel<__nv_bfloat16>, grid, dim3(kSimtThreads), 0, stream,
-                          (const __nv_bfloat16*)dY, (const __nv_bfloat16*)W, keep_rows, M_keep_dev, M, M_keep_cap,
+                          (const __nv_bfloat16*)dY, (const __nv_bfloat16*)W, dy_rows, dx_rows, M_keep_dev, M, M_keep_cap,
                           (int)C_in, (int)C_out, (__nv_bfloat16*)dX, status_word);
     return launch_pdl(simt_dx_kernel<float>, grid, dim3(kSimtThreads), 0, stream,
-                      (const float*)dY, (const float*)W, keep_rows, M_keep_dev, M, M_keep_cap,
+                      (const float*)dY, (const float*)W, dy_rows, dx_rows, M_keep_dev, M, M_keep_cap,
                       (int)C_in, (int)C_out, (float*)dX, status_word);
 }
 

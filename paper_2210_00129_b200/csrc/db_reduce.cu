@@ -81,7 +81,7 @@ db_partial_kernel(const uint4* __restrict__ dY, uint32_t col_vecs, const int32_t
 #pragma unroll
             for (int u = 0; u < kDbUnroll; ++u) {
                 const int64_t mm = m + u * kDbWarps;
-                row[u] = (mm < m_end) ? (int64_t)__ldg(keep_rows + mm) : -1;
+                row[u] = (mm < m_end) ? (int64_t)mapped_row(keep_rows, mm) : -1;
             }
 #pragma unroll
             for (int u = 0; u < kDbUnroll; ++u)

@@ -127,7 +127,10 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
                                void* stream_v) {
     cudaStream_t stream = (cudaStream_t)stream_v;
     if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
-    if (dY == nullptr || keep_rows == nullptr) return SBP_ERR_INVALID_ARG;
+    const bool dy_compact = (flags & SBP_FLAG_DY_COMPACT) != 0, dx_compact = (flags & SBP_FLAG_DX_COMPACT) != 0;
+    // the packed forms address rows by their position m; keep_rows is needed for whichever side is not packed
+    const bool need_rows = !dy_compact || (dX != nullptr && !dx_compact) || (flags & SBP_FLAG_VALIDATE);
+    if (dY == nullptr || (need_rows && keep_rows == nullptr)) return SBP_ERR_INVALID_ARG;
     if (M <= 0 || M >= (1ll << 31) || M_keep_cap < 0 || M_keep_cap > M || C_in <= 0 || C_out <= 0 ||
         C_in >= (1ll << 24) || C_out >= (1ll << 24))
         return SBP_ERR_INVALID_ARG;
@@ -151,6 +154,9 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
                                                       db_scratch_bytes(dt, M_keep_cap, C_out))
                            : nullptr;
 
+    const int32_t* dy_rows = dy_compact ? nullptr : keep_rows;
+    const int32_t* dx_rows = dx_compact ? nullptr : keep_rows;
+    const int64_t M_dx = dx_compact ? M_keep_cap : M;            // rows of the dX tensor
     if (flags & SBP_FLAG_VALIDATE) {
         if (launch_validate_keep_rows(keep_rows, M_keep_dev, M_keep_cap, M, status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
@@ -159,21 +165,21 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     // with the tensor-core kernel running, the bias sums ride along in it; otherwise they get their own kernel
     const bool db_rides = tc && db != nullptr && (dW != nullptr || dX != nullptr);
     if (db != nullptr && !db_rides) {
-        if (launch_db(dt, dY, keep_rows, M_keep_dev, M_keep_cap, C_out, db, accumulate, ws_db, kDbMaxSplits,
+        if (launch_db(dt, dY, dy_rows, M_keep_dev, M_keep_cap, C_out, db, accumulate, ws_db, kDbMaxSplits,
                       status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
     }
     if (tc) {
         // both products (and the bias sums) in one persistent tensor-core kernel
-        const sbp_status s = launch_tc_backward(X_keep, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW,
+        const sbp_status s = launch_tc_backward(X_keep, dY, W, dy_rows, dx_rows, M_keep_dev, M_dx, M_keep_cap, C_in, C_out, dW,
                                                 accumulate, dX, db_rides ? db : nullptr, ws_dw, ws_db, status_word,
                                                 stream);
         if (s != SBP_OK) return s;
     } else {
-        if (dW != nullptr && launch_simt_dw(dt, X_keep, dY, keep_rows, M_keep_dev, M_keep_cap, C_in, C_out, dW,
+        if (dW != nullptr && launch_simt_dw(dt, X_keep, dY, dy_rows, M_keep_dev, M_keep_cap, C_in, C_out, dW,
                                             accumulate, ws_dw, status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
-        if (dX != nullptr && launch_simt_dx(dt, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dX,
+        if (dX != nullptr && launch_simt_dx(dt, dY, W, dy_rows, dx_rows, M_keep_dev, M_dx, M_keep_cap, C_in, C_out, dX,
                                             status_word, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
     }

@@ -64,6 +64,12 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
 }
 #endif
 
+// Row map of the backward kernels: keep_rows[m], or m itself when the tensor is already compact (Sec. 3.3.1:
+// with the same keep set on consecutive layers the kept rows can stay packed between them).
+__device__ __forceinline__ int32_t mapped_row(const int32_t* rows, int64_t m) {
+    return rows != nullptr ? __ldg(rows + m) : (int32_t)m;
+}
+
 // Number of valid kept rows: the device-side count when given, else the host capacity.
 __device__ __forceinline__ int64_t load_m_keep(const int32_t* M_keep_dev, int64_t M_keep_cap) {
     if (M_keep_dev == nullptr) return M_keep_cap;
@@ -137,9 +143,11 @@ cudaError_t launch_simt_dw(sbp_dtype dt, const void* X_keep, const void* dY, con
                            const int32_t* M_keep_dev, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
                            float* dW, bool accumulate, float* workspace, const int32_t* status_word,
                            cudaStream_t stream);
-cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const int32_t* keep_rows,
-                           const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
-                           int64_t C_out, void* dX, const int32_t* status_word, cudaStream_t stream);
+// dy_rows / dx_rows: row m of the product reads row dy_rows[m] of dY and writes row dx_rows[m] of dX
+// (nullptr = m itself); M = rows of dX
+cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const int32_t* dy_rows,
+                           const int32_t* dx_rows, const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap,
+                           int64_t C_in, int64_t C_out, void* dX, const int32_t* status_word, cudaStream_t stream);
 
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
@@ -148,8 +156,9 @@ int    tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out,
                                 bool want_db);
 // dW (nullable) and dX (nullable) of one layer in a single persistent kernel (+ the split reduce); when db is
 // given its column sums ride along in the same kernel (db_workspace: kNumSMs * C_out floats) + one reduce
-sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
-                              const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
+// (dy_rows / dx_rows as for launch_simt_dx)
+sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* dy_rows,
+                              const int32_t* dx_rows, const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in,
                               int64_t C_out, float* dW, bool accumulate, void* dX, float* db, float* workspace,
                               float* db_workspace, int32_t* status_word, cudaStream_t stream);
 

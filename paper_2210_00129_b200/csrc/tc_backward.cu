@@ -71,7 +71,8 @@ static_assert(sizeof(TcControl) <= 256, "control block");
 
 struct TcParams {
     const __nv_bfloat16* dY;
-    const int32_t* keep_rows;
+    const int32_t* dy_rows;        // row m of the products reads row dy_rows[m] of dY (nullptr: row m)
+    const int32_t* dx_rows;        // ... and writes row dx_rows[m] of dX (nullptr: row m); M = rows of dX
     const int32_t* M_keep_dev;
     int64_t M, M_keep_cap;
     int C_in, C_out;
@@ -169,8 +170,8 @@ __device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile&
     const int64_t m0 = (int64_t)t.row_tile * kBM;
     const int64_t m = m0 + wq * 32 + lane;
     const bool valid = m < M_keep;
-    const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
-    const int64_t prev = (valid && m > 0) ? (int64_t)__ldg(p.keep_rows + m - 1) : -1;
+    const int64_t cur = valid ? (int64_t)mapped_row(p.dx_rows, m) : -1;
+    const int64_t prev = (valid && m > 0) ? (int64_t)mapped_row(p.dx_rows, m - 1) : -1;
     const int nvalid = __popc(__ballot_sync(0xffffffffu, valid));
     if (nvalid == 0) return;
     const int64_t lo = __shfl_sync(0xffffffffu, prev, 0) + 1;
@@ -341,7 +342,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 for (int i = 0; i < kInstr; ++i) {
                     int64_t m = m0 + (gw * kInstr + i) * 4 + sub;
                     if (m >= M_keep) m = M_keep - 1;                  // padding rows of the last tile: never stored
-                    src[i] = p.dY + (int64_t)__ldg(p.keep_rows + m) * C_out + chunk * 8;
+                    src[i] = p.dY + (int64_t)mapped_row(p.dy_rows, m) * C_out + chunk * 8;
                 }
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
                     const int s = it % kStages;
@@ -376,7 +377,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                         for (int h = 0; h < kIdxPerLane; ++h) {
                             const int64_t mrow = (int64_t)(t.kb_begin + k_first + u) * kBK + gw * kRows + h * 32 + (lane % kRows);
-                            nxt[u][h] = (k_first + u < t.num_kb && mrow < M_keep) ? __ldg(p.keep_rows + mrow) : -1;
+                            nxt[u][h] = (k_first + u < t.num_kb && mrow < M_keep) ? mapped_row(p.dy_rows, mrow) : -1;
                         }
                 };
                 fetch_ids(0);
@@ -440,7 +441,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                 for (int64_t mc = m_begin; mc < m_end; mc += kBiasChunk) {
                     // stage the chunk's row ids once, so that the dY loads below depend on no other load
-                    if (t < kBiasChunk) ids[t] = (mc + t < m_end) ? __ldg(p.keep_rows + mc + t) : -1;
+                    if (t < kBiasChunk) ids[t] = (mc + t < m_end) ? mapped_row(p.dy_rows, mc + t) : -1;
                     asm volatile("bar.sync 1, %0;" ::"n"(kBiasThreads) : "memory");
                     if (cv < V) {
                         for (int r0 = rg; r0 < kBiasChunk; r0 += RG * kBiasDepth) {
@@ -504,7 +505,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const int64_t m0 = (int64_t)t.row_tile * kBM;
                 const int64_t m = m0 + warp * 32 + lane;
                 const bool valid = m < M_keep;
-                const int64_t cur = valid ? (int64_t)__ldg(p.keep_rows + m) : -1;
+                const int64_t cur = valid ? (int64_t)mapped_row(p.dx_rows, m) : -1;
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
                 if (threadIdx.x == 0) ptx::bulk_wait_read<0>();       // the staging memory is no longer read by TMA stores of a dW tile
                 ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);            // the four epilogue warps go on, or give up, together
@@ -806,8 +807,8 @@ int tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bo
     return 1 + ((reduce_dw || want_db) ? 1 : 0);       // the two reductions share one launch
 }
 
-sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* keep_rows,
-                              const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
+sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W, const int32_t* dy_rows,
+                              const int32_t* dx_rows, const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
                               float* dW, bool accumulate, void* dX, float* db, float* workspace, float* db_workspace,
                               int32_t* status_word, cudaStream_t stream) {
     const bool want_dw = dW != nullptr, want_dx = dX != nullptr;
@@ -822,7 +823,8 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
         return SBP_ERR_CUDA;
     TcParams prm;
     prm.dY = static_cast<const __nv_bfloat16*>(dY);
-    prm.keep_rows = keep_rows;
+    prm.dy_rows = dy_rows;
+    prm.dx_rows = dx_rows;
     prm.M_keep_dev = M_keep_dev;
     prm.M = M;
     prm.M_keep_cap = M_keep_cap;

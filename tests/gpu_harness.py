@@ -44,8 +44,10 @@ def run_forward_cache(dtype, X_dev, keep_rows_dev, M_keep_cap, M_keep_dev=None):
 
 
 def run_backward(dtype, X_keep_dev, dY_dev, W_dev, keep_rows_dev, M_keep_cap, M_keep_dev=None, flags=0,
-                 want=("dW", "db", "dX"), init=None, with_status=True):
-    M, C_out = dY_dev.shape
+                 want=("dW", "db", "dX"), init=None, with_status=True, M=None, dX_rows=None):
+    """M: rows of the layer (default: rows of dY, which a packed dY does not have); dX_rows: rows of the dX buffer."""
+    C_out = dY_dev.shape[1]
+    M = dY_dev.shape[0] if M is None else M
     C_in = W_dev.shape[0] if W_dev is not None else X_keep_dev.shape[1]
     code = dt_code(dtype)
     nbytes = sbp.sbp_linear_backward_workspace_bytes(code, M, M_keep_cap, C_in, C_out)
@@ -54,7 +56,8 @@ def run_backward(dtype, X_keep_dev, dY_dev, W_dev, keep_rows_dev, M_keep_cap, M_
     fill = float("nan")
     dW = torch.full((C_in, C_out), fill, dtype=torch.float32, device="cuda") if "dW" in want else None
     db = torch.full((C_out,), fill, dtype=torch.float32, device="cuda") if "db" in want else None
-    dX = torch.full((M, C_in), fill, dtype=dY_dev.dtype, device="cuda") if "dX" in want else None
+    dX = torch.full((M if dX_rows is None else max(dX_rows, 1), C_in), fill, dtype=dY_dev.dtype,
+                    device="cuda") if "dX" in want else None
     if init is not None:
         if dW is not None: dW.copy_(init["dW"])
         if db is not None: db.copy_(init["db"])
