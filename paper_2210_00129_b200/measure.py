@@ -1,6 +1,6 @@
 """Per-call timing sweep over the paper's layer shapes, against the roofline of each call.
 
-    python -m paper_2210_00129_b200.measure [--group vit|convnext|detection|sampler|all] [--iters 24]
+    python -m paper_2210_00129_b200.measure [--group vit|convnext|detection|blocks|sampler|all] [--iters 24]
 
 For every layer of the chosen groups (ViT-B/16 MLP and attention projections at four keep ratios,
 ConvNeXt-B point-wise layers of the four stages with random and grid masks, the detection-resolution
@@ -156,6 +156,50 @@ def measure_layer(bench, spec, pk):
     return dict(name=name, M=M, M_keep=M_keep, t=t, tmin=tmin, bound=bound, flop=flop, bytes=by)
 
 
+def mlp_block(bench, B, H, W_, d, h, r):
+    """Backward of a two-layer block d -> h -> d (a ViT MLP, a ConvNeXt block's point-wise pair; upper layer first)
+    with the same keep set on both layers: the gradient between the layers scattered to all rows and gathered
+    again, against kept packed (Eq. 9)."""
+    M = B * H * W_
+    cap = B * sbp.sbp_keep_count(0, H, W_, r)
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    rn = lambda *sh: torch.randn(*sh, device="cuda", generator=gen)
+    n_sets = 3
+    sets = []
+    for _ in range(n_sets):
+        sets.append(dict(X0k=rn(cap, d).bfloat16(), X1k=rn(cap, h).bfloat16(), dY=(rn(M, d) * 0.01).bfloat16(),
+                         W1=(rn(d, h) * 0.02).bfloat16(), W2=(rn(h, d) * 0.02).bfloat16(),
+                         dW1=torch.zeros(d, h, device="cuda"), db1=torch.zeros(h, device="cuda"),
+                         dW2=torch.zeros(h, d, device="cuda"), db2=torch.zeros(d, device="cuda"),
+                         dX1=torch.zeros(M, h, device="cuda", dtype=torch.bfloat16),
+                         dX0=torch.zeros(M, d, device="cuda", dtype=torch.bfloat16),
+                         rows=torch.zeros(cap, dtype=torch.int32, device="cuda"),
+                         offs=torch.zeros(B + 1, dtype=torch.int32, device="cuda")))
+    nb = max(sbp.sbp_linear_backward_workspace_bytes(sbp.SBP_BF16, M, cap, d, h),
+             sbp.sbp_linear_backward_workspace_bytes(sbp.SBP_BF16, M, cap, h, d))
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.stream(bench.stream):
+        for s in sets:
+            sbp.sbp_sample_keep(0, B, H, W_, r, 0, 0, 0, 0, s["rows"], s["offs"], stream=bench.sid)
+    bench.stream.synchronize()
+
+    def block(k, packed):
+        s = sets[k]
+        up, low = (sbp.SBP_FLAG_DX_COMPACT, sbp.SBP_FLAG_DY_COMPACT) if packed else (0, 0)
+        sbp.sbp_linear_backward(sbp.SBP_BF16, s["X1k"], s["dY"], s["W2"], s["rows"], None, M, cap, h, d, s["dW2"], s["db2"],
+                                s["dX1"], up, ws, nb, st, stream=bench.sid)
+        sbp.sbp_linear_backward(sbp.SBP_BF16, s["X0k"], s["dX1"], s["W1"], s["rows"], None, M, cap, d, h, s["dW1"], s["db1"],
+                                s["dX0"], low, ws, nb, st, stream=bench.sid)
+
+    t_scatter = bench.time_us(lambda k, i: block(k, False), n_sets)
+    t_packed = bench.time_us(lambda k, i: block(k, True), n_sets)
+    assert int(st.item()) == 0
+    flop = 8.0 * cap * d * h
+    return cap, t_scatter, t_packed, flop
+
+
 def sampler_stress(bench, pk):
     """Sampler alone on a shape whose index stream is large enough to read as bandwidth."""
     rows = []
@@ -172,7 +216,7 @@ def sampler_stress(bench, pk):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--group", default="all", choices=["vit", "convnext", "detection", "sampler", "all"])
+    ap.add_argument("--group", default="all", choices=["vit", "convnext", "detection", "blocks", "sampler", "all"])
     ap.add_argument("--iters", type=int, default=24)
     ap.add_argument("--compact", action="store_true", help="one table row per layer: us (t_min / t) per call")
     args = ap.parse_args()
@@ -181,7 +225,7 @@ def main():
     bench = Bench(args.iters)
     print(f"peaks ({kind}): bf16 {pk['bf16_tflops_sustained']:.0f} TFLOP/s sustained, HBM {pk['hbm_gbs']:.0f} GB/s; "
           f"{args.iters} graph-replayed launches per figure, rotating buffer sets larger than L2\n")
-    if args.group != "sampler":
+    if args.group not in ("sampler", "blocks"):
         if args.compact:
             print("us (t_min / t) per call; bound of the whole backward in the last column\n")
             print("| layer | M_keep | sample | cache | db | dW | dX | backward (dW+db+dX) | TFLOP/s | bound |")
@@ -218,6 +262,17 @@ def main():
             print("\n| layer | keep ratio | backward us | at keep 1.0 us | speed-up | 1/r |")
             print("|---|---|---|---|---|---|")
             print("\n".join(lines))
+    if args.group in ("blocks", "all"):
+        print("\n| two-layer block backward, d -> 4d -> d (both layers, dW + db + dX each) | M_keep | gradient between "
+              "the layers scattered, us | packed, us | gain | packed TFLOP/s |")
+        print("|---|---|---|---|---|---|")
+        blocks = [("vit_b16 MLP B=64 r=0.5", 64, 14, 14, 768, 0.5), ("vit_b16 MLP B=128 r=0.25", 128, 14, 14, 768, 0.25),
+                  ("vit_b16 MLP B=128 r=0.5", 128, 14, 14, 768, 0.5), ("vit_b16 MLP B=128 r=0.75", 128, 14, 14, 768, 0.75),
+                  ("convnext_b s1 block", 64, 56, 56, 128, 0.5), ("convnext_b s2 block", 64, 28, 28, 256, 0.5),
+                  ("convnext_b s3 block", 64, 14, 14, 512, 0.5), ("detection 200x334 block", 2, 200, 334, 128, 0.5)]
+        for nm, B, H, W_, d, r in blocks:
+            cap, ts, tp, flop = mlp_block(bench, B, H, W_, d, 4 * d, r)
+            print(f"| {nm} | {cap} | {ts:.1f} | {tp:.1f} | {ts / tp:.2f} | {flop / tp / 1e6:.0f} |")
     if args.group in ("sampler", "all"):
         print("\n| sampler shape | kept ids | us | index stream GB/s | positions per ns |")
         print("|---|---|---|---|---|")
