@@ -21,6 +21,7 @@ _LIB_PATH = os.path.join(_HERE, "libsbp_oracle.so")
 
 MASK_RANDOM = 0
 MASK_GRID = 1
+MASK_TEMPORAL = 2
 FLAG_SHARE_MASK = 1
 
 _lib = None

@@ -34,6 +34,7 @@
 
 #define ORACLE_MASK_RANDOM 0
 #define ORACLE_MASK_GRID   1
+#define ORACLE_MASK_TEMPORAL 2   /* whole frames of a video: H = frames, W = positions per frame */
 #define ORACLE_FLAG_SHARE_MASK 1u
 
 /* ------------------------------------------------------------------ */
@@ -124,6 +125,12 @@ int64_t oracle_keep_count(int mode, int64_t H, int64_t W, double r)
         if (K > N) K = N;
         return K;
     }
+    if (mode == ORACLE_MASK_TEMPORAL) {      /* K_T frames of H, each with all its W positions */
+        int64_t KT = (int64_t)floor(r * (double)H + 0.5);
+        if (KT < 1) KT = 1;
+        if (KT > H) KT = H;
+        return KT * W;
+    }
     if (mode == ORACLE_MASK_GRID) {
         int fam = grid_family(r);
         if (!fam) return -1;
@@ -155,7 +162,11 @@ static int cmp_u64(const void* a, const void* b)
  * per-sample prefix keep_offsets[0..B].  Returns M_keep, or -1 on bad input.
  * Random mode: every position gets the 64-bit score (word << 32) | n; the K
  * positions with the smallest scores are kept (all K-subsets equally likely).
- * Grid mode: a periodic 2x2 lattice whose phase is drawn per sample. */
+ * Grid mode: a periodic 2x2 lattice whose phase is drawn per sample.
+ * Temporal mode (Sec. 3.1 and 3.2.1: a subset of video frames): H frames of W
+ * positions; frame f gets the score (word << 32) | f from the same word stream as
+ * position f of a random-mode map, the K_T frames with the smallest scores are
+ * kept, each with all of its positions. */
 int64_t oracle_sample_keep(int mode, int64_t B, int64_t H, int64_t W, double r,
                            uint64_t seed, uint64_t step, int64_t sample_offset,
                            uint32_t flags, int32_t* keep_rows, int32_t* keep_offsets)
@@ -184,6 +195,25 @@ int64_t oracle_sample_keep(int mode, int64_t B, int64_t H, int64_t W, double r,
             for (int64_t k = 0; k < K; ++k) kept[score[k] & 0xffffffffu] = 1;
             for (int64_t n = 0; n < N; ++n)
                 if (kept[n]) keep_rows[out++] = (int32_t)(b * N + n);
+            keep_offsets[b + 1] = (int32_t)out;
+        }
+        free(score); free(kept);
+    } else if (mode == ORACLE_MASK_TEMPORAL) {
+        int64_t KT = oracle_keep_count(mode, H, W, r) / W;
+        uint64_t* score = (uint64_t*)malloc((size_t)H * sizeof(uint64_t));
+        unsigned char* kept = (unsigned char*)malloc((size_t)H);
+        for (int64_t b = 0; b < B; ++b) {
+            uint32_t gid = (flags & ORACLE_FLAG_SHARE_MASK) ? 0u : (uint32_t)(sample_offset + b);
+            for (int64_t f = 0; f < H; ++f) {
+                uint64_t u = position_word(seed, (uint32_t)step, gid, (uint32_t)f);
+                score[f] = (u << 32) | (uint64_t)f;
+            }
+            qsort(score, (size_t)H, sizeof(uint64_t), cmp_u64);
+            memset(kept, 0, (size_t)H);
+            for (int64_t k = 0; k < KT; ++k) kept[score[k] & 0xffffffffu] = 1;
+            for (int64_t f = 0; f < H; ++f)
+                if (kept[f])
+                    for (int64_t q = 0; q < W; ++q) keep_rows[out++] = (int32_t)(b * N + f * W + q);
             keep_offsets[b + 1] = (int32_t)out;
         }
         free(score); free(kept);

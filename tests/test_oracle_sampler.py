@@ -292,3 +292,43 @@ def test_sampler_rejects_out_of_domain():
         oracle.sample_keep(oracle.MASK_RANDOM, 2, 4, 4, 0.5, sample_offset=2 ** 32 - 1)
     with pytest.raises(ValueError):
         oracle.sample_keep(oracle.MASK_GRID, 1, 4, 4, 0.6)
+
+
+# ---------------------------------------------------------------- temporal (whole-frame) masks
+# Sec. 3.1 / 3.2.1: on video the kept subset can be a subset of frames.  Pins: the brute-force
+# selection written out here, whole frames only, the reduction to the (already pinned) random
+# mask on a map of T positions, sharding invariance, the counts.
+@pytest.mark.parametrize("B,T,P,r,seed,step,off", [(3, 8, 5, 0.5, 0, 0, 0), (2, 16, 49, 0.25, 7, 3, 11),
+                                                   (4, 5, 6, 0.75, 1, 9, 0), (1, 32, 196, 0.5, 2, 1, 4)])
+def test_temporal_keep_matches_full_sort_over_frames(B, T, P, r, seed, step, off):
+    rows, offs = oracle.sample_keep(oracle.MASK_TEMPORAL, B, T, P, r, seed, step, off)
+    KT = max(1, min(T, math.floor(r * T + 0.5)))
+    assert oracle.keep_count(oracle.MASK_TEMPORAL, T, P, r) == KT * P
+    assert list(offs) == [b * KT * P for b in range(B + 1)]
+    want = []
+    for b in range(B):
+        scores = sorted((_philox_bigint([f >> 2, off + b, step, 0], [seed & M32, seed >> 32])[f & 3] << 32) | f
+                        for f in range(T))                        # the independent big-integer Philox above
+        frames = sorted(s & M32 for s in scores[:KT])
+        want += [b * T * P + f * P + q for f in frames for q in range(P)]
+    assert list(rows) == want
+
+
+def test_temporal_mask_is_the_random_mask_over_frames_expanded():
+    B, T, P, r = 5, 12, 7, 0.5
+    rows, _ = oracle.sample_keep(oracle.MASK_TEMPORAL, B, T, P, r, 3, 2, 6)
+    frames, _ = oracle.sample_keep(oracle.MASK_RANDOM, B, T, 1, r, 3, 2, 6)          # ids b*T + f
+    expanded = (frames[:, None].astype(np.int64) * P + np.arange(P)[None, :]).reshape(-1)
+    assert np.array_equal(rows, expanded)
+    # whole frames, nothing else: every kept frame contributes all of its P positions
+    per_frame = np.bincount(rows // P, minlength=B * T)
+    assert set(per_frame.tolist()) <= {0, P}
+
+
+def test_temporal_mask_sharding_and_ratio_one():
+    whole, _ = oracle.sample_keep(oracle.MASK_TEMPORAL, 6, 8, 4, 0.5, 5, 1, 0)
+    a, _ = oracle.sample_keep(oracle.MASK_TEMPORAL, 2, 8, 4, 0.5, 5, 1, 0)
+    b, _ = oracle.sample_keep(oracle.MASK_TEMPORAL, 4, 8, 4, 0.5, 5, 1, 2)
+    assert np.array_equal(whole, np.concatenate([a, b + 2 * 8 * 4]))
+    full, offs = oracle.sample_keep(oracle.MASK_TEMPORAL, 2, 8, 4, 1.0)
+    assert np.array_equal(full, np.arange(2 * 8 * 4)) and list(offs) == [0, 32, 64]
