@@ -52,7 +52,7 @@ typedef enum { SBP_F32 = 0, SBP_BF16 = 1 } sbp_dtype;
 
 /* Sec. 4, "How to sample the gradient keep mask?": uniformly random positions,
  * or a structured periodic ("grid-wise") mask. */
-typedef enum { SBP_MASK_RANDOM = 0, SBP_MASK_GRID = 1 } sbp_mask_mode;
+typedef enum { SBP_MASK_RANDOM = 0, SBP_MASK_GRID = 1, SBP_MASK_TEMPORAL = 2 } sbp_mask_mode;
 
 enum {
     SBP_FLAG_SHARE_MASK = 1,  /* every sample of the call uses sample 0's mask (one mask per iteration, Supp. A.4) */
@@ -71,6 +71,8 @@ const char* sbp_status_string(sbp_status s);
  *   SBP_MASK_RANDOM: the exact count K = clamp(floor(r*H*W + 1/2), 1, H*W).
  *   SBP_MASK_GRID:   the largest count any phase of the mask gives (buffer capacity
  *                    per sample); r must be one of 0.25, 0.5, 0.75, 1.0.
+ *   SBP_MASK_TEMPORAL: H is the number of frames, W the positions per frame;
+ *                    clamp(floor(r*H + 1/2), 1, H) whole frames, times W.
  * Returns -1 when H, W <= 0, r outside (0, 1], or the ratio has no grid mask.
  */
 int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_ratio);
@@ -89,6 +91,11 @@ int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_rat
  *     r = 0.5   keep (h + w) mod 2 == p                           (2 phases)
  *     r = 0.75  complement of the r = 0.25 mask                   (4 phases)
  *     r = 1.0   keep everything
+ * SBP_MASK_TEMPORAL (video: the kept subset is a subset of frames, Sec. 3.1 and the
+ *   frame example of Sec. 3.2.1): a sample is H frames of W positions; frame f gets
+ *   the word of position f above, the K_T frames with the smallest scores are kept,
+ *   each with all W positions (rows (b*H + f)*W + q).  At most 2048 frames
+ *   (SBP_ERR_UNSUPPORTED beyond).
  * The mask depends only on (seed, step, g, n): it does not change with how a
  * batch is split over calls or devices.
  *

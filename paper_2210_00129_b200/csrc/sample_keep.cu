@@ -357,7 +357,60 @@ sample_keep_grid_kernel(int family, uint32_t H, uint32_t W, uint32_t k0, uint32_
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// whole-frame masks for video (Sec. 3.1, 3.2.1: a subset of frames): T frames of P positions, the
+// K_T frames with the smallest scores (word << 32) | f are kept, each with all of its positions.
+// T is small (a clip has tens of frames), so one block ranks the frames by counting.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kMaxFrames = 2048;
+
+__global__ void __launch_bounds__(kSampThreads)
+sample_keep_temporal_kernel(uint32_t T, uint32_t P, uint32_t KT, uint32_t k0, uint32_t k1, uint32_t step,
+                            uint32_t first_sample, int share_mask,
+                            int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
+    __shared__ unsigned long long score[kMaxFrames];
+    __shared__ uint32_t kept[kMaxFrames];        // first a flag per frame, then the ascending list of kept frames
+    __shared__ uint32_t list[kMaxFrames];
+    pdl_launch_dependents();
+    pdl_wait();
+    const uint32_t b = blockIdx.x;
+    const uint32_t gid = share_mask ? 0u : first_sample + b;
+    for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
+        const uint32_t w = philox4x32_10(f >> 2, gid, step, 0u, k0, k1).w[f & 3u];
+        score[f] = ((unsigned long long)w << 32) | f;
+    }
+    __syncthreads();
+    for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
+        const unsigned long long mine = score[f];
+        uint32_t rank = 0;
+        for (uint32_t g = 0; g < T; ++g) rank += score[g] < mine;
+        kept[f] = rank < KT ? 1u : 0u;
+    }
+    __syncthreads();
+    for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
+        if (kept[f]) {
+            uint32_t pos = 0;
+            for (uint32_t g = 0; g < f; ++g) pos += kept[g];
+            list[pos] = f;
+        }
+    }
+    __syncthreads();
+    const uint64_t per_sample = (uint64_t)KT * P;
+    int32_t* out = keep_rows + (uint64_t)b * per_sample;
+    for (uint64_t e = threadIdx.x; e < per_sample; e += kSampThreads) {
+        const uint32_t k = (uint32_t)(e / P), q = (uint32_t)(e - (uint64_t)k * P);
+        out[e] = (int32_t)(((uint64_t)b * T + list[k]) * P + q);
+    }
+    if (threadIdx.x == 0) {
+        keep_offsets[b] = (int32_t)((uint64_t)b * per_sample);
+        if (b + 1 == gridDim.x) keep_offsets[b + 1] = (int32_t)((uint64_t)(b + 1) * per_sample);
+    }
+}
+
 }  // namespace
+
+uint32_t sample_keep_max_frames() { return kMaxFrames; }
 
 cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, int64_t W, int64_t K,
                                uint64_t seed, uint32_t step, uint32_t first_sample, bool share_mask,
@@ -385,6 +438,9 @@ cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, 
         return launch_pdl(sample_keep_random_kernel, grid, block, 0, stream, (uint32_t)(H * W), (uint32_t)K, k0, k1,
                           step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
     }
+    if (mode == SBP_MASK_TEMPORAL)      // H frames of W positions; K = kept frames x W
+        return launch_pdl(sample_keep_temporal_kernel, grid, block, 0, stream, (uint32_t)H, (uint32_t)W, (uint32_t)(K / W),
+                          k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
     return launch_pdl(sample_keep_grid_kernel, grid, block, 0, stream, grid_family, (uint32_t)H, (uint32_t)W, k0, k1,
                       step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
 }

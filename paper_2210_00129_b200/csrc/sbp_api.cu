@@ -59,6 +59,12 @@ int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_rat
         if (K > N) K = N;
         return K;
     }
+    if (mode == SBP_MASK_TEMPORAL) {          // H frames of W positions each: whole frames are kept
+        int64_t KT = (int64_t)floor(keep_ratio * (double)H + 0.5);
+        if (KT < 1) KT = 1;
+        if (KT > H) KT = H;
+        return KT * W;
+    }
     if (mode == SBP_MASK_GRID) {
         const int64_t quarter_max = ((H + 1) / 2) * ((W + 1) / 2);   // phase (0, 0) holds the most lattice points
         const int64_t quarter_min = (H / 2) * (W / 2);               // phase (1, 1) the fewest
@@ -76,7 +82,7 @@ int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_rat
 sbp_status sbp_sample_keep(sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, double keep_ratio,
                            uint64_t seed, uint64_t step, int64_t sample_offset, uint32_t flags,
                            int32_t* keep_rows, int32_t* keep_offsets, void* stream) {
-    if (mode != SBP_MASK_RANDOM && mode != SBP_MASK_GRID) return SBP_ERR_INVALID_ARG;
+    if (mode != SBP_MASK_RANDOM && mode != SBP_MASK_GRID && mode != SBP_MASK_TEMPORAL) return SBP_ERR_INVALID_ARG;
     if (keep_rows == nullptr || keep_offsets == nullptr) return SBP_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(keep_rows) & 3u) || (reinterpret_cast<uintptr_t>(keep_offsets) & 3u))
         return SBP_ERR_INVALID_ARG;
@@ -88,6 +94,7 @@ sbp_status sbp_sample_keep(sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, 
     if (sample_offset < 0 || ((uint64_t)(sample_offset + B - 1) >> 32)) return SBP_ERR_INVALID_ARG;
     const int family = grid_family_of(keep_ratio);
     if (mode == SBP_MASK_GRID && family == 0) return SBP_ERR_UNSUPPORTED;
+    if (mode == SBP_MASK_TEMPORAL && H > (int64_t)sample_keep_max_frames()) return SBP_ERR_UNSUPPORTED;
     const int64_t K = sbp_keep_count(mode, H, W, keep_ratio);
     const cudaError_t e = launch_sample_keep((int)mode, family, B, H, W, K, seed, (uint32_t)step,
                                              (uint32_t)sample_offset, (flags & SBP_FLAG_SHARE_MASK) != 0,

@@ -107,6 +107,7 @@ __device__ __forceinline__ PhiloxWords philox4x32_10(uint32_t c0, uint32_t c1, u
 // Launch entry points of the individual kernels (defined in their own .cu files).
 // None synchronises.
 // ---------------------------------------------------------------------------------------------
+uint32_t sample_keep_max_frames();      // most frames a whole-frame (temporal) mask can choose among
 cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, int64_t W, int64_t K,
                                uint64_t seed, uint32_t step, uint32_t first_sample, bool share_mask,
                                int32_t* keep_rows, int32_t* keep_offsets, cudaStream_t stream);

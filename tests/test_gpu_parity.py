@@ -42,6 +42,11 @@ def relerr(got, want):
     (1, 64, 56, 56, 0.5, 0, 3, 0, 0),
     (1, 5, 7, 7, 0.5, 0, 0, 1, sbp.SBP_FLAG_SHARE_MASK),
     (1, 2, 200, 334, 0.5, 1, 0, 0, 0),
+    (2, 4, 8, 196, 0.5, 0, 0, 0, 0),                     # whole frames of a video clip: 8 frames of 14x14 tokens
+    (2, 3, 16, 49, 0.25, 7, 3, 11, 0),
+    (2, 2, 5, 6, 0.75, 1, 9, 0, sbp.SBP_FLAG_SHARE_MASK),
+    (2, 1, 1500, 3, 0.5, 2, 1, 4, 0),                    # many frames: several sweeps of the ranking loops
+    (2, 5, 32, 1, 1.0, 0, 0, 0, 0),
 ])
 def test_keep_indices_bit_exact(mode, B, H, W, r, seed, step, off, flags):
     want_rows, want_offs = oracle.sample_keep(mode, B, H, W, r, seed, step, off, flags)
