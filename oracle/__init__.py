@@ -58,6 +58,8 @@ def _load():
     lib.oracle_linear_backward.restype = None
     lib.oracle_full_backward.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, vp]
     lib.oracle_full_backward.restype = None
+    lib.oracle_linear_forward.argtypes = [vp, vp, vp, i64, i64, i64, vp]
+    lib.oracle_linear_forward.restype = None
     lib.oracle_num_threads.argtypes = []
     lib.oracle_num_threads.restype = ctypes.c_int
     _lib = lib
@@ -114,6 +116,18 @@ def forward_cache(X: np.ndarray, keep_rows: np.ndarray) -> np.ndarray:
     _load().oracle_forward_cache(_ptr(X), X.shape[1] * X.dtype.itemsize, _ptr(rows),
                                  rows.shape[0], _ptr(out))
     return out
+
+
+def linear_forward(X, W, bias=None):
+    """Y = X W (+ bias) in fp64 (Eq. 2)."""
+    X, W = _f64(X), _f64(W)
+    M, C_in = X.shape
+    C_out = W.shape[1]
+    assert W.shape == (C_in, C_out)
+    b = _f64(bias) if bias is not None else None
+    Y = np.empty((M, C_out))
+    _load().oracle_linear_forward(_ptr(X), _ptr(W), _ptr(b), M, C_in, C_out, _ptr(Y))
+    return Y
 
 
 def linear_backward(X_keep, dY, W, keep_rows, want=("dW", "db", "dX")):

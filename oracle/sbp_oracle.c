@@ -246,6 +246,30 @@ void oracle_forward_cache(const void* X, int64_t row_bytes, const int32_t* keep_
 }
 
 /* ------------------------------------------------------------------ */
+/* forward of the layer (Eq. 2; with SBP every row is still computed,   */
+/* Eq. 4 and Algorithm 1: only what is cached differs)                  */
+/* ------------------------------------------------------------------ */
+
+/* Y[m, j] = sum_i X[m, i] * W[i, j] (+ bias[j] when bias is not NULL), the sum over i
+ * in ascending order.  X [M, C_in], W [C_in, C_out] row-major, Y [M, C_out]. */
+void oracle_linear_forward(const double* X, const double* W, const double* bias,
+                           int64_t M, int64_t C_in, int64_t C_out, double* Y)
+{
+    #pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        double* y = Y + m * C_out;
+        for (int64_t j = 0; j < C_out; ++j) y[j] = 0.0;
+        for (int64_t i = 0; i < C_in; ++i) {
+            double x = X[m * C_in + i];
+            const double* w = W + i * C_out;
+            for (int64_t j = 0; j < C_out; ++j) y[j] += x * w[j];
+        }
+        if (bias)
+            for (int64_t j = 0; j < C_out; ++j) y[j] += bias[j];
+    }
+}
+
+/* ------------------------------------------------------------------ */
 /* SBP backward of a linear layer (Eq. 5; bias gradient by the same     */
 /* masking of dY; nothing is rescaled, Eq. 1)                           */
 /* ------------------------------------------------------------------ */

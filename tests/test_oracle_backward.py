@@ -194,3 +194,39 @@ def test_synthetic_inputs_are_reproducible_gaussians():
     # 1 + 2^-8 is a tie -> even (1.0); 1 + 3*2^-8 is a tie -> even (1 + 2^-6)
     assert bits.tolist() == [0x3F80, 0x3F80, 0x3F82, 0xC020, 0x0000]
     assert synth.bf16_bits_to_f64(bits).tolist() == [1.0, 1.0, 1.015625, -2.5, 0.0]
+
+
+# ---------------------------------------------------------------- forward (Eq. 2, Eq. 4)
+def test_forward_hand_worked_integers():
+    X = np.array([[1, 2], [0, -1], [3, 1]], dtype=np.float64)
+    W = np.array([[2, 0, 1], [1, -1, 4]], dtype=np.float64)
+    b = np.array([10, 20, 30], dtype=np.float64)
+    assert oracle.linear_forward(X, W).tolist() == [[4, -2, 9], [-1, 1, -4], [7, -1, 7]]
+    assert oracle.linear_forward(X, W, b).tolist() == [[14, 18, 39], [9, 21, 26], [17, 19, 37]]
+
+
+def test_forward_equals_library_matmul_and_splits_by_rows():
+    rng = np.random.default_rng(3)
+    X, W, b = rng.standard_normal((37, 19)), rng.standard_normal((19, 23)), rng.standard_normal(23)
+    Y = oracle.linear_forward(X, W, b)
+    assert np.allclose(Y, X @ W + b, rtol=1e-13, atol=1e-13)
+    assert not np.allclose(Y, X @ W, atol=1e-3) and not np.allclose(Y, (W.T @ X.T).T[:, ::-1] + b, atol=1e-3)
+    # Eq. 4: the forward of the kept rows and of the dropped rows, put back in place, is the full forward
+    keep = np.sort(rng.choice(37, 18, replace=False))
+    drop = np.setdiff1d(np.arange(37), keep)
+    Z = np.empty_like(Y)
+    Z[keep] = oracle.linear_forward(X[keep], W, b)
+    Z[drop] = oracle.linear_forward(X[drop], W, b)
+    assert np.array_equal(Z, Y)
+
+
+def test_forward_and_backward_are_adjoint():
+    # <Y(W + E) - Y(W), G> = <E, dW(G)> and <Y(X + D) - Y(X), G> = <D, dX(G)> exactly (bilinearity, Eq. 2 and Eq. 3)
+    rng = np.random.default_rng(4)
+    X, W = rng.integers(-3, 4, (11, 6)).astype(np.float64), rng.integers(-3, 4, (6, 5)).astype(np.float64)
+    G, E, D = (rng.integers(-3, 4, s).astype(np.float64) for s in ((11, 5), (6, 5), (11, 6)))
+    full = oracle.full_backward(X, G, W)
+    assert np.sum((oracle.linear_forward(X, W + E) - oracle.linear_forward(X, W)) * G) == np.sum(E * full["dW"])
+    assert np.sum((oracle.linear_forward(X + D, W) - oracle.linear_forward(X, W)) * G) == np.sum(D * full["dX"])
+    b = rng.integers(-3, 4, 5).astype(np.float64)
+    assert np.sum((oracle.linear_forward(X, W, b) - oracle.linear_forward(X, W)) * G) == np.sum(b * full["db"])
