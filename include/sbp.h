@@ -130,6 +130,28 @@ sbp_status sbp_forward_cache(sbp_dtype dt, const void* X /* dev */, int64_t M, i
                              const int32_t* M_keep_dev /* dev, nullable */,
                              int64_t M_keep_cap, void* X_keep /* dev */, void* stream);
 
+/*
+ * Forward of the layer with the SBP cache fused in (Eq. 2: Y = X W; with SBP every
+ * row is still computed, Eq. 4, and only the kept rows of the input are retained for
+ * the backward pass, Algorithm 1):
+ *   Y[m, j]      = sum_i X[m, i] * W[i, j] + bias[j]            dt [M, C_out]
+ *   X_keep[m, :] = X[keep_rows[m], :] for m < M_keep, zero rows up to M_keep_cap
+ * X [M, C_in], W [C_in, C_out], bias fp32 [C_out] or NULL.  X_keep may be NULL (no
+ * cache: keep_rows and M_keep_dev are then ignored); otherwise it is what
+ * sbp_forward_cache would produce, written by the same launch so that X is read
+ * from memory once.  SBP_BF16: bf16 inputs and output, fp32 accumulation on the
+ * tensor cores, one rounding of (sum + bias) to bf16.  SBP_F32: fp32 FMA arithmetic.
+ * C_in and C_out must be multiples of 8 (bf16) / 4 (fp32), else SBP_ERR_UNSUPPORTED.
+ * flags: SBP_FLAG_PLAIN_FMA or 0.  status_word as for sbp_linear_backward.
+ * SBP_ERR_INVALID_ARG for null or misaligned (16 bytes) pointers and bad sizes.
+ */
+sbp_status sbp_linear_forward(sbp_dtype dt, const void* X /* dev */, const void* W /* dev */,
+                              const float* bias /* dev, nullable */, int64_t M, int64_t C_in, int64_t C_out,
+                              void* Y /* dev */, const int32_t* keep_rows /* dev, nullable with X_keep */,
+                              const int32_t* M_keep_dev /* dev, nullable */, int64_t M_keep_cap,
+                              void* X_keep /* dev, nullable */, uint32_t flags,
+                              int32_t* status_word /* dev, nullable */, void* stream);
+
 /* Scratch bytes sbp_linear_backward needs for these sizes (never 0). */
 size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap,
                                            int64_t C_in, int64_t C_out);

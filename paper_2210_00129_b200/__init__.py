@@ -24,7 +24,7 @@ SBP_MASK_RANDOM, SBP_MASK_GRID, SBP_MASK_TEMPORAL = 0, 1, 2
 SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
 SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT = 16, 32
 
-EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache",
+EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
            "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static")
 
@@ -56,6 +56,8 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_sample_keep.restype = ci
     lib.sbp_forward_cache.argtypes = [ci, vp, i64, i64, vp, vp, i64, vp, vp]
     lib.sbp_forward_cache.restype = ci
+    lib.sbp_linear_forward.argtypes = [ci, vp, vp, vp, i64, i64, i64, vp, vp, vp, i64, vp, u32, vp, vp]
+    lib.sbp_linear_forward.restype = ci
     lib.sbp_linear_backward_workspace_bytes.argtypes = [ci, i64, i64, i64, i64]
     lib.sbp_linear_backward_workspace_bytes.restype = sz
     lib.sbp_linear_backward.argtypes = [ci, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp, u32, vp, sz, vp, vp]
@@ -119,6 +121,17 @@ def sbp_forward_cache(dt, X, M, C, keep_rows, M_keep_dev, M_keep_cap, X_keep, st
                                          _ptr(X_keep), _stream(stream))
     if check:
         _check(s, "sbp_forward_cache")
+    return s
+
+
+def sbp_linear_forward(dt, X, W, bias, M, C_in, C_out, Y, keep_rows=None, M_keep_dev=None, M_keep_cap=0, X_keep=None,
+                       flags=0, status_word=None, stream=None, check=True) -> int:
+    """Y = X W + bias; with X_keep given the same launch also writes the forward cache."""
+    s = load_library().sbp_linear_forward(dt, _ptr(X), _ptr(W), _ptr(bias), M, C_in, C_out, _ptr(Y), _ptr(keep_rows),
+                                          _ptr(M_keep_dev), M_keep_cap, _ptr(X_keep), flags, _ptr(status_word),
+                                          _stream(stream))
+    if check:
+        _check(s, "sbp_linear_forward")
     return s
 
 

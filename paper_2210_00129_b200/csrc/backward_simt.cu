@@ -184,7 +184,69 @@ simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t*
     }
 }
 
+
+// Forward of the layer, Y[m, j] = sum_i X[m, i] * W[i, j] + bias[j] (Eq. 2): 64 x 64 outputs per block.
+// The X tile is loaded along i (its contiguous side) and stored transposed, the W tile along j.
+template <typename T>
+__global__ void __launch_bounds__(kSimtThreads)
+simt_forward_kernel(const T* __restrict__ X, const T* __restrict__ W, const float* __restrict__ bias, int64_t M,
+                    int C_in, int C_out, T* __restrict__ Y, const int32_t* __restrict__ status_word) {
+    __shared__ __align__(16) float As[kTileK][kTile + 4];
+    __shared__ __align__(16) float Bs[kTileK][kTile];
+    pdl_launch_dependents();
+    pdl_wait();
+    if (status_word != nullptr && *status_word != 0) return;
+    const int64_t m0 = (int64_t)blockIdx.x * kTile;
+    const int j0 = blockIdx.y * kTile;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int ar = threadIdx.x >> 2, ac = (threadIdx.x & 3) * 4;      // X loader: tile row, 4 of the 16 k columns
+    const int bk = threadIdx.x >> 4, bc = (threadIdx.x & 15) * 4;     // W loader: k row, 4 of the 64 columns
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    float acc[4][4] = {};
+    for (int i0 = 0; i0 < C_in; i0 += kTileK) {
+        float4 a = zero4, b = zero4;
+        if (m0 + ar < M && i0 + ac < C_in) a = load4<T>(X + (m0 + ar) * C_in + i0 + ac);
+        if (i0 + bk < C_in && j0 + bc < C_out) b = load4<T>(W + (int64_t)(i0 + bk) * C_out + j0 + bc);
+        As[ac + 0][ar] = a.x; As[ac + 1][ar] = a.y; As[ac + 2][ar] = a.z; As[ac + 3][ar] = a.w;
+        *reinterpret_cast<float4*>(&Bs[bk][bc]) = b;
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kTileK; ++k) {
+            const float4 av = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+            const float4 bv = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+            const float a4[4] = {av.x, av.y, av.z, av.w}, b4[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(a4[r], b4[c], acc[r][c]);
+        }
+        __syncthreads();
+    }
+    const int j = j0 + tx * 4;
+    if (j < C_out) {
+        float4 bv = zero4;
+        if (bias != nullptr) bv = __ldg(reinterpret_cast<const float4*>(bias + j));
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int64_t m = m0 + ty * 4 + r;
+            if (m < M)
+                store4<T>(Y + m * C_out + j, make_float4(acc[r][0] + bv.x, acc[r][1] + bv.y, acc[r][2] + bv.z, acc[r][3] + bv.w));
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_simt_forward(sbp_dtype dt, const void* X, const void* W, const float* bias, int64_t M, int64_t C_in,
+                                int64_t C_out, void* Y, const int32_t* status_word, cudaStream_t stream) {
+    const dim3 grid((unsigned)((M + kTile - 1) / kTile), (unsigned)((C_out + kTile - 1) / kTile));
+    if (dt == SBP_BF16)
+        return launch_pdl(simt_forward_kernel<__nv_bfloat16>, grid, dim3(kSimtThreads), 0, stream,
+                          (const __nv_bfloat16*)X, (const __nv_bfloat16*)W, bias, M, (int)C_in, (int)C_out,
+                          (__nv_bfloat16*)Y, status_word);
+    return launch_pdl(simt_forward_kernel<float>, grid, dim3(kSimtThreads), 0, stream, (const float*)X, (const float*)W,
+                      bias, M, (int)C_in, (int)C_out, (float*)Y, status_word);
+}
 
 size_t simt_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
     const int s = simt_dw_splits(M_keep_cap, C_in, C_out);

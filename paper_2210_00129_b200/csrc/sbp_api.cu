@@ -115,6 +115,33 @@ sbp_status sbp_forward_cache(sbp_dtype dt, const void* X, int64_t M, int64_t C, 
     return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
 }
 
+sbp_status sbp_linear_forward(sbp_dtype dt, const void* X, const void* W, const float* bias, int64_t M, int64_t C_in,
+                              int64_t C_out, void* Y, const int32_t* keep_rows, const int32_t* M_keep_dev,
+                              int64_t M_keep_cap, void* X_keep, uint32_t flags, int32_t* status_word, void* stream_v) {
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (X == nullptr || W == nullptr || Y == nullptr) return SBP_ERR_INVALID_ARG;
+    if (M <= 0 || M >= (1ll << 31) || C_in <= 0 || C_out <= 0 || C_in >= (1ll << 24) || C_out >= (1ll << 24))
+        return SBP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(bias) || !aligned16(X_keep))
+        return SBP_ERR_INVALID_ARG;
+    if (X_keep != nullptr) {
+        if (keep_rows == nullptr || (reinterpret_cast<uintptr_t>(keep_rows) & 3u) || M_keep_cap < 0 || M_keep_cap > M)
+            return SBP_ERR_INVALID_ARG;
+    }
+    const int64_t mult = (dt == SBP_BF16) ? 8 : 4;
+    if (C_in % mult != 0 || C_out % mult != 0) return SBP_ERR_UNSUPPORTED;
+    if (dt == SBP_BF16 && !(flags & SBP_FLAG_PLAIN_FMA) && tc_forward_supported(M, C_in, C_out))
+        return launch_tc_forward(X, W, bias, M, C_in, C_out, Y, keep_rows, M_keep_dev, M_keep_cap, X_keep, status_word,
+                                 stream);
+    if (launch_simt_forward(dt, X, W, bias, M, C_in, C_out, Y, status_word, stream) != cudaSuccess) return SBP_ERR_CUDA;
+    if (X_keep != nullptr &&
+        launch_gather_rows(X, C_in * (dt == SBP_BF16 ? 2 : 4), keep_rows, M_keep_dev, M_keep_cap, X_keep, stream) !=
+            cudaSuccess)
+        return SBP_ERR_CUDA;
+    return SBP_OK;
+}
+
 size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                            int64_t C_out) {
     if (M <= 0 || M_keep_cap < 0 || C_in <= 0 || C_out <= 0) return 256;
