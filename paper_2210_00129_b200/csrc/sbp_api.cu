@@ -131,9 +131,25 @@ sbp_status sbp_linear_forward(sbp_dtype dt, const void* X, const void* W, const 
     }
     const int64_t mult = (dt == SBP_BF16) ? 8 : 4;
     if (C_in % mult != 0 || C_out % mult != 0) return SBP_ERR_UNSUPPORTED;
-    if (dt == SBP_BF16 && !(flags & SBP_FLAG_PLAIN_FMA) && tc_forward_supported(M, C_in, C_out))
-        return launch_tc_forward(X, W, bias, M, C_in, C_out, Y, keep_rows, M_keep_dev, M_keep_cap, X_keep, status_word,
-                                 stream);
+    if (dt == SBP_BF16 && !(flags & SBP_FLAG_PLAIN_FMA) && tc_forward_supported(M, C_in, C_out)) {
+        // The cache rides along in the product kernel (four side warps per SM, about 12 GB/s each SM) when that
+        // copy takes no more than a quarter of the product's own time (a longer one slows the operand loads down more than
+        // a second launch costs); otherwise the stand-alone gather kernel follows.
+        bool ride = X_keep != nullptr;
+        if (ride) {
+            const double copy_us = (double)M_keep_cap * (double)C_in * 2.0 / (double)kNumSMs / 12e3;
+            const double flop_us = 2.0 * (double)M * (double)C_in * (double)C_out / 1.0e9;            // at 1000 TFLOP/s
+            const double byte_us = ((double)M * (double)(C_in + C_out) * 2.0) / 5.0e6;                 // at 5 TB/s
+            ride = copy_us <= 0.25 * (flop_us > byte_us ? flop_us : byte_us);
+        }
+        const sbp_status s = launch_tc_forward(X, W, bias, M, C_in, C_out, Y, keep_rows, M_keep_dev, M_keep_cap,
+                                               ride ? X_keep : nullptr, status_word, stream);
+        if (s != SBP_OK) return s;
+        if (X_keep != nullptr && !ride &&
+            launch_gather_rows(X, C_in * 2, keep_rows, M_keep_dev, M_keep_cap, X_keep, stream) != cudaSuccess)
+            return SBP_ERR_CUDA;
+        return SBP_OK;
+    }
     if (launch_simt_forward(dt, X, W, bias, M, C_in, C_out, Y, status_word, stream) != cudaSuccess) return SBP_ERR_CUDA;
     if (X_keep != nullptr &&
         launch_gather_rows(X, C_in * (dt == SBP_BF16 ? 2 : 4), keep_rows, M_keep_dev, M_keep_cap, X_keep, stream) !=

@@ -172,7 +172,7 @@ tc_forward_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             const int64_t vpr = C_in / 8;                                  // 16-byte vectors per row
             const int64_t all = p.M_keep_cap * vpr, valid = M_keep * vpr;
             const int64_t stride = (int64_t)gridDim.x * kFwdSideThreads;
-            constexpr int kU = 4;
+            constexpr int kU = 16;                                        // 16-byte loads in flight per thread
             for (int64_t base = (int64_t)blockIdx.x * kFwdSideThreads + (threadIdx.x - kFwdSideWarp0 * 32); base < all;
                  base += stride * kU) {
                 int64_t src[kU];

@@ -1,6 +1,6 @@
 """Per-call timing sweep over the paper's layer shapes, against the roofline of each call.
 
-    python -m paper_2210_00129_b200.measure [--group vit|convnext|detection|blocks|sampler|all] [--iters 24]
+    python -m paper_2210_00129_b200.measure [--group vit|convnext|detection|forward|blocks|sampler|all] [--iters 24]
 
 For every layer of the chosen groups (ViT-B/16 MLP and attention projections at four keep ratios,
 ConvNeXt-B point-wise layers of the four stages with random and grid masks, the detection-resolution
@@ -200,6 +200,49 @@ def mlp_block(bench, B, H, W_, d, h, r):
     return cap, t_scatter, t_packed, flop
 
 
+def forward_layers(bench, pk):
+    """sbp_linear_forward with the cache fused in, against the forward alone followed by sbp_forward_cache."""
+    rows = []
+    for name, B, H, W_, C_in, C_out, r in (("vit_b16 fc1 B=64", 64, 14, 14, 768, 3072, 0.5), ("vit_b16 fc2 B=64", 64, 14, 14, 3072, 768, 0.5),
+                                           ("vit_b16 fc1 B=128", 128, 14, 14, 768, 3072, 0.5), ("vit_b16 qkv B=128", 128, 14, 14, 768, 2304, 0.5),
+                                           ("convnext_b s1 pw1", 64, 56, 56, 128, 512, 0.5), ("convnext_b s1 pw2", 64, 56, 56, 512, 128, 0.5),
+                                           ("convnext_b s3 pw1", 64, 14, 14, 512, 2048, 0.5)):
+        M = B * H * W_
+        cap = B * sbp.sbp_keep_count(0, H, W_, r)
+        gen = torch.Generator(device="cuda").manual_seed(7)
+        set_bytes = (M * C_in + M * C_out + C_in * C_out + cap * C_in) * 2
+        n_sets = max(3, int(400e6 // set_bytes) + 1)
+        sets = [dict(X=torch.randn(M, C_in, device="cuda", generator=gen).bfloat16(),
+                     W=(torch.randn(C_in, C_out, device="cuda", generator=gen) * 0.02).bfloat16(),
+                     b=torch.randn(C_out, device="cuda", generator=gen), Y=torch.zeros(M, C_out, device="cuda", dtype=torch.bfloat16),
+                     Xk=torch.zeros(cap, C_in, device="cuda", dtype=torch.bfloat16), rows=torch.zeros(cap, dtype=torch.int32, device="cuda"),
+                     offs=torch.zeros(B + 1, dtype=torch.int32, device="cuda")) for _ in range(n_sets)]
+        torch.cuda.synchronize()
+        with torch.cuda.stream(bench.stream):
+            for s in sets:
+                sbp.sbp_sample_keep(0, B, H, W_, r, 0, 0, 0, 0, s["rows"], s["offs"], stream=bench.sid)
+        bench.stream.synchronize()
+
+        def fused(k, i):
+            s = sets[k]
+            sbp.sbp_linear_forward(sbp.SBP_BF16, s["X"], s["W"], s["b"], M, C_in, C_out, s["Y"], s["rows"], None, cap, s["Xk"],
+                                   stream=bench.sid)
+
+        def separate(k, i):
+            s = sets[k]
+            sbp.sbp_linear_forward(sbp.SBP_BF16, s["X"], s["W"], s["b"], M, C_in, C_out, s["Y"], stream=bench.sid)
+            sbp.sbp_forward_cache(sbp.SBP_BF16, s["X"], M, C_in, s["rows"], None, cap, s["Xk"], stream=bench.sid)
+
+        tf, ts = bench.time_us(fused, n_sets), bench.time_us(separate, n_sets)
+        flop = 2.0 * M * C_in * C_out
+        by = (M * C_in + C_in * C_out + M * C_out + cap * C_in) * 2.0
+        tmin = max(flop / (pk["bf16_tflops_sustained"] * 1e12), by / (pk["hbm_gbs"] * 1e9)) * 1e6
+        rows.append((name, M, tf, ts, tmin, flop / tf / 1e6))
+        del sets
+        torch.cuda.empty_cache()
+    return rows
+
+
 def sampler_stress(bench, pk):
     """Sampler alone on a shape whose index stream is large enough to read as bandwidth."""
     rows = []
@@ -216,7 +259,7 @@ def sampler_stress(bench, pk):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--group", default="all", choices=["vit", "convnext", "detection", "blocks", "sampler", "all"])
+    ap.add_argument("--group", default="all", choices=["vit", "convnext", "detection", "forward", "blocks", "sampler", "all"])
     ap.add_argument("--iters", type=int, default=24)
     ap.add_argument("--compact", action="store_true", help="one table row per layer: us (t_min / t) per call")
     args = ap.parse_args()
@@ -225,7 +268,7 @@ def main():
     bench = Bench(args.iters)
     print(f"peaks ({kind}): bf16 {pk['bf16_tflops_sustained']:.0f} TFLOP/s sustained, HBM {pk['hbm_gbs']:.0f} GB/s; "
           f"{args.iters} graph-replayed launches per figure, rotating buffer sets larger than L2\n")
-    if args.group not in ("sampler", "blocks"):
+    if args.group not in ("sampler", "blocks", "forward"):
         if args.compact:
             print("us (t_min / t) per call; bound of the whole backward in the last column\n")
             print("| layer | M_keep | sample | cache | db | dW | dX | backward (dW+db+dX) | TFLOP/s | bound |")
@@ -262,6 +305,12 @@ def main():
             print("\n| layer | keep ratio | backward us | at keep 1.0 us | speed-up | 1/r |")
             print("|---|---|---|---|---|---|")
             print("\n".join(lines))
+    if args.group in ("forward", "all"):
+        print("\n| forward Y = XW + b with the cache (sbp_linear_forward) | M | fused us | forward + sbp_forward_cache us | "
+              "t_min us | t_min/t | TFLOP/s |")
+        print("|---|---|---|---|---|---|---|")
+        for name, M, tf, ts, tmin, tfl in forward_layers(bench, pk):
+            print(f"| {name} | {M} | {tf:.1f} | {ts:.1f} | {tmin:.1f} | {tmin / tf:.2f} | {tfl:.0f} |")
     if args.group in ("blocks", "all"):
         print("\n| two-layer block backward, d -> 4d -> d (both layers, dW + db + dX each) | M_keep | gradient between "
               "the layers scattered, us | packed, us | gain | packed TFLOP/s |")
