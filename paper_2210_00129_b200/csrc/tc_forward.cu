@@ -32,7 +32,7 @@ constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
 constexpr uint32_t kAccCols = 256;
 constexpr int kEpiBarrier = 2;
-constexpr uint32_t kEpiBytes = 4 * 4096;             // one 4 KB transpose buffer per epilogue warp
+constexpr uint32_t kEpiBytes = 4 * 4096 + 2 * 256 * 4;   // one 4 KB transpose buffer per epilogue warp + two bias strips
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kEpiBytes + 1024;
 
 struct FwdControl {
@@ -201,12 +201,21 @@ tc_forward_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         bool ok = true;
         uint8_t* wbuf = smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256 + warp * 4096;
         const int sub = lane >> 3, ch = lane & 7;
+        int staged_n0[2] = {-1, -1};
         for (uint32_t q = blockIdx.x; q < total; q += gridDim.x, ++used) {
             const uint32_t acc = used & 1u;
             const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
             const int64_t m0 = (int64_t)(q / ncol) * kBM + warp * 32;
             const int n0 = (int)((q % ncol) * BN);
             const int strip_cols = (C_out - n0 < BN) ? C_out - n0 : BN;     // multiple of 8
+            // The tile's strip of the bias goes to shared memory first (two buffers, by tile parity): read from
+            // global memory inside the loop below, its 64 dependent loads per tile doubled the kernel's time.
+            float* bias_s = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256 + 4 * 4096) +
+                            (used & 1u) * 256;
+            if (p.bias != nullptr && staged_n0[used & 1u] != n0) {        // with one or two column tiles the strip never changes
+                for (int c = threadIdx.x; c < BN; c += 128) bias_s[c] = (n0 + c < C_out) ? __ldg(p.bias + n0 + c) : 0.f;
+                staged_n0[used & 1u] = n0;
+            }
             if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
             ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);                      // the four warps go on, or give up, together
             if (!ok) break;
@@ -222,10 +231,9 @@ tc_forward_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
                 for (int qd = 0; qd < 8; ++qd) {
                     float* f = (qd < 4) ? &va[qd * 8] : &vb[(qd - 4) * 8];
-                    const int col = n0 + c0 + qd * 8;
-                    if (p.bias != nullptr && c0 + qd * 8 < strip_cols) {
-                        const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + col));
-                        const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + col + 4));
+                    if (p.bias != nullptr) {
+                        const float4 b0 = *reinterpret_cast<const float4*>(bias_s + c0 + qd * 8);
+                        const float4 b1 = *reinterpret_cast<const float4*>(bias_s + c0 + qd * 8 + 4);
                         f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
                         f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
                     }
