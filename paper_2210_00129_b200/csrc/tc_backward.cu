@@ -81,7 +81,6 @@ struct TcParams {
     int64_t dw_split_stride;       // elements between partial buffers
     int dw_splits;
     int dw_accumulate;             // add into dW_out (only with one split)
-    int dw_tma;                    // dW tiles leave through TMA stores (dW_out is 16-byte aligned)
     float* db_partial;             // nullptr: no bias sums; else [gridDim.x, C_out] per-CTA column sums of kept dY rows
     int32_t* status_word;
 };
@@ -548,7 +547,6 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 }
             } else {
                 // ---- dW tile: accumulator row = output column j, accumulator column = output row i ----
-                // a warp-wide store of one accumulator column covers 32 consecutive j: 128 contiguous bytes
                 const int j = (int)(t.row_tile * kBM) + warp * 32 + lane;
                 const int i0 = (int)(t.col_tile * BNW);
                 float* out_col = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i0 * C_out + j;
@@ -561,23 +559,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);            // the four epilogue warps go on, or give up, together
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                // The two cases are separate loops of explicit stores on purpose: written as one conditional
-                // expression the compiler reads the old value in both cases, and a plain write then waits
-                // for a load of memory it is about to overwrite.
                 const bool add_in = p.dw_accumulate != 0;
-                auto store_cols = [&](const float (&v)[32], int c0) {    // 32 accumulator columns = 32 rows of dW
-                    if (j >= C_out) return;
-                    if (add_in) {
-#pragma unroll
-                        for (int r = 0; r < 32; ++r)
-                            if (i0 + c0 + r < C_in) out_col[(int64_t)(c0 + r) * C_out] += v[r];
-                    } else {
-#pragma unroll
-                        for (int r = 0; r < 32; ++r)
-                            if (i0 + c0 + r < C_in) ptx::st_global_f32(out_col + (int64_t)(c0 + r) * C_out, v[r]);
-                    }
-                };
-                if (p.dw_tma) {
+                {
                     // 16 rows of dW x 128 columns at a time: registers -> staging buffer -> one TMA store (or
                     // reduce-add), which clips at the edges of dW.  A buffer is rewritten three chunks later;
                     // the issuing thread has by then waited for all but the newest store to have read theirs.
@@ -602,19 +585,6 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             else ptx::tma_store_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
                             ptx::bulk_commit();
                         }
-                    }
-                } else {
-                    float va[32], vb[32];
-                    ptx::tmem_ld_32x32(taddr, va);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int c0 = 0; c0 < BNW; c0 += 64) {
-                        ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 32), vb);
-                        store_cols(va, c0);
-                        ptx::tmem_ld_wait();
-                        if (c0 + 64 < BNW) ptx::tmem_ld_32x32(taddr + (uint32_t)(c0 + 64), va);
-                        store_cols(vb, c0 + 32);
-                        ptx::tmem_ld_wait();
                     }
                 }
             }
@@ -835,9 +805,8 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     prm.dw_split_stride = C_in * C_out;
     prm.dw_splits = pl.splits;
     prm.dw_accumulate = (pl.splits == 1 && accumulate) ? 1 : 0;
-    // TMA stores need a 16-byte aligned base; any other dW pointer takes the plain-store epilogue
-    prm.dw_tma = (want_dw && reinterpret_cast<uintptr_t>(prm.dW_out) % 16 == 0) ? 1 : 0;
-    if (prm.dw_tma) {
+    // the dW tiles leave through TMA stores: dW and the workspace are 16-byte aligned (checked at the entry point)
+    if (want_dw) {
         if (!make_map_dw(&map_dw, prm.dW_out, pl.splits, C_in, C_out)) return SBP_ERR_CUDA;
     } else {
         map_dw = map_x;                                              // never used
