@@ -41,7 +41,8 @@ constexpr uint32_t kUmmaK = 16;          // reduction depth of one tcgen05.mma f
 constexpr uint32_t kRowBytes = 128;      // bytes per swizzled smem row
 constexpr uint32_t kAtomBytes = 1024;    // 8 rows x 128 B: one swizzle atom
 constexpr uint32_t kBlock64Bytes = 64 * kRowBytes;   // a 64-row slab (MN-major operands: one 64-wide block)
-constexpr int kStages = 4;
+constexpr int kStages = 4;               // ring depth with 256-wide tiles (48 KB stages)
+constexpr int kStagesNarrow = 6;         // ... when both tile kinds are 128 wide (32 KB stages): same 192 KB, half as many again in flight
 constexpr uint32_t kABytes = kBM * kRowBytes;        // 16 KB
 constexpr uint32_t kBBytesMax = 256 * kRowBytes;     // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytesMax;
@@ -55,13 +56,15 @@ constexpr int kEpiChunk = 16;            // accumulator columns (= rows of dW) p
 constexpr int kEpiBufs = 3;              // staging buffers the dW epilogue rotates through
 constexpr uint32_t kEpiBufBytes = kEpiChunk * kBM * sizeof(float);   // 8 KB: 16 rows of dW x 128 columns
 constexpr int kEpiBarrier = 2;           // named barrier of the four epilogue warps
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 256 + kBiasSmemBytes + kEpiBufs * kEpiBufBytes + 1024;   // ring + control + bias + staging + slack
+constexpr uint32_t kRingBytes = kStages * kStageBytes;
+static_assert(kRingBytes == kStagesNarrow * (kABytes + 128 * kRowBytes), "both ring shapes fill the same memory");
+constexpr uint32_t kSmemBytes = kRingBytes + 256 + kBiasSmemBytes + kEpiBufs * kEpiBufBytes + 1024;   // ring + control + bias + staging + slack
 static_assert((256 + kBiasSmemBytes) % 128 == 0, "staging buffers start on a 128-byte boundary");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory per block");
 
 struct TcControl {
-    uint64_t full_bar[kStages];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
-    uint64_t empty_bar[kStages];   // 1 arrival: tcgen05.commit of the MMAs that read the stage
+    uint64_t full_bar[kStagesNarrow];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
+    uint64_t empty_bar[kStagesNarrow];   // 1 arrival: tcgen05.commit of the MMAs that read the stage
     uint64_t acc_full[2];          // 1 arrival: all MMAs of the tile in this accumulator have finished
     uint64_t acc_empty[2];         // 4 arrivals: each epilogue warp has read the accumulator out
     uint32_t tmem_slot;
@@ -160,7 +163,17 @@ __device__ __forceinline__ uint32_t swizzled(uint32_t row, uint32_t chunk) {
 // row (to the end of dX if it holds the very last kept row).  The rows are walked in windows of 32; a
 // warp-wide OR marks the kept rows of a window, the rest get zeros.  One warp, no other data needed:
 // the side warps run this for every dX tile of the block while the tensor pipe works.
-template <int BNX>
+// Row lookups of the kernel: with kPacked false both row maps are the keep_rows list (the usual, scattered
+// form) and the lookup is a plain load; the packed forms for chained layers allow a null map (row m itself).
+// Kept apart at compile time (and, in the usual form, read through one pointer): the extra test and the
+// second pointer, small as they are, cost the usual form 5 us on ViT-B fc1.
+template <bool kPacked>
+__device__ __forceinline__ int32_t map_row(const int32_t* rows, int64_t m) {
+    if constexpr (kPacked) return mapped_row(rows, m);
+    else return __ldg(rows + m);
+}
+
+template <int BNX, bool kPacked>
 __device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile& t, int64_t M_keep, int wq, int lane) {
     const int C_in = p.C_in;
     const int n0 = (int)(t.col_tile * BNX);
@@ -169,8 +182,8 @@ __device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile&
     const int64_t m0 = (int64_t)t.row_tile * kBM;
     const int64_t m = m0 + wq * 32 + lane;
     const bool valid = m < M_keep;
-    const int64_t cur = valid ? (int64_t)mapped_row(p.dx_rows, m) : -1;
-    const int64_t prev = (valid && m > 0) ? (int64_t)mapped_row(p.dx_rows, m - 1) : -1;
+    const int64_t cur = valid ? (int64_t)map_row<kPacked>(kPacked ? p.dx_rows : p.dy_rows, m) : -1;
+    const int64_t prev = (valid && m > 0) ? (int64_t)map_row<kPacked>(kPacked ? p.dx_rows : p.dy_rows, m - 1) : -1;
     const int nvalid = __popc(__ballot_sync(0xffffffffu, valid));
     if (nvalid == 0) return;
     const int64_t lo = __shfl_sync(0xffffffffu, prev, 0) + 1;
@@ -203,20 +216,24 @@ __device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile&
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int BNX, int BNW, int kBiasDepth>
+template <int BNX, int BNW, int kBiasDepth, bool kPacked>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                    const __grid_constant__ CUtensorMap map_dw, const TcParams p) {
+    // narrow layers (both tile kinds 128 wide) move 32 KB per stage: six stages then fill the ring
+    constexpr bool kNarrow = BNX <= 128 && BNW <= 128;
+    constexpr int kS = kNarrow ? kStagesNarrow : kStages;
+    constexpr uint32_t kSB = kABytes + (kNarrow ? 128u : 256u) * kRowBytes;
     extern __shared__ uint8_t smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
     const uint32_t ring = (raw_addr + 1023u) & ~1023u;              // swizzle atoms need 1024-byte alignment
-    TcControl* ctl = reinterpret_cast<TcControl*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes);
+    TcControl* ctl = reinterpret_cast<TcControl*>(smem_raw + (ring - raw_addr) + kRingBytes);
 
     // ---- set-up that needs nothing from earlier kernels: overlaps their tail ----
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kS; ++s) {
             ptx::mbar_init(ptx::smem_addr(&ctl->full_bar[s]), 1 + kGatherThreads);
             ptx::mbar_init(ptx::smem_addr(&ctl->empty_bar[s]), 1);
         }
@@ -255,11 +272,11 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 if (q >= sched.total) break;
                 const Tile t = decode_tile(sched, q);
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
-                    const int s = it % kStages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                    const int s = it % kS;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kS) & 1u) ^ 1u, abort_flag, status_word);
                     if (!ok) break;
                     const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
-                    const uint32_t a_dst = ring + s * kStageBytes;
+                    const uint32_t a_dst = ring + s * kSB;
                     if (t.is_dw) {                                   // X_keep tile: BNW/64 blocks of 64 columns x 64 kept rows
                         const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.col_tile * BNW);
                         ptx::mbar_arrive_expect_tx(full, BNW * kRowBytes);
@@ -273,10 +290,10 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 }
             }
             if (!ok) {   // let the copies already issued land before shared memory goes away
-                for (uint32_t j = (it > (uint32_t)kStages ? it - kStages : 0u); j < it; ++j) {
-                    const uint32_t bar = ptx::smem_addr(&ctl->full_bar[j % kStages]);
+                for (uint32_t j = (it > (uint32_t)kS ? it - kS : 0u); j < it; ++j) {
+                    const uint32_t bar = ptx::smem_addr(&ctl->full_bar[j % kS]);
                     for (int spin = 0; spin < (1 << 14); ++spin)
-                        if (ptx::mbar_try_wait(bar, (j / kStages) & 1u)) break;
+                        if (ptx::mbar_try_wait(bar, (j / kS) & 1u)) break;
                 }
             }
         }
@@ -303,12 +320,12 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const uint32_t k_step = t.is_dw ? kUmmaK * kRowBytes : kUmmaK * 2;
                 const uint32_t lbo = t.is_dw ? kBlock64Bytes : 16;
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
-                    const int s = it % kStages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / kStages) & 1u, abort_flag, status_word);
+                    const int s = it % kS;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->full_bar[s]), (it / kS) & 1u, abort_flag, status_word);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     ptx::fence_async_proxy();        // the gathered operand was written by cp.async (generic proxy)
-                    const uint32_t a_addr = ring + s * kStageBytes, b_addr = a_addr + kABytes;
+                    const uint32_t a_addr = ring + s * kSB, b_addr = a_addr + kABytes;
 #pragma unroll
                     for (uint32_t u = 0; u < kBK / kUmmaK; ++u) {
                         const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, kAtomBytes);
@@ -341,14 +358,14 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 for (int i = 0; i < kInstr; ++i) {
                     int64_t m = m0 + (gw * kInstr + i) * 4 + sub;
                     if (m >= M_keep) m = M_keep - 1;                  // padding rows of the last tile: never stored
-                    src[i] = p.dY + (int64_t)mapped_row(p.dy_rows, m) * C_out + chunk * 8;
+                    src[i] = p.dY + (int64_t)map_row<kPacked>(p.dy_rows, m) * C_out + chunk * 8;
                 }
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
-                    const int s = it % kStages;
-                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                    const int s = it % kS;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kS) & 1u) ^ 1u, abort_flag, status_word);
                     ok = __all_sync(0xffffffffu, ok);                 // the warp leaves the loop together
                     if (!ok) break;
-                    const uint32_t a_dst = ring + s * kStageBytes;
+                    const uint32_t a_dst = ring + s * kSB;
                     const int col = (int)(k * kBK + chunk * 8);
                     const uint32_t bytes = (col < C_out) ? 16u : 0u;  // columns past C_out read as zero
                     const int off = (col < C_out) ? (int)(k * kBK) : 0;
@@ -376,7 +393,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                         for (int h = 0; h < kIdxPerLane; ++h) {
                             const int64_t mrow = (int64_t)(t.kb_begin + k_first + u) * kBK + gw * kRows + h * 32 + (lane % kRows);
-                            nxt[u][h] = (k_first + u < t.num_kb && mrow < M_keep) ? mapped_row(p.dy_rows, mrow) : -1;
+                            nxt[u][h] = (k_first + u < t.num_kb && mrow < M_keep) ? map_row<kPacked>(p.dy_rows, mrow) : -1;
                         }
                 };
                 fetch_ids(0);
@@ -390,11 +407,11 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 #pragma unroll
                     for (int u = 0; u < kAhead; ++u) {
                         if (k0 + u >= t.num_kb) break;
-                        const int s = it % kStages;
-                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kStages) & 1u) ^ 1u, abort_flag, status_word);
+                        const int s = it % kS;
+                        ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kS) & 1u) ^ 1u, abort_flag, status_word);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
-                        const uint32_t a_dst = ring + s * kStageBytes;
+                        const uint32_t a_dst = ring + s * kSB;
 #pragma unroll
                         for (int i = 0; i < kInstr; ++i) {
                             const int rl = i * 2 + (int)sub;                                  // row within this warp's share
@@ -417,12 +434,12 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const uint32_t q = list_position(pass);
                 if (q >= sched.total) break;
                 const Tile t = decode_tile(sched, q);
-                if (!t.is_dw) zero_dropped_rows<BNX>(p, t, M_keep, warp - kBiasWarp0, lane);
+                if (!t.is_dw) zero_dropped_rows<BNX, kPacked>(p, t, M_keep, warp - kBiasWarp0, lane);
             }
         }
         // db partial of this CTA's share of the kept rows
         if (p.db_partial != nullptr) {
-            float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256);
+            float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kRingBytes + 256);
             const int t = threadIdx.x - kBiasWarp0 * 32;
             const int V = C_out >> 3;                                  // 16-byte column vectors per row
             int VT = 16;                                               // vectors covered per pass (power of two <= 128)
@@ -440,7 +457,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                 for (int64_t mc = m_begin; mc < m_end; mc += kBiasChunk) {
                     // stage the chunk's row ids once, so that the dY loads below depend on no other load
-                    if (t < kBiasChunk) ids[t] = (mc + t < m_end) ? mapped_row(p.dy_rows, mc + t) : -1;
+                    if (t < kBiasChunk) ids[t] = (mc + t < m_end) ? map_row<kPacked>(p.dy_rows, mc + t) : -1;
                     asm volatile("bar.sync 1, %0;" ::"n"(kBiasThreads) : "memory");
                     if (cv < V) {
                         for (int r0 = rg; r0 < kBiasChunk; r0 += RG * kBiasDepth) {
@@ -504,7 +521,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const int64_t m0 = (int64_t)t.row_tile * kBM;
                 const int64_t m = m0 + warp * 32 + lane;
                 const bool valid = m < M_keep;
-                const int64_t cur = valid ? (int64_t)mapped_row(p.dx_rows, m) : -1;
+                const int64_t cur = valid ? (int64_t)map_row<kPacked>(kPacked ? p.dx_rows : p.dy_rows, m) : -1;
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
                 if (threadIdx.x == 0) ptx::bulk_wait_read<0>();       // the staging memory is no longer read by TMA stores of a dW tile
                 ok = !ptx::bar_or<kEpiBarrier, 128>(!ok);            // the four epilogue warps go on, or give up, together
@@ -514,7 +531,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 // different rows costs 32 memory transactions.  So the warp transposes 64 columns at a
                 // time through its own 4 KB of (swizzled) shared memory and writes four rows x 128
                 // contiguous bytes per instruction.
-                uint8_t* wbuf = smem_raw + (ring - raw_addr) + kStages * kStageBytes + 256 + kBiasSmemBytes + warp * 4096;
+                uint8_t* wbuf = smem_raw + (ring - raw_addr) + kRingBytes + 256 + kBiasSmemBytes + warp * 4096;
                 const int cur32 = valid ? (int)cur : -1;
                 const int sub = lane >> 3, ch = lane & 7;
                 float va[32], vb[32];
@@ -567,7 +584,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     const int j0 = (int)(t.row_tile * kBM);
                     const int live = (C_in - i0 < BNW) ? C_in - i0 : BNW;
                     const int chunks = (live + kEpiChunk - 1) / kEpiChunk;
-                    const uint32_t stage_off = (ring - raw_addr) + kStages * kStageBytes + 256 + kBiasSmemBytes;
+                    const uint32_t stage_off = (ring - raw_addr) + kRingBytes + 256 + kBiasSmemBytes;
 #pragma unroll 1
                     for (int c = 0; c < chunks; ++c, ++staged) {
                         float v[kEpiChunk];
@@ -738,14 +755,22 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     return pl;
 }
 
+template <int BNX, int BNW, int DEPTH, bool PACKED>
+cudaError_t launch_fused_variant(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
+                                 const CUtensorMap& map_dw, const TcParams& prm) {
+    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW, DEPTH, PACKED>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (once != cudaSuccess) return once;
+    return launch_pdl(tc_backward_kernel<BNX, BNW, DEPTH, PACKED>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x,
+                      map_dw, prm);
+}
+
 template <int BNX, int BNW, int DEPTH>
 cudaError_t launch_fused_depth(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
                                const CUtensorMap& map_dw, const TcParams& prm) {
-    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW, DEPTH>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (once != cudaSuccess) return once;
-    return launch_pdl(tc_backward_kernel<BNX, BNW, DEPTH>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x,
-                      map_dw, prm);
+    const bool packed = prm.dy_rows == nullptr || prm.dx_rows == nullptr;
+    return packed ? launch_fused_variant<BNX, BNW, DEPTH, true>(grid, stream, map_w, map_x, map_dw, prm)
+                  : launch_fused_variant<BNX, BNW, DEPTH, false>(grid, stream, map_w, map_x, map_dw, prm);
 }
 
 template <int BNX, int BNW>
