@@ -263,6 +263,16 @@ sbp_status sbp_bias_grad_static(sbp_dtype dt, const void* dY /* dev */, const in
                                 const int32_t* M_keep_dev /* dev, nullable */, int64_t M, int64_t M_keep_cap,
                                 int64_t C_out, float* db /* dev */, uint32_t flags, void* stream);
 
+/*
+ * Diagnostic (no counterpart in the paper): runs the library's bounded device-side wait
+ * on a barrier that is never completed, with a limit of limit_ms (0 < limit_ms <= 2000).
+ * On return of the kernel *completed (dev) is 0 and *status_word (dev, zero before the
+ * call) holds SBP_ERR_TIMEOUT; the stream and the context remain usable.  This is the
+ * mechanism every pipeline kernel uses instead of an unbounded spin.
+ */
+sbp_status sbp_selftest_bounded_wait(double limit_ms, int32_t* status_word /* dev */,
+                                     int32_t* completed /* dev */, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,7 @@ SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT = 16, 32
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
-           "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static")
+           "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static", "sbp_selftest_bounded_wait")
 
 _lib = None
 
@@ -56,6 +56,8 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_sample_keep.restype = ci
     lib.sbp_forward_cache.argtypes = [ci, vp, i64, i64, vp, vp, i64, vp, vp]
     lib.sbp_forward_cache.restype = ci
+    lib.sbp_selftest_bounded_wait.argtypes = [dbl, vp, vp, vp]
+    lib.sbp_selftest_bounded_wait.restype = ci
     lib.sbp_linear_forward.argtypes = [ci, vp, vp, vp, i64, i64, i64, vp, vp, vp, i64, vp, u32, vp, vp]
     lib.sbp_linear_forward.restype = ci
     lib.sbp_linear_backward_workspace_bytes.argtypes = [ci, i64, i64, i64, i64]
@@ -179,4 +181,12 @@ def sbp_bias_grad_static(dt, dY, keep_rows, M_keep_dev, M, M_keep_cap, C_out, db
                                             _ptr(db), flags, _stream(stream))
     if check:
         _check(s, "sbp_bias_grad_static")
+    return s
+
+
+def sbp_selftest_bounded_wait(limit_ms, status_word, completed, stream=None, check=True) -> int:
+    """Runs a device-side wait that cannot complete; it must give up after limit_ms and report SBP_ERR_TIMEOUT."""
+    s = load_library().sbp_selftest_bounded_wait(float(limit_ms), _ptr(status_word), _ptr(completed), _stream(stream))
+    if check:
+        _check(s, "sbp_selftest_bounded_wait")
     return s

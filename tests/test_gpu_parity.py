@@ -260,3 +260,23 @@ def test_full_path_sampler_to_gradients_on_device():
     assert relerr(host(got["dW"]), want["dW"]) <= 5e-3
     assert relerr(host(got["db"]), want["db"]) <= 5e-3
     assert relerr(synth.to_f64(host(got["dX"]), "bf16"), want["dX"]) <= 5e-3
+
+
+def test_bounded_wait_gives_up_reports_and_leaves_the_stream_usable():
+    # a device-side wait that nothing will ever satisfy: it must expire after its limit, set the status word,
+    # let the kernel return, and the next call on the same stream must work as usual
+    import time
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    completed = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    sbp.sbp_selftest_bounded_wait(200.0, status, completed)
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert int(status.item()) == sbp.SBP_ERR_TIMEOUT and int(completed.item()) == 0
+    assert 0.19 <= waited < 1.5
+    rows, offs, _ = run_sample_keep(0, 2, 14, 14, 0.5)
+    want_rows, want_offs = oracle.sample_keep(0, 2, 14, 14, 0.5)
+    assert np.array_equal(host(offs), want_offs) and np.array_equal(host(rows)[:len(want_rows)], want_rows)
+    assert sbp.sbp_selftest_bounded_wait(0.0, status, completed, check=False) == sbp.SBP_ERR_INVALID_ARG
+    assert sbp.sbp_selftest_bounded_wait(5000.0, status, completed, check=False) == sbp.SBP_ERR_INVALID_ARG
