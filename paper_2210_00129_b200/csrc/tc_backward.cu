@@ -380,7 +380,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 constexpr int kRows = 64 / kGatherWarps;             // rows of a stage this warp copies
                 constexpr int kIdxPerLane = (kRows + 31) / 32;       // row ids each lane holds per stage
                 constexpr int kInstr = kRows / 2;
-                constexpr int kAhead = 4;                            // row ids are fetched this many stages early
+                constexpr int kAhead = 8;                            // row ids are fetched this many stages early
                 const uint32_t c = lane & 15;                        // 16-byte chunk within the 256-byte row piece
                 const uint32_t sub = lane >> 4;                      // which of the two rows of this instruction
                 const int col = (int)(t.row_tile * kBM) + (int)c * 8;
