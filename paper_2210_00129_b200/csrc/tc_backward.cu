@@ -2,12 +2,13 @@
 //
 //   dX tiles:  D[m, i] = sum_j dY[keep_rows[m], j] * W[i, j]            (both operands K-major)
 //              A = kept rows of dY, gathered straight from the full dY; B = W tile (TMA);
-//              the epilogue rounds to bf16, scatters each row to dX[keep_rows[m], :] and
-//              zero-fills the dropped rows between kept rows.
+//              the epilogue rounds to bf16 and writes each row to dX[keep_rows[m], :] (whole 128-byte
+//              pieces of four rows per store, through a shared-memory transpose).
 //   dW tiles:  D[j, i] = sum_m dY[keep_rows[m], j] * X_keep[m, i]       (both operands MN-major)
 //              computed transposed so that the gathered operand is again the 128-row side:
-//              A = gathered dY rows, B = X_keep tile (TMA); the epilogue writes dW[i, j];
-//              long reductions are cut into pieces whose partials a second kernel adds in order.
+//              A = gathered dY rows, B = X_keep tile (TMA); the epilogue stages 16 x 128 pieces of
+//              dW[i, j] and sends them out as TMA stores; long reductions can be cut into pieces
+//              whose partials a second kernel adds in order.
 //
 // ONE persistent kernel runs both products: every CTA (one per SM) walks a static, cost-sorted
 // list of 128 x BN output tiles of either kind.  The operand ring (64-deep, 128-byte-swizzled
@@ -19,9 +20,12 @@
 // copies signal the stage's barrier when they land (cp.async.mbarrier.arrive).  TMA tile::gather4
 // was measured at ~45 ns of issue time per instruction per SM whatever it fetches - far too slow
 // to feed a tile - and is not used.  Every wait is bounded and reports through the status word.
-// Four more warps compute the bias gradient on the side: each CTA sums its share of the kept rows
-// of dY column-wise while the tensor pipe works (the kernel is latency-bound, not bandwidth-bound,
-// so the extra reads are free) and leaves one partial row per CTA for a fixed-order reduce.
+// Four side warps work next to the pipeline: they write the zeros of the dropped rows of dX for the
+// block's dX tiles (ahead of the MMAs, so every row of dX is written exactly once and no memset pass
+// is needed), then sum the block's share of the kept rows of dY column-wise for the bias gradient
+// and leave one partial row per block for a fixed-order reduce.  The row maps are compile-time
+// variants: keep_rows on both sides, or identity on either side for gradients kept packed between
+// chained layers (Sec. 3.3.1).
 #include <mutex>
 
 #include "tc_ptx.cuh"
