@@ -420,6 +420,9 @@ def run_cuda(args, w, name):
                         "peak": peak, "peak_kind": "derived: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz", "unit": "TFLOP/s",
                         "traffic": None}
         roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        if tc_path:     # for context: the same figure against the nominal dense bf16 rate of the part
+            roofline["peak_nominal"] = 2250.0
+            roofline["frac_nominal"] = roofline["achieved"] / 2250.0
         roofline["launch_ms"] = gemm_ms
 
         B_s = pick_oracle_sample(w)
