@@ -5,7 +5,7 @@
 For every layer of the chosen groups (ViT-B/16 MLP and attention projections at four keep ratios,
 ConvNeXt-B point-wise layers of the four stages with random and grid masks, the detection-resolution
 map; Sec. 5 of the paper gives the models) it times `sbp_sample_keep`, `sbp_forward_cache` and
-`sbp_linear_backward` (dW alone, dX alone, db alone, all three) on one GPU and prints a markdown table:
+`sbp_linear_backward` (dW alone, dX alone, db alone, both products, all three) on one GPU and prints a markdown table:
 microseconds, the lower bound `t_min = max(FLOP / peak, bytes / bandwidth)` of the call's algorithmic
 work, `t_min / t`, and the speed-up of the whole backward over keep ratio 1.0.
 
@@ -135,6 +135,7 @@ def measure_layer(bench, spec, pk):
         "db": bench.time_us(lambda k, i: bw(k, 0, 1, 0), n_sets),
         "dW": bench.time_us(lambda k, i: bw(k, 1, 0, 0), n_sets),
         "dX": bench.time_us(lambda k, i: bw(k, 0, 0, 1), n_sets),
+        "dW+dX": bench.time_us(lambda k, i: bw(k, 1, 0, 1), n_sets),
         "bwd": bench.time_us(lambda k, i: bw(k, 1, 1, 1), n_sets),
     }
     assert int(st.item()) == 0, f"status word {int(st.item())} on {name}"
@@ -148,7 +149,8 @@ def measure_layer(bench, spec, pk):
         "dX": M_keep * C_out * es + C_in * C_out * es + M * C_in * es,
     }
     by["bwd"] = M_keep * (C_in + C_out) * es + C_in * C_out * es + 4.0 * C_in * C_out + M * C_in * es + 4 * C_out
-    fl = {"sample": 0.0, "cache": 0.0, "db": 0.0, "dW": flop, "dX": flop, "bwd": 2 * flop}
+    by["dW+dX"] = by["bwd"] - 4 * C_out
+    fl = {"sample": 0.0, "cache": 0.0, "db": 0.0, "dW": flop, "dX": flop, "dW+dX": 2 * flop, "bwd": 2 * flop}
     tmin = {k: max(fl[k] / tf, by[k] / bw_) * 1e6 for k in t}
     bound = {k: ("tensor" if fl[k] / tf > by[k] / bw_ else "hbm") for k in t}
     del sets
@@ -271,8 +273,8 @@ def main():
     if args.group not in ("sampler", "blocks", "forward"):
         if args.compact:
             print("us (t_min / t) per call; bound of the whole backward in the last column\n")
-            print("| layer | M_keep | sample | cache | db | dW | dX | backward (dW+db+dX) | TFLOP/s | bound |")
-            print("|---|---|---|---|---|---|---|---|---|---|")
+            print("| layer | M_keep | sample | cache | db | dW | dX | dW+dX (one launch) | backward (dW+db+dX) | TFLOP/s | bound |")
+            print("|---|---|---|---|---|---|---|---|---|---|---|")
         else:
             print("| layer | M_keep | call | us | t_min us | t_min/t | bound | achieved |")
             print("|---|---|---|---|---|---|---|---|")
@@ -282,13 +284,13 @@ def main():
             m = measure_layer(bench, spec, pk)
             res.append((spec, m))
             if args.compact:
-                cells = " | ".join(f"{m['t'][k]:.1f} ({m['tmin'][k] / m['t'][k]:.2f})" for k in ("cache", "db", "dW", "dX", "bwd"))
+                cells = " | ".join(f"{m['t'][k]:.1f} ({m['tmin'][k] / m['t'][k]:.2f})" for k in ("cache", "db", "dW", "dX", "dW+dX", "bwd"))
                 print(f"| {m['name']} | {m['M_keep']} | {m['t']['sample']:.1f} | {cells} | "
                       f"{2 * m['flop'] / m['t']['bwd'] / 1e6:.0f} | {m['bound']['bwd']} |")
-            for k in (() if args.compact else ("sample", "cache", "db", "dW", "dX", "bwd")):
+            for k in (() if args.compact else ("sample", "cache", "db", "dW", "dX", "dW+dX", "bwd")):
                 us = m["t"][k]
-                if k in ("dW", "dX", "bwd"):
-                    ach = f"{(2 if k == 'bwd' else 1) * m['flop'] / us / 1e6:.0f} TFLOP/s"
+                if k in ("dW", "dX", "dW+dX", "bwd"):
+                    ach = f"{(2 if k in ('bwd', 'dW+dX') else 1) * m['flop'] / us / 1e6:.0f} TFLOP/s"
                 else:
                     ach = f"{m['bytes'][k] / us / 1e3:.0f} GB/s"
                 print(f"| {m['name']} | {m['M_keep']} | {k} | {us:.1f} | {m['tmin'][k]:.1f} | {m['tmin'][k] / us:.2f} | "
