@@ -22,6 +22,7 @@ _LIB_PATH = os.path.join(_HERE, "libsbp_oracle.so")
 MASK_RANDOM = 0
 MASK_GRID = 1
 MASK_TEMPORAL = 2
+MASK_TEMPORAL_GRID = 3
 FLAG_SHARE_MASK = 1
 
 _lib = None

@@ -35,6 +35,7 @@
 #define ORACLE_MASK_RANDOM 0
 #define ORACLE_MASK_GRID   1
 #define ORACLE_MASK_TEMPORAL 2   /* whole frames of a video: H = frames, W = positions per frame */
+#define ORACLE_MASK_TEMPORAL_GRID 3   /* frames on a lattice in time (the "even index on T" example) */
 #define ORACLE_FLAG_SHARE_MASK 1u
 
 /* ------------------------------------------------------------------ */
@@ -112,6 +113,20 @@ static int grid_keeps(int fam, uint32_t p, int64_t h, int64_t w)
     return 0;
 }
 
+/* is frame f kept by the lattice in time of family fam at phase p ?
+ * r = 0.25: every fourth frame; r = 0.5: every second frame (phase 0 is the paper's
+ * "even index on T", Sec. 3.2.1); r = 0.75: all but every fourth; r = 1: all. */
+static int frame_keeps(int fam, uint32_t p, int64_t f)
+{
+    switch (fam) {
+    case 1: return (f & 3) == (int64_t)p;
+    case 2: return (f & 1) == (int64_t)p;
+    case 3: return (f & 3) != (int64_t)p;
+    case 4: return 1;
+    }
+    return 0;
+}
+
 /* Random mode: the exact per-sample count K = clamp(floor(r*N + 1/2), 1, N).
  * Grid mode: the largest count any phase can give (capacity per sample).
  * Returns -1 for arguments outside the method's domain. */
@@ -130,6 +145,18 @@ int64_t oracle_keep_count(int mode, int64_t H, int64_t W, double r)
         if (KT < 1) KT = 1;
         if (KT > H) KT = H;
         return KT * W;
+    }
+    if (mode == ORACLE_MASK_TEMPORAL_GRID) {  /* capacity: the phase that keeps the most frames, times W */
+        int fam = grid_family(r);
+        if (!fam) return -1;
+        int phases = (fam == 2) ? 2 : (fam == 4 ? 1 : 4);
+        int64_t best = 0;
+        for (int p = 0; p < phases; ++p) {
+            int64_t cnt = 0;
+            for (int64_t f = 0; f < H; ++f) cnt += frame_keeps(fam, (uint32_t)p, f);
+            if (cnt > best) best = cnt;
+        }
+        return best * W;
     }
     if (mode == ORACLE_MASK_GRID) {
         int fam = grid_family(r);
@@ -166,7 +193,9 @@ static int cmp_u64(const void* a, const void* b)
  * Temporal mode (Sec. 3.1 and 3.2.1: a subset of video frames): H frames of W
  * positions; frame f gets the score (word << 32) | f from the same word stream as
  * position f of a random-mode map, the K_T frames with the smallest scores are
- * kept, each with all of its positions. */
+ * kept, each with all of its positions.
+ * Temporal grid mode: frames on a lattice in time (every second or fourth frame, or
+ * the complement), the phase drawn per sample like the spatial grid phase. */
 int64_t oracle_sample_keep(int mode, int64_t B, int64_t H, int64_t W, double r,
                            uint64_t seed, uint64_t step, int64_t sample_offset,
                            uint32_t flags, int32_t* keep_rows, int32_t* keep_offsets)
@@ -217,6 +246,18 @@ int64_t oracle_sample_keep(int mode, int64_t B, int64_t H, int64_t W, double r,
             keep_offsets[b + 1] = (int32_t)out;
         }
         free(score); free(kept);
+    } else if (mode == ORACLE_MASK_TEMPORAL_GRID) {
+        /* frames on a lattice in time, the phase drawn per sample from the same word as the spatial grid phase */
+        int fam = grid_family(r);
+        uint32_t phases = (fam == 2) ? 2u : (fam == 4 ? 1u : 4u);
+        for (int64_t b = 0; b < B; ++b) {
+            uint32_t gid = (flags & ORACLE_FLAG_SHARE_MASK) ? 0u : (uint32_t)(sample_offset + b);
+            uint32_t p = grid_phase_word(seed, (uint32_t)step, gid) % phases;
+            for (int64_t f = 0; f < H; ++f)
+                if (frame_keeps(fam, p, f))
+                    for (int64_t q = 0; q < W; ++q) keep_rows[out++] = (int32_t)(b * N + f * W + q);
+            keep_offsets[b + 1] = (int32_t)out;
+        }
     } else {
         int fam = grid_family(r);
         uint32_t phases = (fam == 2) ? 2u : (fam == 4 ? 1u : 4u);

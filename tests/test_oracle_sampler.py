@@ -332,3 +332,51 @@ def test_temporal_mask_sharding_and_ratio_one():
     assert np.array_equal(whole, np.concatenate([a, b + 2 * 8 * 4]))
     full, offs = oracle.sample_keep(oracle.MASK_TEMPORAL, 2, 8, 4, 1.0)
     assert np.array_equal(full, np.arange(2 * 8 * 4)) and list(offs) == [0, 32, 64]
+
+
+# ---------------------------------------------------------------- frames on a lattice in time
+def _frames_of(rows, B, T, P):
+    """Per sample, the sorted list of kept frames; asserts that frames are kept whole."""
+    per_frame = np.bincount(np.asarray(rows) // P, minlength=B * T).reshape(B, T)
+    assert set(per_frame.flatten().tolist()) <= {0, P}
+    return [np.flatnonzero(per_frame[b]).tolist() for b in range(B)]
+
+
+def test_temporal_grid_half_is_even_or_odd_frames_and_contains_the_paper_example():
+    # Sec. 3.2.1: X_keep can be X[:, even index on T, ...].  At r = 0.5 every sample keeps the even or the odd
+    # frames; over many samples both phases occur, and together they cover every frame
+    B, T, P = 64, 9, 5
+    rows, offs = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, B, T, P, 0.5, 4, 2)
+    frames = _frames_of(rows, B, T, P)
+    even, odd = list(range(0, T, 2)), list(range(1, T, 2))
+    assert all(f in (even, odd) for f in frames) and even in frames and odd in frames
+    assert [int(offs[b + 1] - offs[b]) for b in range(B)] == [len(f) * P for f in frames]       # ragged: 5 or 4 frames
+    assert oracle.keep_count(oracle.MASK_TEMPORAL_GRID, T, P, 0.5) == 5 * P
+
+
+def test_temporal_grid_quarter_three_quarter_and_all():
+    B, T, P = 48, 10, 3
+    q, _ = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, B, T, P, 0.25, 9, 1)
+    tq, _ = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, B, T, P, 0.75, 9, 1)
+    fq, ftq = _frames_of(q, B, T, P), _frames_of(tq, B, T, P)
+    for b in range(B):
+        assert len({f % 4 for f in fq[b]}) == 1                                  # one residue class mod 4
+        assert sorted(fq[b] + ftq[b]) == list(range(T))                          # same phase word: exact complements
+    assert {fq[b][0] % 4 for b in range(B)} == {0, 1, 2, 3}                      # all four phases occur
+    full, offs = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, 2, T, P, 1.0)
+    assert np.array_equal(full, np.arange(2 * T * P))
+    with pytest.raises(ValueError):
+        oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, 2, T, P, 0.3)
+
+
+def test_temporal_grid_phase_matches_the_spatial_grid_phase_word_and_sharding():
+    # the phase comes from the same Philox word as the spatial grid masks: on a T x 1 map the r = 0.5
+    # checkerboard keeps (f + 0) mod 2 == p, i.e. the same frames
+    B, T, P = 16, 8, 4
+    rows, _ = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, B, T, P, 0.5, 11, 3, 5)
+    grid, _ = oracle.sample_keep(oracle.MASK_GRID, B, T, 1, 0.5, 11, 3, 5)          # ids b*T + f
+    expanded = (grid[:, None].astype(np.int64) * P + np.arange(P)[None, :]).reshape(-1)
+    assert np.array_equal(rows, expanded)
+    a, _ = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, 6, T, P, 0.5, 11, 3, 5)
+    b, _ = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, 10, T, P, 0.5, 11, 3, 11)
+    assert np.array_equal(rows, np.concatenate([a, b + 6 * T * P]))
