@@ -52,7 +52,7 @@ typedef enum { SBP_F32 = 0, SBP_BF16 = 1 } sbp_dtype;
 
 /* Sec. 4, "How to sample the gradient keep mask?": uniformly random positions,
  * or a structured periodic ("grid-wise") mask. */
-typedef enum { SBP_MASK_RANDOM = 0, SBP_MASK_GRID = 1, SBP_MASK_TEMPORAL = 2 } sbp_mask_mode;
+typedef enum { SBP_MASK_RANDOM = 0, SBP_MASK_GRID = 1, SBP_MASK_TEMPORAL = 2, SBP_MASK_TEMPORAL_GRID = 3 } sbp_mask_mode;
 
 enum {
     SBP_FLAG_SHARE_MASK = 1,  /* every sample of the call uses sample 0's mask (one mask per iteration, Supp. A.4) */
@@ -73,6 +73,8 @@ const char* sbp_status_string(sbp_status s);
  *                    per sample); r must be one of 0.25, 0.5, 0.75, 1.0.
  *   SBP_MASK_TEMPORAL: H is the number of frames, W the positions per frame;
  *                    clamp(floor(r*H + 1/2), 1, H) whole frames, times W.
+ *   SBP_MASK_TEMPORAL_GRID: as SBP_MASK_GRID in time: the largest frame count any phase
+ *                    gives, times W; r must be one of 0.25, 0.5, 0.75, 1.0.
  * Returns -1 when H, W <= 0, r outside (0, 1], or the ratio has no grid mask.
  */
 int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_ratio);
@@ -96,6 +98,12 @@ int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_rat
  *   the word of position f above, the K_T frames with the smallest scores are kept,
  *   each with all W positions (rows (b*H + f)*W + q).  At most 2048 frames
  *   (SBP_ERR_UNSUPPORTED beyond).
+ * SBP_MASK_TEMPORAL_GRID (the "even index on T" example of Sec. 3.2.1): frames on a
+ *   lattice in time with a random phase p per sample, p drawn as for SBP_MASK_GRID:
+ *     r = 0.25  keep f mod 4 == p;  r = 0.5  keep f mod 2 == p (p = 0: the even frames);
+ *     r = 0.75  keep f mod 4 != p;  r = 1.0  keep every frame.
+ *   Counts depend on the phase when H is not a multiple of the period: read M_keep from
+ *   keep_offsets[B].
  * The mask depends only on (seed, step, g, n): it does not change with how a
  * batch is split over calls or devices.
  *

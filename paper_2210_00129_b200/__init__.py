@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libsbp_b200.so")
 SBP_OK, SBP_ERR_INVALID_ARG, SBP_ERR_UNSUPPORTED, SBP_ERR_WORKSPACE = 0, 1, 2, 3
 SBP_ERR_CUDA, SBP_ERR_TIMEOUT, SBP_ERR_BAD_INDICES = 4, 5, 6
 SBP_F32, SBP_BF16 = 0, 1
-SBP_MASK_RANDOM, SBP_MASK_GRID, SBP_MASK_TEMPORAL = 0, 1, 2
+SBP_MASK_RANDOM, SBP_MASK_GRID, SBP_MASK_TEMPORAL, SBP_MASK_TEMPORAL_GRID = 0, 1, 2, 3
 SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
 SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT = 16, 32
 

@@ -365,8 +365,30 @@ sample_keep_grid_kernel(int family, uint32_t H, uint32_t W, uint32_t k0, uint32_
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t kMaxFrames = 2048;
 
+// frames of family `family` (as the spatial grid families: every fourth, every second, all but every fourth, all)
+// at phase p among T frames
+__device__ __forceinline__ uint32_t frame_count(int family, uint32_t p, uint32_t T) {
+    const uint32_t fourth = (T + 3u - p) >> 2;
+    switch (family) {
+        case 1: return fourth;
+        case 2: return (T + 1u - p) >> 1;
+        case 3: return T - fourth;
+        default: return T;
+    }
+}
+__device__ __forceinline__ bool frame_keeps(int family, uint32_t p, uint32_t f) {
+    switch (family) {
+        case 1: return (f & 3u) == p;
+        case 2: return (f & 1u) == p;
+        case 3: return (f & 3u) != p;
+        default: return true;
+    }
+}
+
+// family 0: the K_T frames with the smallest scores; families 1-4: frames on a lattice in time whose phase is
+// drawn per sample like the spatial grid phase (counts, and so the offsets, then depend on the phases)
 __global__ void __launch_bounds__(kSampThreads)
-sample_keep_temporal_kernel(uint32_t T, uint32_t P, uint32_t KT, uint32_t k0, uint32_t k1, uint32_t step,
+sample_keep_temporal_kernel(int family, uint32_t T, uint32_t P, uint32_t KT, uint32_t k0, uint32_t k1, uint32_t step,
                             uint32_t first_sample, int share_mask,
                             int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
     __shared__ unsigned long long score[kMaxFrames];
@@ -376,16 +398,38 @@ sample_keep_temporal_kernel(uint32_t T, uint32_t P, uint32_t KT, uint32_t k0, ui
     pdl_wait();
     const uint32_t b = blockIdx.x;
     const uint32_t gid = share_mask ? 0u : first_sample + b;
-    for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
-        const uint32_t w = philox4x32_10(f >> 2, gid, step, 0u, k0, k1).w[f & 3u];
-        score[f] = ((unsigned long long)w << 32) | f;
-    }
-    __syncthreads();
-    for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
-        const unsigned long long mine = score[f];
-        uint32_t rank = 0;
-        for (uint32_t g = 0; g < T; ++g) rank += score[g] < mine;
-        kept[f] = rank < KT ? 1u : 0u;
+    uint64_t frames_before = (uint64_t)b * KT;                       // kept frames of the samples before this one
+    if (family == 0) {
+        for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
+            const uint32_t w = philox4x32_10(f >> 2, gid, step, 0u, k0, k1).w[f & 3u];
+            score[f] = ((unsigned long long)w << 32) | f;
+        }
+        __syncthreads();
+        for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
+            const unsigned long long mine = score[f];
+            uint32_t rank = 0;
+            for (uint32_t g = 0; g < T; ++g) rank += score[g] < mine;
+            kept[f] = rank < KT ? 1u : 0u;
+        }
+    } else {
+        const uint32_t p = grid_phase(family, gid, step, k0, k1);
+        for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) kept[f] = frame_keeps(family, p, f) ? 1u : 0u;
+        KT = frame_count(family, p, T);
+        // the offset of this sample is the sum of the closed-form counts of the samples before it
+        if (share_mask) {
+            frames_before = (uint64_t)b * KT;
+        } else {
+            __shared__ unsigned long long red[kSampThreads / 32];
+            unsigned long long part = 0;
+            for (uint32_t s2 = threadIdx.x; s2 < b; s2 += kSampThreads)
+                part += frame_count(family, grid_phase(family, first_sample + s2, step, k0, k1), T);
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+            if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = part;
+            __syncthreads();
+            frames_before = 0;
+            for (int i = 0; i < kSampThreads / 32; ++i) frames_before += red[i];
+        }
     }
     __syncthreads();
     for (uint32_t f = threadIdx.x; f < T; f += kSampThreads) {
@@ -397,14 +441,14 @@ sample_keep_temporal_kernel(uint32_t T, uint32_t P, uint32_t KT, uint32_t k0, ui
     }
     __syncthreads();
     const uint64_t per_sample = (uint64_t)KT * P;
-    int32_t* out = keep_rows + (uint64_t)b * per_sample;
+    int32_t* out = keep_rows + frames_before * P;
     for (uint64_t e = threadIdx.x; e < per_sample; e += kSampThreads) {
         const uint32_t k = (uint32_t)(e / P), q = (uint32_t)(e - (uint64_t)k * P);
         out[e] = (int32_t)(((uint64_t)b * T + list[k]) * P + q);
     }
     if (threadIdx.x == 0) {
-        keep_offsets[b] = (int32_t)((uint64_t)b * per_sample);
-        if (b + 1 == gridDim.x) keep_offsets[b + 1] = (int32_t)((uint64_t)(b + 1) * per_sample);
+        keep_offsets[b] = (int32_t)(frames_before * P);
+        if (b + 1 == gridDim.x) keep_offsets[b + 1] = (int32_t)(frames_before * P + per_sample);
     }
 }
 
@@ -438,8 +482,9 @@ cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, 
         return launch_pdl(sample_keep_random_kernel, grid, block, 0, stream, (uint32_t)(H * W), (uint32_t)K, k0, k1,
                           step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
     }
-    if (mode == SBP_MASK_TEMPORAL)      // H frames of W positions; K = kept frames x W
-        return launch_pdl(sample_keep_temporal_kernel, grid, block, 0, stream, (uint32_t)H, (uint32_t)W, (uint32_t)(K / W),
+    if (mode == SBP_MASK_TEMPORAL || mode == SBP_MASK_TEMPORAL_GRID)      // H frames of W positions; K = kept frames x W
+        return launch_pdl(sample_keep_temporal_kernel, grid, block, 0, stream, mode == SBP_MASK_TEMPORAL ? 0 : grid_family,
+                          (uint32_t)H, (uint32_t)W, (uint32_t)(K / W),
                           k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
     return launch_pdl(sample_keep_grid_kernel, grid, block, 0, stream, grid_family, (uint32_t)H, (uint32_t)W, k0, k1,
                       step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);

@@ -65,6 +65,15 @@ int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_rat
         if (KT > H) KT = H;
         return KT * W;
     }
+    if (mode == SBP_MASK_TEMPORAL_GRID) {     // capacity: the phase (0) that keeps the most frames, times W
+        switch (grid_family_of(keep_ratio)) {
+            case 1: return ((H + 3) / 4) * W;
+            case 2: return ((H + 1) / 2) * W;
+            case 3: return (H - H / 4) * W;          // all but the phase-3 class, the smallest one
+            case 4: return H * W;
+            default: return -1;
+        }
+    }
     if (mode == SBP_MASK_GRID) {
         const int64_t quarter_max = ((H + 1) / 2) * ((W + 1) / 2);   // phase (0, 0) holds the most lattice points
         const int64_t quarter_min = (H / 2) * (W / 2);               // phase (1, 1) the fewest
@@ -82,7 +91,8 @@ int64_t sbp_keep_count(sbp_mask_mode mode, int64_t H, int64_t W, double keep_rat
 sbp_status sbp_sample_keep(sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, double keep_ratio,
                            uint64_t seed, uint64_t step, int64_t sample_offset, uint32_t flags,
                            int32_t* keep_rows, int32_t* keep_offsets, void* stream) {
-    if (mode != SBP_MASK_RANDOM && mode != SBP_MASK_GRID && mode != SBP_MASK_TEMPORAL) return SBP_ERR_INVALID_ARG;
+    if (mode != SBP_MASK_RANDOM && mode != SBP_MASK_GRID && mode != SBP_MASK_TEMPORAL && mode != SBP_MASK_TEMPORAL_GRID)
+        return SBP_ERR_INVALID_ARG;
     if (keep_rows == nullptr || keep_offsets == nullptr) return SBP_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(keep_rows) & 3u) || (reinterpret_cast<uintptr_t>(keep_offsets) & 3u))
         return SBP_ERR_INVALID_ARG;
@@ -93,8 +103,9 @@ sbp_status sbp_sample_keep(sbp_mask_mode mode, int64_t B, int64_t H, int64_t W, 
     if (step >> 32) return SBP_ERR_INVALID_ARG;
     if (sample_offset < 0 || ((uint64_t)(sample_offset + B - 1) >> 32)) return SBP_ERR_INVALID_ARG;
     const int family = grid_family_of(keep_ratio);
-    if (mode == SBP_MASK_GRID && family == 0) return SBP_ERR_UNSUPPORTED;
-    if (mode == SBP_MASK_TEMPORAL && H > (int64_t)sample_keep_max_frames()) return SBP_ERR_UNSUPPORTED;
+    if ((mode == SBP_MASK_GRID || mode == SBP_MASK_TEMPORAL_GRID) && family == 0) return SBP_ERR_UNSUPPORTED;
+    if ((mode == SBP_MASK_TEMPORAL || mode == SBP_MASK_TEMPORAL_GRID) && H > (int64_t)sample_keep_max_frames())
+        return SBP_ERR_UNSUPPORTED;
     const int64_t K = sbp_keep_count(mode, H, W, keep_ratio);
     const cudaError_t e = launch_sample_keep((int)mode, family, B, H, W, K, seed, (uint32_t)step,
                                              (uint32_t)sample_offset, (flags & SBP_FLAG_SHARE_MASK) != 0,

@@ -40,9 +40,9 @@ def test_status_strings(lib):
     assert sbp.status_string(99) == "unknown status"
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
 def test_keep_count_matches_the_rule(lib, mode):
-    ratios = (0.25, 0.5, 0.75, 1.0) if mode == 1 else (0.01, 0.25, 0.3, 0.5, 0.75, 0.999, 1.0)
+    ratios = (0.25, 0.5, 0.75, 1.0) if mode in (1, 3) else (0.01, 0.25, 0.3, 0.5, 0.75, 0.999, 1.0)
     for H, W in [(1, 1), (14, 14), (7, 7), (3, 5), (56, 56), (200, 334), (16, 1)]:
         for r in ratios:
             assert sbp.sbp_keep_count(mode, H, W, r) == oracle.keep_count(mode, H, W, r)
@@ -63,7 +63,8 @@ def test_host_detected_errors_return_before_any_launch(lib):
     assert sbp.sbp_sample_keep(0, 2 ** 20, 2 ** 6, 2 ** 6, 0.5, 0, 0, 0, 0, fake, fake, stream=0, check=False) == sbp.SBP_ERR_INVALID_ARG
     assert sbp.sbp_sample_keep(1, 2, 4, 4, 0.6, 0, 0, 0, 0, fake, fake, stream=0, check=False) == sbp.SBP_ERR_UNSUPPORTED
     assert sbp.sbp_sample_keep(2, 2, 4096, 4, 0.5, 0, 0, 0, 0, fake, fake, stream=0, check=False) == sbp.SBP_ERR_UNSUPPORTED   # too many frames
-    assert sbp.sbp_sample_keep(3, 2, 4, 4, 0.5, 0, 0, 0, 0, fake, fake, stream=0, check=False) == sbp.SBP_ERR_INVALID_ARG
+    assert sbp.sbp_sample_keep(4, 2, 4, 4, 0.5, 0, 0, 0, 0, fake, fake, stream=0, check=False) == sbp.SBP_ERR_INVALID_ARG
+    assert sbp.sbp_sample_keep(3, 2, 4, 4, 0.6, 0, 0, 0, 0, fake, fake, stream=0, check=False) == sbp.SBP_ERR_UNSUPPORTED
     # forward cache: misaligned pointer, row bytes not a multiple of 16
     assert sbp.sbp_forward_cache(1, fake + 2, 8, 8, fake, None, 4, fake, stream=0, check=False) == sbp.SBP_ERR_INVALID_ARG
     assert sbp.sbp_forward_cache(1, fake, 8, 4, fake, None, 4, fake, stream=0, check=False) == sbp.SBP_ERR_UNSUPPORTED

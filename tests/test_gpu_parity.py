@@ -47,6 +47,11 @@ def relerr(got, want):
     (2, 2, 5, 6, 0.75, 1, 9, 0, sbp.SBP_FLAG_SHARE_MASK),
     (2, 1, 1500, 3, 0.5, 2, 1, 4, 0),                    # many frames: several sweeps of the ranking loops
     (2, 5, 32, 1, 1.0, 0, 0, 0, 0),
+    (3, 64, 9, 5, 0.5, 4, 2, 0, 0),                      # every second frame, ragged counts (5 or 4 of 9 frames)
+    (3, 48, 10, 3, 0.25, 9, 1, 7, 0),
+    (3, 600, 7, 2, 0.75, 9, 1, 0, 0),                    # more samples than threads: the offset sum loops
+    (3, 5, 6, 49, 0.5, 2, 0, 3, sbp.SBP_FLAG_SHARE_MASK),
+    (3, 3, 8, 196, 1.0, 0, 0, 0, 0),
 ])
 def test_keep_indices_bit_exact(mode, B, H, W, r, seed, step, off, flags):
     want_rows, want_offs = oracle.sample_keep(mode, B, H, W, r, seed, step, off, flags)
