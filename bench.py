@@ -428,6 +428,11 @@ def run_cuda(args, w, name):
         B_s = pick_oracle_sample(w)
         import oracle
         cpu_s, cpu_flops = oracle_sample_step(w, B_s, 1000)
+        cpu_threads = oracle.num_threads()
+        B_1 = max(1, B_s // 8)                              # single-thread figure on a smaller slice
+        oracle.set_num_threads(1)
+        cpu1_s, cpu1_flops = oracle_sample_step(w, B_1, 1000)
+        oracle.set_num_threads(cpu_threads)
         launches_per_step = 2 + sbp.sbp_linear_backward_kernel_count(code, M, cap_total, C_in, C_out, True, True, True, 0)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -440,9 +445,11 @@ def run_cuda(args, w, name):
                        "launch": ("CUDA graph replay, one captured step (3 C-ABI calls) per buffer set" if args.launch == "graph"
                                   else "direct C-ABI calls")},
             "roofline": roofline,
-            "cpu_baseline": {"value": cpu_flops / cpu_s / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+            "cpu_baseline": {"value": cpu_flops / cpu_s / 1e12, "unit": UNIT, "cores": cpu_threads,
                              "kind": "oracle", "seconds": cpu_s,
-                             "sample": f"first {B_s} of {B} samples of {name}, whole path once, fp64"},
+                             "sample": f"first {B_s} of {B} samples of {name}, whole path once, fp64",
+                             "single_thread": {"value": cpu1_flops / cpu1_s / 1e12, "unit": UNIT, "seconds": cpu1_s,
+                                               "sample": f"first {B_1} of {B} samples"}},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps, "api": "sbp_step_host (pinned host tensors; steps alternate between two streams so copies overlap)"},
             "gpu_launches": launches_per_step * args.steps,

@@ -61,6 +61,8 @@ def _load():
     lib.oracle_full_backward.restype = None
     lib.oracle_linear_forward.argtypes = [vp, vp, vp, i64, i64, i64, vp]
     lib.oracle_linear_forward.restype = None
+    lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
+    lib.oracle_set_num_threads.restype = None
     lib.oracle_num_threads.argtypes = []
     lib.oracle_num_threads.restype = ctypes.c_int
     _lib = lib
@@ -73,6 +75,10 @@ def _ptr(a):
 
 def _f64(a):
     return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def set_num_threads(n: int) -> None:
+    _load().oracle_set_num_threads(int(n))
 
 
 def num_threads() -> int:

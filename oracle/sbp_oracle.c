@@ -399,6 +399,16 @@ void oracle_full_backward(const double* X, const double* dY, const double* W,
     }
 }
 
+/* sets the number of threads the row loops use (for the single-thread baseline timing) */
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* threads the row loops above will use */
 int oracle_num_threads(void)
 {
