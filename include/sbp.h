@@ -60,7 +60,8 @@ enum {
     SBP_FLAG_VALIDATE = 4,    /* check keep_rows on the device before use; result in the status word */
     SBP_FLAG_PLAIN_FMA = 8,   /* bf16 only: use the CUDA-core FMA kernels instead of the tensor-core ones */
     SBP_FLAG_DY_COMPACT = 16, /* dY holds only the kept rows, packed: [M_keep_cap, C_out] (chained layers, Sec. 3.3.1) */
-    SBP_FLAG_DX_COMPACT = 32  /* dX receives only the kept rows, packed: [M_keep_cap, C_in]; no zero rows are written */
+    SBP_FLAG_DX_COMPACT = 32, /* dX receives only the kept rows, packed: [M_keep_cap, C_in]; no zero rows are written */
+    SBP_FLAG_W_OUT_IN = 64    /* W, and dW, are stored [C_out, C_in] (the usual layout of framework linear layers) */
 };
 
 const char* sbp_status_string(sbp_status s);
@@ -150,7 +151,8 @@ sbp_status sbp_forward_cache(sbp_dtype dt, const void* X /* dev */, int64_t M, i
  * from memory once.  SBP_BF16: bf16 inputs and output, fp32 accumulation on the
  * tensor cores, one rounding of (sum + bias) to bf16.  SBP_F32: fp32 FMA arithmetic.
  * C_in and C_out must be multiples of 8 (bf16) / 4 (fp32), else SBP_ERR_UNSUPPORTED.
- * flags: SBP_FLAG_PLAIN_FMA or 0.  status_word as for sbp_linear_backward.
+ * flags: SBP_FLAG_PLAIN_FMA, SBP_FLAG_W_OUT_IN (W is [C_out, C_in]; read in place, no
+ * copy) or 0.  status_word as for sbp_linear_backward.
  * SBP_ERR_INVALID_ARG for null or misaligned (16 bytes) pointers and bad sizes.
  */
 sbp_status sbp_linear_forward(sbp_dtype dt, const void* X /* dev */, const void* W /* dev */,
@@ -186,6 +188,12 @@ size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_ke
  * dY instead of row keep_rows[m] of the full one.  The layer at the block's boundary
  * uses neither flag on its side facing the rest of the network.  With both flags
  * keep_rows is not used and may be NULL.
+ *
+ * Weight layout.  The paper writes Y = X W with W [C_in, C_out] (Sec. 3.2.1), and that
+ * is the native layout here.  With SBP_FLAG_W_OUT_IN both W and dW are [C_out, C_in]
+ * (dW[j, i] as above with the indices swapped): W is transposed into the workspace
+ * before the products and dW is transposed out of it after them (two small extra
+ * launches); the results are the same numbers.
  *
  * SBP_BF16: inputs bf16, products accumulated in fp32 on the tensor cores, dX
  * rounded to bf16 (nearest even).  SBP_F32: plain fp32 FMA arithmetic.

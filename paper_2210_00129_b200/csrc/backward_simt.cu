@@ -189,8 +189,8 @@ simt_dx_kernel(const T* __restrict__ dY, const T* __restrict__ W, const int32_t*
 // The X tile is loaded along i (its contiguous side) and stored transposed, the W tile along j.
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads)
-simt_forward_kernel(const T* __restrict__ X, const T* __restrict__ W, const float* __restrict__ bias, int64_t M,
-                    int C_in, int C_out, T* __restrict__ Y, const int32_t* __restrict__ status_word) {
+simt_forward_kernel(const T* __restrict__ X, const T* __restrict__ W, int w_out_in, const float* __restrict__ bias,
+                    int64_t M, int C_in, int C_out, T* __restrict__ Y, const int32_t* __restrict__ status_word) {
     __shared__ __align__(16) float As[kTileK][kTile + 4];
     __shared__ __align__(16) float Bs[kTileK][kTile];
     pdl_launch_dependents();
@@ -206,9 +206,14 @@ simt_forward_kernel(const T* __restrict__ X, const T* __restrict__ W, const floa
     for (int i0 = 0; i0 < C_in; i0 += kTileK) {
         float4 a = zero4, b = zero4;
         if (m0 + ar < M && i0 + ac < C_in) a = load4<T>(X + (m0 + ar) * C_in + i0 + ac);
-        if (i0 + bk < C_in && j0 + bc < C_out) b = load4<T>(W + (int64_t)(i0 + bk) * C_out + j0 + bc);
         As[ac + 0][ar] = a.x; As[ac + 1][ar] = a.y; As[ac + 2][ar] = a.z; As[ac + 3][ar] = a.w;
-        *reinterpret_cast<float4*>(&Bs[bk][bc]) = b;
+        if (!w_out_in) {
+            if (i0 + bk < C_in && j0 + bc < C_out) b = load4<T>(W + (int64_t)(i0 + bk) * C_out + j0 + bc);
+            *reinterpret_cast<float4*>(&Bs[bk][bc]) = b;
+        } else {                                                      // W [C_out, C_in]: loaded along i like the X tile
+            if (j0 + ar < C_out && i0 + ac < C_in) b = load4<T>(W + (int64_t)(j0 + ar) * C_in + i0 + ac);
+            Bs[ac + 0][ar] = b.x; Bs[ac + 1][ar] = b.y; Bs[ac + 2][ar] = b.z; Bs[ac + 3][ar] = b.w;
+        }
         __syncthreads();
 #pragma unroll
         for (int k = 0; k < kTileK; ++k) {
@@ -237,15 +242,15 @@ simt_forward_kernel(const T* __restrict__ X, const T* __restrict__ W, const floa
 
 }  // namespace
 
-cudaError_t launch_simt_forward(sbp_dtype dt, const void* X, const void* W, const float* bias, int64_t M, int64_t C_in,
-                                int64_t C_out, void* Y, const int32_t* status_word, cudaStream_t stream) {
+cudaError_t launch_simt_forward(sbp_dtype dt, const void* X, const void* W, bool w_out_in, const float* bias, int64_t M,
+                                int64_t C_in, int64_t C_out, void* Y, const int32_t* status_word, cudaStream_t stream) {
     const dim3 grid((unsigned)((M + kTile - 1) / kTile), (unsigned)((C_out + kTile - 1) / kTile));
     if (dt == SBP_BF16)
         return launch_pdl(simt_forward_kernel<__nv_bfloat16>, grid, dim3(kSimtThreads), 0, stream,
-                          (const __nv_bfloat16*)X, (const __nv_bfloat16*)W, bias, M, (int)C_in, (int)C_out,
-                          (__nv_bfloat16*)Y, status_word);
+                          (const __nv_bfloat16*)X, (const __nv_bfloat16*)W, w_out_in ? 1 : 0, bias, M, (int)C_in,
+                          (int)C_out, (__nv_bfloat16*)Y, status_word);
     return launch_pdl(simt_forward_kernel<float>, grid, dim3(kSimtThreads), 0, stream, (const float*)X, (const float*)W,
-                      bias, M, (int)C_in, (int)C_out, (float*)Y, status_word);
+                      w_out_in ? 1 : 0, bias, M, (int)C_in, (int)C_out, (float*)Y, status_word);
 }
 
 size_t simt_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out) {

@@ -153,15 +153,17 @@ sbp_status sbp_linear_forward(sbp_dtype dt, const void* X, const void* W, const 
             const double byte_us = ((double)M * (double)(C_in + C_out) * 2.0) / 5.0e6;                 // at 5 TB/s
             ride = copy_us <= 0.25 * (flop_us > byte_us ? flop_us : byte_us);
         }
-        const sbp_status s = launch_tc_forward(X, W, bias, M, C_in, C_out, Y, keep_rows, M_keep_dev, M_keep_cap,
-                                               ride ? X_keep : nullptr, status_word, stream);
+        const sbp_status s = launch_tc_forward(X, W, (flags & SBP_FLAG_W_OUT_IN) != 0, bias, M, C_in, C_out, Y, keep_rows,
+                                               M_keep_dev, M_keep_cap, ride ? X_keep : nullptr, status_word, stream);
         if (s != SBP_OK) return s;
         if (X_keep != nullptr && !ride &&
             launch_gather_rows(X, C_in * 2, keep_rows, M_keep_dev, M_keep_cap, X_keep, stream) != cudaSuccess)
             return SBP_ERR_CUDA;
         return SBP_OK;
     }
-    if (launch_simt_forward(dt, X, W, bias, M, C_in, C_out, Y, status_word, stream) != cudaSuccess) return SBP_ERR_CUDA;
+    if (launch_simt_forward(dt, X, W, (flags & SBP_FLAG_W_OUT_IN) != 0, bias, M, C_in, C_out, Y, status_word, stream) !=
+        cudaSuccess)
+        return SBP_ERR_CUDA;
     if (X_keep != nullptr &&
         launch_gather_rows(X, C_in * (dt == SBP_BF16 ? 2 : 4), keep_rows, M_keep_dev, M_keep_cap, X_keep, stream) !=
             cudaSuccess)
@@ -169,9 +171,24 @@ sbp_status sbp_linear_forward(sbp_dtype dt, const void* X, const void* W, const 
     return SBP_OK;
 }
 
+namespace {
+size_t base_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+// after the kernels' own scratch: room for W and dW in the [C_in, C_out] layout, used with SBP_FLAG_W_OUT_IN
+size_t w_copy_bytes(sbp_dtype dt, int64_t C_in, int64_t C_out) {
+    return align_up((size_t)C_in * (size_t)C_out * (dt == SBP_BF16 ? 2 : 4), 256);
+}
+size_t dw_copy_bytes(int64_t C_in, int64_t C_out) { return align_up((size_t)C_in * (size_t)C_out * 4, 256); }
+}  // namespace
+
 size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                            int64_t C_out) {
     if (M <= 0 || M_keep_cap < 0 || C_in <= 0 || C_out <= 0) return 256;
+    return base_workspace_bytes(dt, M, M_keep_cap, C_in, C_out) + w_copy_bytes(dt, C_in, C_out) +
+           dw_copy_bytes(C_in, C_out);
+}
+
+namespace {
+size_t base_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
     const size_t db_part = db_scratch_bytes(dt, M_keep_cap, C_out);
     size_t dw_part = simt_dw_workspace_bytes(M_keep_cap, C_in, C_out);
     if (dt == SBP_BF16 && tc_shapes_supported(M, M_keep_cap, C_in, C_out)) {
@@ -180,13 +197,15 @@ size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_ke
     }
     return db_part + align_up(dw_part, 256) + 256;
 }
+}  // namespace
 
-sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY, const void* W,
-                               const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M,
-                               int64_t M_keep_cap, int64_t C_in, int64_t C_out, float* dW, float* db, void* dX,
-                               uint32_t flags, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                               void* stream_v) {
-    cudaStream_t stream = (cudaStream_t)stream_v;
+namespace {
+// the backward with W and dW in the paper's [C_in, C_out] layout
+sbp_status backward_in_out(sbp_dtype dt, const void* X_keep, const void* dY, const void* W,
+                           const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M,
+                           int64_t M_keep_cap, int64_t C_in, int64_t C_out, float* dW, float* db, void* dX,
+                           uint32_t flags, void* workspace, size_t workspace_bytes, size_t workspace_required,
+                           int32_t* status_word, cudaStream_t stream) {
     if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
     const bool dy_compact = (flags & SBP_FLAG_DY_COMPACT) != 0, dx_compact = (flags & SBP_FLAG_DX_COMPACT) != 0;
     // the packed forms address rows by their position m; keep_rows is needed for whichever side is not packed
@@ -206,7 +225,7 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     const bool need_ws = (dW != nullptr) || (db != nullptr);
     if (need_ws) {
         if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-            workspace_bytes < sbp_linear_backward_workspace_bytes(dt, M, M_keep_cap, C_in, C_out))
+            workspace_bytes < workspace_required)
             return SBP_ERR_WORKSPACE;
     }
     const bool accumulate = (flags & SBP_FLAG_ACCUMULATE) != 0;
@@ -247,10 +266,61 @@ sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY,
     return SBP_OK;
 }
 
+}  // namespace
+
+sbp_status sbp_linear_backward(sbp_dtype dt, const void* X_keep, const void* dY, const void* W,
+                               const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M,
+                               int64_t M_keep_cap, int64_t C_in, int64_t C_out, float* dW, float* db, void* dX,
+                               uint32_t flags, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                               void* stream_v) {
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    if (!(flags & SBP_FLAG_W_OUT_IN) || (dW == nullptr && dX == nullptr))
+        return backward_in_out(dt, X_keep, dY, W, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, dW, db, dX, flags,
+                               workspace, workspace_bytes,
+                               (M > 0 && M_keep_cap >= 0 && C_in > 0 && C_out > 0)
+                                   ? sbp_linear_backward_workspace_bytes(dt, M, M_keep_cap, C_in, C_out) : 0,
+                               status_word, stream);
+    // W and dW are [C_out, C_in]: transpose W into the workspace, run the products on the copies, transpose dW out
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (M <= 0 || M_keep_cap < 0 || C_in <= 0 || C_out <= 0 || C_in >= (1ll << 24) || C_out >= (1ll << 24))
+        return SBP_ERR_INVALID_ARG;
+    if ((dX != nullptr && W == nullptr) || !aligned16(W) || !aligned16(dW)) return SBP_ERR_INVALID_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < sbp_linear_backward_workspace_bytes(dt, M, M_keep_cap, C_in, C_out))
+        return SBP_ERR_WORKSPACE;
+    const size_t base = base_workspace_bytes(dt, M, M_keep_cap, C_in, C_out);
+    void* w_copy = static_cast<char*>(workspace) + base;
+    float* dw_copy = reinterpret_cast<float*>(static_cast<char*>(workspace) + base + w_copy_bytes(dt, C_in, C_out));
+    const uint32_t inner = flags & ~(uint32_t)SBP_FLAG_W_OUT_IN;
+    if (dX != nullptr &&
+        launch_transpose(dt == SBP_BF16 ? 2 : 4, W, w_copy, C_out, C_in, status_word, stream) != cudaSuccess)
+        return SBP_ERR_CUDA;
+    const bool accumulate = (flags & SBP_FLAG_ACCUMULATE) != 0;
+    sbp_status s;
+    if (accumulate && dW != nullptr) {
+        // dW is produced fresh in the copy and added in by the transpose; db accumulates in place on its own
+        s = backward_in_out(dt, X_keep, dY, dX != nullptr ? w_copy : nullptr, keep_rows, M_keep_dev, M, M_keep_cap, C_in,
+                            C_out, dw_copy, nullptr, dX, inner & ~(uint32_t)SBP_FLAG_ACCUMULATE, workspace, base, base,
+                            status_word, stream);
+        if (s == SBP_OK && db != nullptr)
+            s = backward_in_out(dt, nullptr, dY, nullptr, keep_rows, M_keep_dev, M, M_keep_cap, C_in, C_out, nullptr, db,
+                                nullptr, inner & ~(uint32_t)SBP_FLAG_VALIDATE, workspace, base, base, status_word, stream);
+    } else {
+        s = backward_in_out(dt, X_keep, dY, dX != nullptr ? w_copy : nullptr, keep_rows, M_keep_dev, M, M_keep_cap, C_in,
+                            C_out, dW != nullptr ? dw_copy : nullptr, db, dX, inner, workspace, base, base, status_word, stream);
+    }
+    if (s != SBP_OK) return s;
+    if (dW != nullptr &&
+        launch_transpose_add_f32(dw_copy, dW, C_in, C_out, accumulate, status_word, stream) != cudaSuccess)
+        return SBP_ERR_CUDA;
+    return SBP_OK;
+}
+
 int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out,
                                      int want_dW, int want_db, int want_dX, uint32_t flags) {
     const bool tc = use_tensor_cores(dt, flags, M, M_keep_cap, C_in, C_out);
     int n = (flags & SBP_FLAG_VALIDATE) ? 1 : 0;
+    if ((flags & SBP_FLAG_W_OUT_IN) && (want_dW || want_dX)) n += (want_dX ? 1 : 0) + (want_dW ? 1 : 0);   // transposes
     const bool db_rides = tc && want_db && (want_dW || want_dX);
     if (want_db && !db_rides) n += 2;                      // strip partials + fixed-order reduce
     if (tc) return n + tc_backward_kernel_count(M_keep_cap, C_in, C_out, want_dW != 0, want_dX != 0, db_rides);

@@ -150,12 +150,19 @@ cudaError_t launch_simt_dx(sbp_dtype dt, const void* dY, const void* W, const in
                            const int32_t* dx_rows, const int32_t* M_keep_dev, int64_t M, int64_t M_keep_cap,
                            int64_t C_in, int64_t C_out, void* dX, const int32_t* status_word, cudaStream_t stream);
 
+// transposes for weights in the [C_out, C_in] layout
+cudaError_t launch_transpose(int elem_bytes, const void* in, void* out, int64_t rows, int64_t cols,
+                             const int32_t* status_word, cudaStream_t stream);
+cudaError_t launch_transpose_add_f32(const float* in, float* out, int64_t rows, int64_t cols, bool accumulate,
+                                     const int32_t* status_word, cudaStream_t stream);
+
 // forward of the layer, Y = X W + bias (bias nullable)
-cudaError_t launch_simt_forward(sbp_dtype dt, const void* X, const void* W, const float* bias, int64_t M, int64_t C_in,
-                                int64_t C_out, void* Y, const int32_t* status_word, cudaStream_t stream);
+// w_out_in: W is stored [C_out, C_in] instead of [C_in, C_out]
+cudaError_t launch_simt_forward(sbp_dtype dt, const void* X, const void* W, bool w_out_in, const float* bias, int64_t M,
+                                int64_t C_in, int64_t C_out, void* Y, const int32_t* status_word, cudaStream_t stream);
 bool   tc_forward_supported(int64_t M, int64_t C_in, int64_t C_out);
 // bf16 forward on the tensor cores; when X_keep is given the same kernel also writes the forward cache
-sbp_status launch_tc_forward(const void* X, const void* W, const float* bias, int64_t M, int64_t C_in, int64_t C_out,
+sbp_status launch_tc_forward(const void* X, const void* W, bool w_out_in, const float* bias, int64_t M, int64_t C_in, int64_t C_out,
                              void* Y, const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap,
                              void* X_keep, int32_t* status_word, cudaStream_t stream);
 

@@ -55,6 +55,7 @@ struct FwdParams {
     const int32_t* keep_rows;
     const int32_t* M_keep_dev;
     int64_t M_keep_cap;
+    int w_out_in;                  // W is [C_out, C_in]: the B tile is K-major and arrives as one TMA box
     int32_t* status_word;
 };
 
@@ -120,9 +121,13 @@ tc_forward_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     const uint32_t a_dst = ring + s * kStageBytes;
                     ptx::mbar_arrive_expect_tx(full, kABytes + BN * kRowBytes);
                     ptx::tma_load_2d(a_dst, &map_x, (int)(k * kBK), row0, full);                 // 128 rows x 64 columns of X
+                    if (p.w_out_in) {                                                           // BN rows (j) x 64 columns (i) of W
+                        ptx::tma_load_2d(a_dst + kABytes, &map_w, (int)(k * kBK), n0, full);
+                    } else {
 #pragma unroll
-                    for (int b = 0; b < BN / 64; ++b)                                           // 64 rows (i) x 64 columns (j) of W
-                        ptx::tma_load_2d(a_dst + kABytes + b * kBlock64Bytes, &map_w, n0 + b * 64, (int)(k * kBK), full);
+                        for (int b = 0; b < BN / 64; ++b)                                       // 64 rows (i) x 64 columns (j) of W
+                            ptx::tma_load_2d(a_dst + kABytes + b * kBlock64Bytes, &map_w, n0 + b * 64, (int)(k * kBK), full);
+                    }
                 }
             }
             if (!ok) {   // let the copies already issued land before shared memory goes away
@@ -139,7 +144,9 @@ tc_forward_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         if (lane == 0) {
             uint32_t it = 0, used = 0;
             bool ok = true;
-            const uint32_t idesc = ptx::umma_idesc_bf16(kBM, BN, false, true);   // A K-major, B MN-major
+            // A K-major; B MN-major for W [C_in, C_out], K-major for W [C_out, C_in]
+            const uint32_t idesc = ptx::umma_idesc_bf16(kBM, BN, false, p.w_out_in == 0);
+            const uint32_t b_step = p.w_out_in ? kUmmaK * 2 : kUmmaK * kRowBytes, b_lbo = p.w_out_in ? 16u : kBlock64Bytes;
             for (uint32_t q = blockIdx.x; q < total && ok; q += gridDim.x, ++used) {
                 const uint32_t acc = used & 1u;
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[acc]), ((used >> 1) & 1u) ^ 1u, abort_flag, status_word);
@@ -156,7 +163,7 @@ tc_forward_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     for (uint32_t u = 0; u < kBK / kUmmaK; ++u) {
                         // A: a 16-deep slice is 32 bytes along the swizzled row; B: 16 rows, 64-wide blocks 8 KB apart
                         const uint64_t da = ptx::umma_desc_sw128(a_addr + u * kUmmaK * 2, 16, kAtomBytes);
-                        const uint64_t db = ptx::umma_desc_sw128(b_addr + u * kUmmaK * kRowBytes, kBlock64Bytes, kAtomBytes);
+                        const uint64_t db = ptx::umma_desc_sw128(b_addr + u * b_step, b_lbo, kAtomBytes);
                         ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
                     }
                     ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));
@@ -312,12 +319,15 @@ bool tc_forward_supported(int64_t M, int64_t C_in, int64_t C_out) {
     return M >= kBM && M < (1ll << 31) && C_in >= 128 && C_out >= 128 && C_in % 8 == 0 && C_out % 8 == 0;
 }
 
-sbp_status launch_tc_forward(const void* X, const void* W, const float* bias, int64_t M, int64_t C_in, int64_t C_out,
+sbp_status launch_tc_forward(const void* X, const void* W, bool w_out_in, const float* bias, int64_t M, int64_t C_in, int64_t C_out,
                              void* Y, const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap,
                              void* X_keep, int32_t* status_word, cudaStream_t stream) {
     CUtensorMap map_x, map_w;
-    if (!make_map(&map_x, X, M, C_in, (uint32_t)kBM) || !make_map(&map_w, W, C_in, C_out, 64u)) return SBP_ERR_CUDA;
+    const int bn = C_out >= 256 ? 256 : 128;
+    if (!make_map(&map_x, X, M, C_in, (uint32_t)kBM)) return SBP_ERR_CUDA;
+    if (w_out_in ? !make_map(&map_w, W, C_out, C_in, (uint32_t)bn) : !make_map(&map_w, W, C_in, C_out, 64u)) return SBP_ERR_CUDA;
     FwdParams prm;
+    prm.w_out_in = w_out_in ? 1 : 0;
     prm.bias = bias;
     prm.Y = static_cast<__nv_bfloat16*>(Y);
     prm.M = M;
@@ -329,7 +339,6 @@ sbp_status launch_tc_forward(const void* X, const void* W, const float* bias, in
     prm.M_keep_dev = M_keep_dev;
     prm.M_keep_cap = M_keep_cap;
     prm.status_word = status_word;
-    const int bn = C_out >= 256 ? 256 : 128;
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((C_out + bn - 1) / bn);
     const dim3 grid((unsigned)(tiles < kNumSMs ? tiles : kNumSMs));
     const cudaError_t e = bn == 256 ? launch_forward<256>(grid, stream, map_x, map_w, prm)
