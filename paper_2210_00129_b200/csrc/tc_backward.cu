@@ -55,7 +55,9 @@ constexpr int kBiasChunk = 64;           // kept rows whose ids the bias warps s
 // 16-byte loads each side-warp thread keeps in flight for the bias sums: a template parameter of the kernel,
 // 8 or 16.  The deep queue finishes long row lists in time; with short lists it only takes memory
 // bandwidth from the operand copies (ViT-B fc1: 5 us per call), so the host picks per shape.
-constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float) + kBiasChunk * sizeof(int);   // cross-row-group sums + staged row ids
+// cross-row-group sums + staged row ids, padded so that the staging buffers after it start on a 1024-byte boundary
+// (one of them holds a swizzled tensor-core operand)
+constexpr uint32_t kBiasSmemBytes = kBiasThreads * 8 * sizeof(float) + kBiasChunk * sizeof(int) + 512;
 constexpr int kEpiChunk = 16;            // accumulator columns (= rows of dW) per TMA store of the dW epilogue
 constexpr int kEpiBufs = 3;              // staging buffers the dW epilogue rotates through
 constexpr uint32_t kEpiBufBytes = kEpiChunk * kBM * sizeof(float);   // 8 KB: 16 rows of dW x 128 columns
@@ -63,7 +65,7 @@ constexpr int kEpiBarrier = 2;           // named barrier of the four epilogue w
 constexpr uint32_t kRingBytes = kStages * kStageBytes;
 static_assert(kRingBytes == kStagesNarrow * (kABytes + 128 * kRowBytes), "both ring shapes fill the same memory");
 constexpr uint32_t kSmemBytes = kRingBytes + 256 + kBiasSmemBytes + kEpiBufs * kEpiBufBytes + 1024;   // ring + control + bias + staging + slack
-static_assert((256 + kBiasSmemBytes) % 128 == 0, "staging buffers start on a 128-byte boundary");
+static_assert((256 + kBiasSmemBytes) % 1024 == 0, "staging buffers start on a 1024-byte boundary");
 static_assert(kSmemBytes <= 227 * 1024, "shared memory per block");
 
 struct TcControl {
@@ -88,6 +90,8 @@ struct TcParams {
     int64_t dw_split_stride;       // elements between partial buffers
     int dw_splits;
     int dw_accumulate;             // add into dW_out (only with one split)
+    int db_from_mma;               // narrow layers: db comes out of the dW tiles (a column of ones appended to X_keep);
+                                   // db_partial is then [dw_splits, C_out]
     float* db_partial;             // nullptr: no bias sums; else [gridDim.x, C_out] per-CTA column sums of kept dY rows
     int32_t* status_word;
 };
@@ -250,6 +254,21 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         ptx::prefetch_tensormap(&map_w);
         ptx::prefetch_tensormap(&map_x);
     }
+    // Narrow layers leave half of each accumulator slot unused, which makes room for the bias gradient as one more
+    // output column of the dW tiles: db[j] = sum_m dY[m, j] * 1.  The "column of ones" is a constant 64 x 64 operand
+    // block (MN-major, only its first column set) kept in the third staging buffer; a second, 16-wide MMA per k-step
+    // multiplies it with the same gathered rows of dY.
+    const uint32_t dw_bufs = (kNarrow && p.db_from_mma) ? kEpiBufs - 1 : kEpiBufs;   // staging buffers left to the dW epilogue
+    const uint32_t ones_off = (ring - raw_addr) + kRingBytes + 256 + kBiasSmemBytes + (kEpiBufs - 1) * kEpiBufBytes;
+    if constexpr (kNarrow) {
+        if (p.db_from_mma) {
+            for (uint32_t w = threadIdx.x; w < kBlock64Bytes / 4; w += kTcThreads) {
+                const uint32_t row = w >> 5, word = w & 31u;            // 128-byte rows of 32 words; column 0 sits in chunk (row & 7)
+                reinterpret_cast<uint32_t*>(smem_raw + ones_off)[w] = (word == ((row & 7u) << 2)) ? 0x00003F80u : 0u;
+            }
+            ptx::fence_async_proxy();                                    // read by the tensor core (async proxy)
+        }
+    }
     if (warp == 5) ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -335,6 +354,12 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, kAtomBytes);
                         const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, kAtomBytes);
                         ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
+                        if constexpr (kNarrow) {
+                            if (t.is_dw && t.col_tile == 0 && p.db_from_mma) {   // the bias column: accumulator columns 128..143, column 128 is db
+                                const uint64_t d1 = ptx::umma_desc_sw128(raw_addr + ones_off + u * k_step, kBlock64Bytes, kAtomBytes);
+                                ptx::umma_bf16(d_tmem + 128u, da, d1, ptx::umma_idesc_bf16(kBM, 16, true, true), (k | u) != 0u);
+                            }
+                        }
                     }
                     ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));      // stage reusable once these MMAs retire
                 }
@@ -442,7 +467,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         // db partial of this CTA's share of the kept rows
-        if (p.db_partial != nullptr) {
+        if (p.db_partial != nullptr && !(kNarrow && p.db_from_mma)) {
             float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kRingBytes + 256);
             const int t = threadIdx.x - kBiasWarp0 * 32;
             const int V = C_out >> 3;                                  // 16-byte column vectors per row
@@ -571,9 +596,11 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const int j = (int)(t.row_tile * kBM) + warp * 32 + lane;
                 const int i0 = (int)(t.col_tile * BNW);
                 float* out_col = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i0 * C_out + j;
+                const bool bias_col = kNarrow && p.db_from_mma && t.col_tile == 0;
                 if (t.num_kb == 0) {                                 // a piece without kept rows contributes zero
                     if (!p.dw_accumulate && j < C_out)
                         for (int c0 = 0; c0 < BNW && i0 + c0 < C_in; ++c0) out_col[(int64_t)c0 * C_out] = 0.f;
+                    if (bias_col && j < C_out) p.db_partial[(int64_t)t.split * C_out + j] = 0.f;
                     continue;
                 }
                 if (lane == 0) ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_full[acc]), (used >> 1) & 1u, abort_flag, status_word);
@@ -594,18 +621,27 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         float v[kEpiChunk];
                         ptx::tmem_ld_32x16(taddr + (uint32_t)(c * kEpiChunk), v);
                         ptx::tmem_ld_wait();
-                        const uint32_t buf_off = stage_off + (staged % kEpiBufs) * kEpiBufBytes;
+                        const uint32_t buf_off = stage_off + (staged % dw_bufs) * kEpiBufBytes;
                         float* buf = reinterpret_cast<float*>(smem_raw + buf_off) + warp * 32 + lane;
 #pragma unroll
                         for (int r = 0; r < kEpiChunk; ++r) buf[r * kBM] = v[r];
                         ptx::fence_async_proxy();
-                        if (threadIdx.x == 0) ptx::bulk_wait_read<1>();
+                        if (threadIdx.x == 0) {                          // the buffer written next must have been read out
+                            if (dw_bufs >= 3) ptx::bulk_wait_read<1>();
+                            else ptx::bulk_wait_read<0>();
+                        }
                         ptx::bar_named<kEpiBarrier, 128>();
                         if (threadIdx.x == 0) {
                             if (add_in) ptx::tma_reduce_add_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
                             else ptx::tma_store_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
                             ptx::bulk_commit();
                         }
+                    }
+                    if (bias_col) {                                  // accumulator column 128: this piece's share of db
+                        float v[kEpiChunk];
+                        ptx::tmem_ld_32x16(taddr + 128u, v);
+                        ptx::tmem_ld_wait();
+                        if (j < C_out) p.db_partial[(int64_t)t.split * C_out + j] = v[0];
                     }
                 }
             }
@@ -841,6 +877,10 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
         map_dw = map_x;                                              // never used
     }
     prm.db_partial = (db != nullptr) ? db_workspace : nullptr;
+    // narrow layers (both tile kinds 128 wide): db is one more output column of the dW tiles, one partial row per split
+    const bool db_from_mma = db != nullptr && want_dw && pl.bnx <= 128 && pl.bnw <= 128;
+    prm.db_from_mma = db_from_mma ? 1 : 0;
+    const int db_rows = db_from_mma ? pl.splits : 0;                 // 0: one row per block (set below)
     prm.status_word = status_word;
     int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
     if (ctas < 1) ctas = 1;
@@ -867,12 +907,12 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     const bool reduce_dw = want_dw && pl.splits > 1, reduce_db = db != nullptr;
     cudaError_t r = cudaSuccess;
     if (reduce_dw && reduce_db)
-        r = launch_reduce_partials_pair(workspace, pl.splits, C_in * C_out, dW, db_workspace, (int)ctas, C_out, db,
+        r = launch_reduce_partials_pair(workspace, pl.splits, C_in * C_out, dW, db_workspace, db_rows ? db_rows : (int)ctas, C_out, db,
                                         accumulate, status_word, stream);
     else if (reduce_dw)
         r = launch_reduce_partials(workspace, pl.splits, C_in * C_out, dW, accumulate, status_word, stream);
     else if (reduce_db)
-        r = launch_reduce_partials(db_workspace, (int)ctas, C_out, db, accumulate, status_word, stream);
+        r = launch_reduce_partials(db_workspace, db_rows ? db_rows : (int)ctas, C_out, db, accumulate, status_word, stream);
     if (r != cudaSuccess) return SBP_ERR_CUDA;
     return SBP_OK;
 }
