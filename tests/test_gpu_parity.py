@@ -197,7 +197,7 @@ def test_nothing_kept_gives_all_zero_gradients(dtype, C_in, C_out):
         assert not np.any(host(got[k]).view(np.uint8)), k
 
 
-@pytest.mark.parametrize("dtype,C_in,C_out", [("f32", 32, 64), ("bf16", 256, 384)])
+@pytest.mark.parametrize("dtype,C_in,C_out", [("f32", 32, 64), ("bf16", 256, 384), ("bf16", 128, 264)])   # last: bias from the dW tiles
 def test_accumulate_flag_adds_into_dw_and_db(dtype, C_in, C_out):
     M, X, Wt, dY, keep = _case(dtype, 4, 14, 14, C_in, C_out, 0.5, sig=(1.0, 0.1, 1.0))
     rows_d = torch.from_numpy(keep).cuda()
