@@ -170,6 +170,9 @@ sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t 
                                   int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
     __shared__ SampShared sh;
     __shared__ uint32_t slice_counts[2];          // positions of this slice below / equal to the threshold
+    // Two histograms used alternately: the one a pass clears was last read by the other blocks two passes
+    // earlier, before the cluster barrier of the pass in between, so one barrier per pass is enough.
+    __shared__ uint32_t hist2[2][256];
     pdl_launch_dependents();
     pdl_wait();
     const uint32_t rank = cluster_rank();
@@ -187,21 +190,22 @@ sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t 
     }
 
     uint32_t prefix = 0, known = 0, remaining = K;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = threadIdx.x; i < 256; i += kSampThreads) sh.hist[i] = 0;
+    for (int shift = 24, pass = 0; shift >= 0; shift -= 8, ++pass) {
+        uint32_t* hist = hist2[pass & 1];
+        for (int i = threadIdx.x; i < 256; i += kSampThreads) hist[i] = 0;
         __syncthreads();
         for (uint32_t q = g_begin + threadIdx.x; q < g_end; q += kSampThreads) {
             const PhiloxWords pw = position_words(q, gid, step, k0, k1);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const uint32_t n = 4u * q + e;
-                if (n < N && (pw.w[e] & known) == prefix) atomicAdd(&sh.hist[(pw.w[e] >> shift) & 0xffu], 1u);
+                if (n < N && (pw.w[e] & known) == prefix) atomicAdd(&hist[(pw.w[e] >> shift) & 0xffu], 1u);
             }
         }
         cluster_sync();                                   // every slice's histogram is complete
         uint32_t cnt = 0;
         if (threadIdx.x < 256)
-            for (uint32_t r = 0; r < (uint32_t)C; ++r) cnt += cluster_load(&sh.hist[threadIdx.x], r);
+            for (uint32_t r = 0; r < (uint32_t)C; ++r) cnt += cluster_load(&hist[threadIdx.x], r);
         const uint2 sc = block_excl_scan(cnt, sh.warp_sums_a);
         if (threadIdx.x < 256 && sc.x < remaining && remaining <= sc.x + cnt) {
             sh.sel_digit = threadIdx.x;
@@ -211,7 +215,7 @@ sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t 
         prefix |= sh.sel_digit << shift;
         known |= 0xffu << shift;
         remaining -= sh.sel_below;
-        cluster_sync();                                   // nobody still reads a histogram that is about to be cleared
+        __syncthreads();                                  // sel_digit / sel_below are read before the next pass rewrites them
     }
     const uint32_t threshold = prefix;
 
