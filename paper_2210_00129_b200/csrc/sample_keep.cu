@@ -166,8 +166,11 @@ __device__ __forceinline__ uint32_t cluster_load(const uint32_t* local_ptr, uint
 template <int C>
 __global__ void __launch_bounds__(kSampThreads)
 sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint32_t step,
-                                  uint32_t first_sample, int share_mask,
+                                  uint32_t first_sample, int share_mask, int cache_words,
                                   int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
+    // The selection looks at every word six times (four digit passes, the tie count, the compaction).  When the
+    // slice's words fit in shared memory they are generated once and kept there; otherwise each look recomputes them.
+    extern __shared__ uint4 word_cache[];
     __shared__ SampShared sh;
     __shared__ uint32_t slice_counts[2];          // positions of this slice below / equal to the threshold
     // Two histograms used alternately: the one a pass clears was last read by the other blocks two passes
@@ -189,13 +192,28 @@ sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t 
         if (b == 0) keep_offsets[0] = 0;
     }
 
+    if (cache_words) {
+        for (uint32_t q = g_begin + threadIdx.x; q < g_end; q += kSampThreads) {
+            const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+            word_cache[q - g_begin] = make_uint4(pw.w[0], pw.w[1], pw.w[2], pw.w[3]);
+        }
+        __syncthreads();
+    }
+    auto words_of = [&](uint32_t q) {
+        if (!cache_words) return position_words(q, gid, step, k0, k1);
+        const uint4 v = word_cache[q - g_begin];
+        PhiloxWords pw;
+        pw.w[0] = v.x; pw.w[1] = v.y; pw.w[2] = v.z; pw.w[3] = v.w;
+        return pw;
+    };
+
     uint32_t prefix = 0, known = 0, remaining = K;
     for (int shift = 24, pass = 0; shift >= 0; shift -= 8, ++pass) {
         uint32_t* hist = hist2[pass & 1];
         for (int i = threadIdx.x; i < 256; i += kSampThreads) hist[i] = 0;
         __syncthreads();
         for (uint32_t q = g_begin + threadIdx.x; q < g_end; q += kSampThreads) {
-            const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+            const PhiloxWords pw = words_of(q);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const uint32_t n = 4u * q + e;
@@ -222,7 +240,7 @@ sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t 
     // slice counts -> rank of this slice's first tie and its first output slot
     uint32_t lt = 0, eq = 0;
     for (uint32_t q = g_begin + threadIdx.x; q < g_end; q += kSampThreads) {
-        const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+        const PhiloxWords pw = words_of(q);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (4u * q + e < N) {
@@ -248,7 +266,7 @@ sample_keep_random_cluster_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t 
         const uint32_t q = q0 + threadIdx.x;
         uint32_t lt_mask = 0, eq_mask = 0;
         if (q < g_end) {
-            const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+            const PhiloxWords pw = words_of(q);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 if (4u * q + e < N) {
@@ -460,6 +478,22 @@ sample_keep_temporal_kernel(int family, uint32_t T, uint32_t P, uint32_t KT, uin
 
 uint32_t sample_keep_max_frames() { return kMaxFrames; }
 
+namespace {
+constexpr size_t kClusterCacheMax = 160 * 1024;
+
+template <int C>
+cudaError_t launch_cluster_sampler(dim3 grid, dim3 block, size_t cache_bytes, cudaStream_t stream, int64_t N, int64_t K,
+                                   uint32_t k0, uint32_t k1, uint32_t step, uint32_t first_sample, bool share_mask,
+                                   int32_t* keep_rows, int32_t* keep_offsets) {
+    static cudaError_t once = cudaFuncSetAttribute(sample_keep_random_cluster_kernel<C>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterCacheMax);
+    if (once != cudaSuccess) return once;
+    return launch_pdl_cluster(sample_keep_random_cluster_kernel<C>, grid, block, cache_bytes, C, stream, (uint32_t)N,
+                              (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, cache_bytes ? 1 : 0, keep_rows,
+                              keep_offsets);
+}
+}  // namespace
+
 cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, int64_t W, int64_t K,
                                uint64_t seed, uint32_t step, uint32_t first_sample, bool share_mask,
                                int32_t* keep_rows, int32_t* keep_offsets, cudaStream_t stream) {
@@ -471,16 +505,13 @@ cudaError_t launch_sample_keep(int mode, int grid_family, int64_t B, int64_t H, 
         int cluster = 1;
         if (K < N && N > 8192 && B * 8 <= 4 * kNumSMs) cluster = N > 32768 ? 8 : (N > 16384 ? 4 : 2);
         const dim3 cgrid((unsigned)(B * cluster));
+        // shared-memory cache of the slice's words (16 bytes per group of four positions), when it fits
+        const int64_t slice_groups = (((N + 3) / 4) + cluster - 1) / cluster;
+        const size_t cache_bytes = (size_t)slice_groups * 16 <= kClusterCacheMax ? (size_t)slice_groups * 16 : 0;
         switch (cluster) {
-            case 8:
-                return launch_pdl_cluster(sample_keep_random_cluster_kernel<8>, cgrid, block, 0, 8, stream, (uint32_t)N,
-                                          (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
-            case 4:
-                return launch_pdl_cluster(sample_keep_random_cluster_kernel<4>, cgrid, block, 0, 4, stream, (uint32_t)N,
-                                          (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
-            case 2:
-                return launch_pdl_cluster(sample_keep_random_cluster_kernel<2>, cgrid, block, 0, 2, stream, (uint32_t)N,
-                                          (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, keep_rows, keep_offsets);
+            case 8: return launch_cluster_sampler<8>(cgrid, block, cache_bytes, stream, N, K, k0, k1, step, first_sample, share_mask, keep_rows, keep_offsets);
+            case 4: return launch_cluster_sampler<4>(cgrid, block, cache_bytes, stream, N, K, k0, k1, step, first_sample, share_mask, keep_rows, keep_offsets);
+            case 2: return launch_cluster_sampler<2>(cgrid, block, cache_bytes, stream, N, K, k0, k1, step, first_sample, share_mask, keep_rows, keep_offsets);
             default: break;
         }
         return launch_pdl(sample_keep_random_kernel, grid, block, 0, stream, (uint32_t)(H * W), (uint32_t)K, k0, k1,
