@@ -56,6 +56,9 @@ sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint
                           uint32_t first_sample, int share_mask,
                           int32_t* __restrict__ keep_rows, int32_t* __restrict__ keep_offsets) {
     __shared__ SampShared sh;
+    // the selection looks at every word five times: maps of up to 8192 positions keep their words here
+    constexpr uint32_t kCacheGroups = 2048;
+    __shared__ uint4 word_cache[kCacheGroups];
     pdl_launch_dependents();
     pdl_wait();                 // earlier kernels of the stream may still be reading the index buffers
     const uint32_t b = blockIdx.x;
@@ -68,6 +71,22 @@ sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint
         if (b == 0) keep_offsets[0] = 0;
     }
 
+    const bool cached = groups <= kCacheGroups && K < N;
+    if (cached) {
+        for (uint32_t q = threadIdx.x; q < groups; q += kSampThreads) {
+            const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+            word_cache[q] = make_uint4(pw.w[0], pw.w[1], pw.w[2], pw.w[3]);
+        }
+        __syncthreads();
+    }
+    auto words_of = [&](uint32_t q) {
+        if (!cached) return position_words(q, gid, step, k0, k1);
+        const uint4 v = word_cache[q];
+        PhiloxWords pw;
+        pw.w[0] = v.x; pw.w[1] = v.y; pw.w[2] = v.z; pw.w[3] = v.w;
+        return pw;
+    };
+
     // ---- radix select: threshold word `prefix` and how many positions equal to it are kept ----
     uint32_t prefix = 0, known = 0, remaining = K;
     if (K < N) {
@@ -75,7 +94,7 @@ sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint
             for (int i = threadIdx.x; i < 256; i += kSampThreads) sh.hist[i] = 0;
             __syncthreads();
             for (uint32_t q = threadIdx.x; q < groups; q += kSampThreads) {
-                const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+                const PhiloxWords pw = words_of(q);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const uint32_t n = 4u * q + e;
@@ -110,7 +129,7 @@ sample_keep_random_kernel(uint32_t N, uint32_t K, uint32_t k0, uint32_t k1, uint
 #pragma unroll
                 for (int e = 0; e < 4; ++e) if (4u * q + e < N) lt_mask |= 1u << e;
             } else {
-                const PhiloxWords pw = position_words(q, gid, step, k0, k1);
+                const PhiloxWords pw = words_of(q);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     if (4u * q + e < N) {
