@@ -162,7 +162,8 @@ sbp_status sbp_linear_forward(sbp_dtype dt, const void* X /* dev */, const void*
                               void* X_keep /* dev, nullable */, uint32_t flags,
                               int32_t* status_word /* dev, nullable */, void* stream);
 
-/* Scratch bytes sbp_linear_backward needs for these sizes (never 0). */
+/* Scratch bytes sbp_linear_backward needs for these sizes, whatever flags the call uses (never 0):
+ * partial sums of split reductions, and room for one copy of W and of dW for SBP_FLAG_W_OUT_IN. */
 size_t sbp_linear_backward_workspace_bytes(sbp_dtype dt, int64_t M, int64_t M_keep_cap,
                                            int64_t C_in, int64_t C_out);
 
