@@ -9,6 +9,7 @@
  *
  *   sbp_sample_keep      draw the kept positions of every sample      (Sec. 3.2.1, Sec. 4)
  *   sbp_forward_cache    X_keep = X[keep_rows, :]                     (Algorithm 1)
+ *   sbp_linear_forward   Y = X W + b, with that cache written by the same launch (Eq. 2)
  *   sbp_linear_backward  dW = X_keep^T dY_keep, db = sum dY_keep,
  *                        dX = scatter(dY_keep W^T), zeros elsewhere   (Eq. 5)
  *
@@ -17,7 +18,7 @@
  * Conventions
  *   - M = B*N rows, N = H*W positions per sample, row id = b*N + h*W + w.
  *   - All matrices are row-major, dense (no padding), inner stride 1.
- *     W is [C_in, C_out] (the paper's orientation, Y = X W).
+ *     W is [C_in, C_out] (the paper's orientation, Y = X W) unless SBP_FLAG_W_OUT_IN says otherwise.
  *   - "dev" pointers are CUDA device pointers owned by the caller; the library
  *     allocates and frees nothing and keeps no pointer after a call returns.
  *     Device buffers must be 16-byte aligned.
