@@ -231,6 +231,14 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
                                      uint32_t flags);
 
 /*
+ * Diagnostic (pure host function; no counterpart in the paper): how many times this process has
+ * searched for the cut of the weight-gradient reduction of a layer shape.  The answer for a shape
+ * is remembered for the life of the process, so the count stops growing once every shape of a
+ * model has been seen: neither sbp_linear_backward nor the workspace-size query repeats a search.
+ */
+int64_t sbp_plan_search_count(void);
+
+/*
  * One whole SBP step of a layer for callers whose tensors live in HOST memory: copies X, dY, W
  * to the device, draws the keep set (Sec. 4), builds the forward cache (Algorithm 1), runs the
  * backward (Eq. 5) and copies dW, db, dX (and optionally the indices) back, all enqueued on

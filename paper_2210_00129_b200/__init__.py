@@ -26,7 +26,8 @@ SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT, SBP_FLAG_W_OUT_IN = 16, 32, 64
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
-           "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static", "sbp_selftest_bounded_wait")
+           "sbp_plan_search_count", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
+           "sbp_selftest_bounded_wait")
 
 _lib = None
 
@@ -66,6 +67,8 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_linear_backward.restype = ci
     lib.sbp_linear_backward_kernel_count.argtypes = [ci, i64, i64, i64, i64, ci, ci, ci, u32]
     lib.sbp_linear_backward_kernel_count.restype = ci
+    lib.sbp_plan_search_count.argtypes = []
+    lib.sbp_plan_search_count.restype = i64
     lib.sbp_step_host_arena_bytes.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl]
     lib.sbp_step_host_arena_bytes.restype = sz
     lib.sbp_step_host.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl, u64, u64, i64, u32,
@@ -155,6 +158,10 @@ def sbp_linear_backward_kernel_count(dt, M, M_keep_cap, C_in, C_out, want_dW=Tru
                                      flags=0) -> int:
     return int(load_library().sbp_linear_backward_kernel_count(dt, M, M_keep_cap, C_in, C_out, int(want_dW),
                                                                int(want_db), int(want_dX), flags))
+
+
+def sbp_plan_search_count() -> int:
+    return int(load_library().sbp_plan_search_count())
 
 
 def sbp_step_host_arena_bytes(dt, mode, B, H, W, C_in, C_out, keep_ratio) -> int:

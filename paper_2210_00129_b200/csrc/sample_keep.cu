@@ -504,9 +504,8 @@ template <int C>
 cudaError_t launch_cluster_sampler(dim3 grid, dim3 block, size_t cache_bytes, cudaStream_t stream, int64_t N, int64_t K,
                                    uint32_t k0, uint32_t k1, uint32_t step, uint32_t first_sample, bool share_mask,
                                    int32_t* keep_rows, int32_t* keep_offsets) {
-    static cudaError_t once = cudaFuncSetAttribute(sample_keep_random_cluster_kernel<C>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterCacheMax);
-    if (once != cudaSuccess) return once;
+    const cudaError_t opt = opt_in_dynamic_smem<sample_keep_random_cluster_kernel<C>>((int)kClusterCacheMax);
+    if (opt != cudaSuccess) return opt;
     return launch_pdl_cluster(sample_keep_random_cluster_kernel<C>, grid, block, cache_bytes, C, stream, (uint32_t)N,
                               (uint32_t)K, k0, k1, step, first_sample, share_mask ? 1 : 0, cache_bytes ? 1 : 0, keep_rows,
                               keep_offsets);

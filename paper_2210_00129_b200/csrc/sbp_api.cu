@@ -329,6 +329,8 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
     return n;
 }
 
+int64_t sbp_plan_search_count(void) { return tc_plan_searches(); }
+
 namespace {
 struct StepArena {
     size_t X, dY, W, rows, offs, Xk, dW, db, dX, status, ws, ws_bytes, total;

@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/sbp.h"
 
 namespace sbp {
@@ -41,6 +43,25 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+// Opt a kernel in to more than 48 KB of dynamic shared memory.  The attribute belongs to the (kernel, device) pair,
+// so it is set once per device a process launches the kernel on, not once per process.
+constexpr int kMaxDevices = 64;
+template <auto Kernel>
+inline cudaError_t opt_in_dynamic_smem(int bytes) {
+    static std::mutex mu;
+    static bool done[kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!done[dev]) {
+        e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    return cudaSuccess;
 }
 // the same with thread-block clusters of `cluster_x` CTAs along x
 template <typename... KArgs, typename... Args>
@@ -169,6 +190,7 @@ sbp_status launch_tc_forward(const void* X, const void* W, bool w_out_in, const 
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
+int64_t tc_plan_searches();              // split-plan searches run so far in this process
 int    tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx,
                                 bool want_db);
 // dW (nullable) and dX (nullable) of one layer in a single persistent kernel (+ the split reduce); when db is

@@ -26,7 +26,9 @@
 // and leave one partial row per block for a fixed-order reduce.  The row maps are compile-time
 // variants: keep_rows on both sides, or identity on either side for gradients kept packed between
 // chained layers (Sec. 3.3.1).
+#include <map>
 #include <mutex>
+#include <tuple>
 
 #include "tc_ptx.cuh"
 
@@ -751,6 +753,15 @@ double estimate_cost(int64_t x_tiles, int64_t x_kb, int64_t w_tiles, int64_t w_k
     return worst;
 }
 
+struct PlanKey {
+    int64_t cap, ci, co;
+    bool dx;
+    bool operator<(const PlanKey& o) const { return std::tie(cap, ci, co, dx) < std::tie(o.cap, o.ci, o.co, o.dx); }
+};
+std::mutex g_plan_mutex;
+std::map<PlanKey, int> g_plan_memo;
+int64_t g_plan_searches = 0;
+
 Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
     Plan pl;
     pl.bnx = (C_in >= 256) ? 256 : 128;
@@ -761,20 +772,17 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
     pl.splits = 1;
     if (want_dw) {
-        // the same answer for the same shape: remember the last few shapes instead of searching on every call
-        struct Memo { int64_t cap, ci, co; int flags, splits; };
-        static Memo memo[8];
-        static int memo_next = 0;
-        static std::mutex memo_mutex;
-        const int flags = want_dx ? 1 : 0;
+        // The same answer for the same shape: every shape a process has asked about is remembered (a few
+        // dozen bytes per layer shape, never evicted), so a model's layers do not push each other out.
+        const PlanKey key{M_keep_cap, C_in, C_out, want_dx};
         bool known = false;
         {
-            std::lock_guard<std::mutex> lock(memo_mutex);
-            for (const Memo& m : memo)
-                if (m.splits > 0 && m.cap == M_keep_cap && m.ci == C_in && m.co == C_out && m.flags == flags) {
-                    pl.splits = m.splits;
-                    known = true;
-                }
+            std::lock_guard<std::mutex> lock(g_plan_mutex);
+            const auto it = g_plan_memo.find(key);
+            if (it != g_plan_memo.end()) {
+                pl.splits = it->second;
+                known = true;
+            }
         }
         if (!known) {
             int64_t max_s = w_kb < 64 ? w_kb : 64;
@@ -786,9 +794,9 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
                 const double c = estimate_cost(x_tiles, x_kb, w_tiles, w_kb, sp, C_in * C_out);
                 if (sp == 1 || c < best * 0.995) { best = c; pl.splits = (int)sp; }
             }
-            std::lock_guard<std::mutex> lock(memo_mutex);
-            memo[memo_next] = Memo{M_keep_cap, C_in, C_out, flags, pl.splits};
-            memo_next = (memo_next + 1) % 8;
+            std::lock_guard<std::mutex> lock(g_plan_mutex);
+            g_plan_memo[key] = pl.splits;
+            ++g_plan_searches;
         }
     }
     pl.tiles = x_tiles + w_tiles * pl.splits;
@@ -798,9 +806,8 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
 template <int BNX, int BNW, int DEPTH, bool PACKED>
 cudaError_t launch_fused_variant(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
                                  const CUtensorMap& map_dw, const TcParams& prm) {
-    static cudaError_t once = cudaFuncSetAttribute(tc_backward_kernel<BNX, BNW, DEPTH, PACKED>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (once != cudaSuccess) return once;
+    const cudaError_t opt = opt_in_dynamic_smem<tc_backward_kernel<BNX, BNW, DEPTH, PACKED>>((int)kSmemBytes);
+    if (opt != cudaSuccess) return opt;
     return launch_pdl(tc_backward_kernel<BNX, BNW, DEPTH, PACKED>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x,
                       map_dw, prm);
 }
@@ -821,6 +828,11 @@ cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_
 }
 
 }  // namespace
+
+int64_t tc_plan_searches() {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    return g_plan_searches;
+}
 
 bool tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out) {
     // every TMA box (64 columns x up to 128/256 rows) must fit inside its matrix

@@ -306,9 +306,8 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, ui
 template <int BN>
 cudaError_t launch_forward(dim3 grid, cudaStream_t stream, const CUtensorMap& map_x, const CUtensorMap& map_w,
                            const FwdParams& prm) {
-    static cudaError_t once = cudaFuncSetAttribute(tc_forward_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)kSmemBytes);
-    if (once != cudaSuccess) return once;
+    const cudaError_t opt = opt_in_dynamic_smem<tc_forward_kernel<BN>>((int)kSmemBytes);
+    if (opt != cudaSuccess) return opt;
     return launch_pdl(tc_forward_kernel<BN>, grid, dim3(kFwdThreads), kSmemBytes, stream, map_x, map_w, prm);
 }
 

@@ -92,6 +92,23 @@ def test_workspace_query_grows_with_the_problem(lib):
     assert sbp.sbp_linear_backward_workspace_bytes(1, 0, 0, 0, 0) == 256
 
 
+def test_split_plans_are_searched_once_per_shape(lib):
+    # more layer shapes than any small cache would hold (ConvNeXt-B alone has eight point-wise shapes):
+    # the second round of queries must not search again
+    shapes = [(64 * hw * hw, d_in, d_out) for d, hw in ((128, 56), (256, 28), (512, 14), (1024, 7), (192, 28))
+              for d_in, d_out in ((d, 4 * d), (4 * d, d))]
+    assert len(shapes) == 10
+    for M, ci, co in shapes:
+        sbp.sbp_linear_backward_workspace_bytes(1, M, M // 2, ci, co)
+    seen = sbp.sbp_plan_search_count()
+    assert seen >= len(shapes)
+    for _ in range(3):
+        for M, ci, co in shapes:
+            sbp.sbp_linear_backward_workspace_bytes(1, M, M // 2, ci, co)
+            sbp.sbp_linear_backward_kernel_count(1, M, M // 2, ci, co)
+    assert sbp.sbp_plan_search_count() == seen
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(sbp, "_lib", None)
     monkeypatch.setattr(sbp, "LIB_PATH", str(tmp_path / "nope.so"))

@@ -285,6 +285,46 @@ def test_grid_phase_is_fresh_per_step_and_sample():
     assert firsts == {0, 1}
 
 
+def test_grid_phase_is_the_stated_philox_word():
+    """The phase rule: p = Philox4x32-10({0, g, step, 1}, seed)[0] mod #phases, with g the global sample id.
+    Recomputed here with the independent big-integer Philox; another counter word, tag or output lane fails."""
+    H, W, N = 6, 4, 24
+    for seed, step, offset in [(0, 0, 0), (3, 17, 5), (0xDEADBEEF12345678, 2 ** 32 - 1, 2 ** 31), (9, 1, 2 ** 32 - 4)]:
+        key = [seed & M32, seed >> 32]
+        B = 4
+        for r, phases in ((0.25, 4), (0.5, 2), (0.75, 4)):
+            rows, offs = oracle.sample_keep(oracle.MASK_GRID, B, H, W, r, seed=seed, step=step, sample_offset=offset)
+            for b in range(B):
+                p = _philox_bigint([0, (offset + b) & M32, step, 1], key)[0] % phases
+                if r == 0.5:
+                    want = [n for n in range(N) if ((n // W + n % W) & 1) == p]
+                else:
+                    hit = [n for n in range(N) if ((n // W) & 1, (n % W) & 1) == (p >> 1, p & 1)]
+                    want = hit if r == 0.25 else [n for n in range(N) if n not in hit]
+                got = (rows[offs[b]:offs[b + 1]] - b * N).tolist()
+                assert got == want, (seed, step, offset, r, b)
+    # one mask for the whole call: every sample takes global sample 0's phase
+    rows, offs = oracle.sample_keep(oracle.MASK_GRID, 3, H, W, 0.5, seed=5, step=2, sample_offset=7,
+                                    flags=oracle.FLAG_SHARE_MASK)
+    p = _philox_bigint([0, 0, 2, 1], [5, 0])[0] % 2
+    for b in range(3):
+        assert (rows[offs[b]:offs[b + 1]] - b * N).tolist() == [n for n in range(N) if ((n // W + n % W) & 1) == p]
+
+
+def test_temporal_grid_phase_is_the_same_philox_word():
+    T, Wf = 9, 2
+    for seed, step, offset in [(1, 0, 0), (77, 5, 3)]:
+        key = [seed & M32, seed >> 32]
+        for r, period in ((0.25, 4), (0.5, 2), (0.75, 4)):
+            rows, offs = oracle.sample_keep(oracle.MASK_TEMPORAL_GRID, 3, T, Wf, r, seed=seed, step=step,
+                                            sample_offset=offset)
+            for b in range(3):
+                p = _philox_bigint([0, offset + b, step, 1], key)[0] % period
+                frames = [f for f in range(T) if ((f % period == p) != (r == 0.75))]
+                want = [f * Wf + q for f in frames for q in range(Wf)]
+                assert (rows[offs[b]:offs[b + 1]] - b * T * Wf).tolist() == want, (seed, r, b)
+
+
 def test_sampler_rejects_out_of_domain():
     with pytest.raises(ValueError):
         oracle.sample_keep(oracle.MASK_RANDOM, 1, 4, 4, 0.5, step=2 ** 32)
