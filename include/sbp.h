@@ -247,8 +247,8 @@ int64_t sbp_plan_search_count(void);
  *
  * X_host [B*H*W, C_in], dY_host [B*H*W, C_out], W_host [C_in, C_out]: element type dt.
  * dW_host [C_in, C_out] fp32, db_host [C_out] fp32, dX_host [B*H*W, C_in] dt.
- * keep_rows_host (nullable, capacity B * sbp_keep_count(...)), keep_offsets_host (nullable,
- * B + 1 entries), status_host (nullable, one int32: the device status word of the step).
+ * keep_rows_host (nullable, capacity B * sbp_keep_count(...); entries past keep_offsets[B] are
+ * unspecified), keep_offsets_host (nullable, B + 1 entries), status_host (nullable, one int32: the device status word of the step).
  * arena (dev): caller-owned scratch of at least sbp_step_host_arena_bytes(...) bytes, 256-byte
  * aligned; holds the device copies of every tensor during the step.  Nothing is allocated.
  * flags: SBP_FLAG_SHARE_MASK, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA (accumulation is not offered).

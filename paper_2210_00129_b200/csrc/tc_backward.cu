@@ -95,6 +95,9 @@ struct TcParams {
     int db_from_mma;               // narrow layers: db comes out of the dW tiles (a column of ones appended to X_keep);
                                    // db_partial is then [dw_splits, C_out]
     float* db_partial;             // nullptr: no bias sums; else [gridDim.x, C_out] per-CTA column sums of kept dY rows
+    int dw_ctas;                   // 0: every block walks the one cost-sorted list of both tile kinds; > 0: the first
+                                   // dw_ctas blocks take the dW pieces, the others the dX tiles, both sweeping the kept
+                                   // rows in the same order (memory-bound layers: see next_tile)
     int32_t* status_word;
 };
 
@@ -105,6 +108,8 @@ struct Schedule {
     uint32_t splits;
     bool w_first;                                     // the costlier kind is handed out first
     uint32_t total;
+    uint32_t dw_ctas;                                 // role split (see next_tile); 0 = one list for all blocks
+    uint32_t x_rtiles, slab_len, slab_full;           // dX row tiles; row tiles per slab (the first slab_full slabs have one more)
 };
 struct Tile {
     bool is_dw;
@@ -125,6 +130,10 @@ __device__ __forceinline__ Schedule make_schedule(const TcParams& p, int64_t M_k
     s.w_kb_per = (s.w_kb_total + s.splits - 1) / s.splits;
     s.w_first = s.w_kb_per >= s.x_kb;
     s.total = s.x_tiles + s.w_tiles;
+    s.dw_ctas = (p.dw_ctas > 0 && s.x_tiles > 0 && s.w_tiles > 0 && (uint32_t)p.dw_ctas < gridDim.x) ? (uint32_t)p.dw_ctas : 0u;
+    s.x_rtiles = s.x_ntiles ? s.x_tiles / s.x_ntiles : 0u;
+    s.slab_len = s.x_rtiles / s.splits;               // slab z holds slab_len (+1 for z < slab_full) consecutive row tiles
+    s.slab_full = s.x_rtiles % s.splits;
     return s;
 }
 
@@ -156,6 +165,42 @@ __device__ __forceinline__ Tile decode_tile(const Schedule& s, uint32_t q) {
 __device__ __forceinline__ uint32_t list_position(uint32_t pass) {
     const uint32_t G = gridDim.x, b = blockIdx.x;
     return pass * G + ((pass & 1u) ? (G - 1u - b) : b);
+}
+
+// The tile a block works on in its pass-th round, false when it has none left.
+// One list (dw_ctas == 0): the cost-sorted list of both kinds, dealt out as list_position says.
+// Role split (memory-bound layers): blocks [0, dw_ctas) take the dW pieces - piece `split` reduces over the split-th
+// slab of kept rows - and the other blocks take the dX tiles in slab-interleaved order (first row tile of every slab,
+// then the second of every slab, ...).  Both groups then move through every slab of kept rows from its start to its
+// end at the same time, so each kept row of dY comes from DRAM once: whichever product reaches a row second finds
+// it in L2 (and, being served from L2, catches up with the other).
+__device__ __forceinline__ bool next_tile(const Schedule& s, uint32_t pass, Tile& t) {
+    if (s.dw_ctas == 0u) {
+        const uint32_t q = list_position(pass);
+        if (q >= s.total) return false;
+        t = decode_tile(s, q);
+        return true;
+    }
+    const uint32_t b = blockIdx.x;
+    if (b < s.dw_ctas) {
+        const uint32_t q = b + pass * s.dw_ctas;
+        if (q >= s.w_tiles) return false;
+        t = decode_tile(s, s.w_first ? q : s.x_tiles + q);
+        return true;
+    }
+    const uint32_t q = (b - s.dw_ctas) + pass * (gridDim.x - s.dw_ctas);
+    if (q >= s.x_tiles) return false;
+    const uint32_t tr = q / s.x_ntiles;               // position of the row tile in the interleaved order
+    const uint32_t lim = s.slab_len * s.splits;       // positions below this: every slab still has a tile at this depth
+    const uint32_t depth = tr < lim ? tr / s.splits : s.slab_len;
+    const uint32_t slab = tr < lim ? tr % s.splits : tr - lim;
+    t.is_dw = false;
+    t.split = 0;
+    t.row_tile = slab * s.slab_len + (slab < s.slab_full ? slab : s.slab_full) + depth;
+    t.col_tile = q % s.x_ntiles;
+    t.kb_begin = 0;
+    t.num_kb = s.x_kb;
+    return true;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -293,9 +338,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             uint32_t it = 0;                                         // stage uses so far, over all tiles
             bool ok = true;
             for (uint32_t pass = 0; ok; ++pass) {
-                const uint32_t q = list_position(pass);
-                if (q >= sched.total) break;
-                const Tile t = decode_tile(sched, q);
+                Tile t;
+                if (!next_tile(sched, pass, t)) break;
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
                     const int s = it % kS;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kS) & 1u) ^ 1u, abort_flag, status_word);
@@ -329,9 +373,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             uint32_t it = 0, used = 0;                               // stage uses, accumulator uses
             bool ok = true;
             for (uint32_t pass = 0; ok; ++pass) {
-                const uint32_t q = list_position(pass);
-                if (q >= sched.total) break;
-                const Tile t = decode_tile(sched, q);
+                Tile t;
+                if (!next_tile(sched, pass, t)) break;
                 if (t.num_kb == 0) continue;
                 const uint32_t acc = used & 1u;
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[acc]), ((used >> 1) & 1u) ^ 1u, abort_flag, status_word);
@@ -376,9 +419,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         uint32_t it = 0;
         bool ok = true;
         for (uint32_t pass = 0; ok; ++pass) {
-            const uint32_t q = list_position(pass);
-            if (q >= sched.total) break;
-            const Tile t = decode_tile(sched, q);
+            Tile t;
+            if (!next_tile(sched, pass, t)) break;
             if (!t.is_dw) {
                 // dX tile: 128 kept rows x 128 bytes per stage; one warp instruction moves 4 rows x 128 B
                 constexpr int kInstr = 32 / kGatherWarps;
@@ -462,9 +504,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         // ---------------- side warps: zeros for the dropped rows of dX, then the bias sums ----------------
         if (p.dX != nullptr && M_keep > 0) {
             for (uint32_t pass = 0;; ++pass) {
-                const uint32_t q = list_position(pass);
-                if (q >= sched.total) break;
-                const Tile t = decode_tile(sched, q);
+                Tile t;
+                if (!next_tile(sched, pass, t)) break;
                 if (!t.is_dw) zero_dropped_rows<BNX, kPacked>(p, t, M_keep, warp - kBiasWarp0, lane);
             }
         }
@@ -540,9 +581,8 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         uint32_t used = 0, staged = 0;                               // accumulator uses, staging-buffer uses
         bool ok = true;
         for (uint32_t pass = 0; ok; ++pass) {
-            const uint32_t q = list_position(pass);
-            if (q >= sched.total) break;
-            const Tile t = decode_tile(sched, q);
+            Tile t;
+            if (!next_tile(sched, pass, t)) break;
             const uint32_t acc = used & 1u;
             const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
             if (!t.is_dw) {
@@ -710,6 +750,7 @@ bool make_map_dw(CUtensorMap* map, const float* base, int64_t splits, int64_t C_
 struct Plan {
     int bnx, bnw;          // accumulator width of dX / dW tiles
     int splits;            // pieces each dW tile's reduction over kept rows is cut into
+    int dw_ctas;           // role split: blocks given to the dW pieces (0 = one list for all blocks)
     int64_t tiles;         // upper bound of the tile count (from the capacity)
 };
 
@@ -759,7 +800,8 @@ struct PlanKey {
     bool operator<(const PlanKey& o) const { return std::tie(cap, ci, co, dx) < std::tie(o.cap, o.ci, o.co, o.dx); }
 };
 std::mutex g_plan_mutex;
-std::map<PlanKey, int> g_plan_memo;
+struct PlanChoice { int splits, dw_ctas; };
+std::map<PlanKey, PlanChoice> g_plan_memo;
 int64_t g_plan_searches = 0;
 
 Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx) {
@@ -771,6 +813,7 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     const int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
     const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
     pl.splits = 1;
+    pl.dw_ctas = 0;
     if (want_dw) {
         // The same answer for the same shape: every shape a process has asked about is remembered (a few
         // dozen bytes per layer shape, never evicted), so a model's layers do not push each other out.
@@ -780,22 +823,48 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
             std::lock_guard<std::mutex> lock(g_plan_mutex);
             const auto it = g_plan_memo.find(key);
             if (it != g_plan_memo.end()) {
-                pl.splits = it->second;
+                pl.splits = it->second.splits;
+                pl.dw_ctas = it->second.dw_ctas;
                 known = true;
             }
         }
         if (!known) {
-            int64_t max_s = w_kb < 64 ? w_kb : 64;
-            if (max_s < 1) max_s = 1;
-            // the search walks every tile: with very many tiles any cut balances, so bound the work
-            while (max_s > 1 && (x_tiles + w_tiles * max_s) * max_s > (1 << 22)) max_s /= 2;
-            double best = 0.0;
-            for (int64_t sp = 1; sp <= max_s; ++sp) {
-                const double c = estimate_cost(x_tiles, x_kb, w_tiles, w_kb, sp, C_in * C_out);
-                if (sp == 1 || c < best * 0.995) { best = c; pl.splits = (int)sp; }
+            // Memory-bound layers (thin ConvNeXt stages, the detection map) with both products: split the blocks
+            // into a dW group and a dX group that sweep the kept rows together (see next_tile), so that DRAM sees
+            // each kept row of dY once.  The groups are sized by the bytes each has to pull into its SMs: the
+            // gathered rows of dY and the dense operand once per tile, plus the dX rows written (the row count of
+            // dX is not known here; twice the kept rows is assumed, the paper's usual keep ratio).
+            const double t_flop = 4.0 * (double)M_keep_cap * (double)C_in * (double)C_out / 1.4e15;
+            const double t_mem = 2.0 * (double)M_keep_cap * (double)(2 * C_in + C_out) / 6.5e12;
+            bool role_split = false;
+            if (want_dx && t_mem >= 0.75 * t_flop && w_tiles > 0 && w_tiles <= kNumSMs / 4) {
+                const double dy = 2.0 * (double)M_keep_cap * (double)C_out, xk = 2.0 * (double)M_keep_cap * (double)C_in;
+                const double w_cols = (double)((C_in + pl.bnw - 1) / pl.bnw), w_rows = (double)((C_out + kBM - 1) / kBM);
+                const double bytes_w = dy * w_cols + xk * w_rows;
+                const double x_cols = (double)((C_in + pl.bnx - 1) / pl.bnx);
+                const double bytes_x = dy * x_cols + (double)x_tiles * (double)pl.bnx * (double)C_out * 2.0 + 2.0 * xk;
+                const double target = bytes_w / (bytes_w + bytes_x) * (double)kNumSMs;
+                int64_t sp = (int64_t)(target / (double)w_tiles + 0.5);
+                const int64_t x_rtiles = (M_keep_cap + kBM - 1) / kBM;
+                if (sp >= 2 && w_kb / sp >= 8 && x_rtiles >= sp && w_tiles * sp <= kNumSMs - 16) {
+                    pl.splits = (int)sp;
+                    pl.dw_ctas = (int)(w_tiles * sp);
+                    role_split = true;
+                }
+            }
+            if (!role_split) {
+                int64_t max_s = w_kb < 64 ? w_kb : 64;
+                if (max_s < 1) max_s = 1;
+                // the search walks every tile: with very many tiles any cut balances, so bound the work
+                while (max_s > 1 && (x_tiles + w_tiles * max_s) * max_s > (1 << 22)) max_s /= 2;
+                double best = 0.0;
+                for (int64_t sp = 1; sp <= max_s; ++sp) {
+                    const double c = estimate_cost(x_tiles, x_kb, w_tiles, w_kb, sp, C_in * C_out);
+                    if (sp == 1 || c < best * 0.995) { best = c; pl.splits = (int)sp; }
+                }
             }
             std::lock_guard<std::mutex> lock(g_plan_mutex);
-            g_plan_memo[key] = pl.splits;
+            g_plan_memo[key] = PlanChoice{pl.splits, pl.dw_ctas};
             ++g_plan_searches;
         }
     }
@@ -894,6 +963,7 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     prm.db_from_mma = db_from_mma ? 1 : 0;
     const int db_rows = db_from_mma ? pl.splits : 0;                 // 0: one row per block (set below)
     prm.status_word = status_word;
+    prm.dw_ctas = pl.dw_ctas;
     int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
     if (ctas < 1) ctas = 1;
     const dim3 grid((unsigned)ctas);
