@@ -61,6 +61,12 @@ def _load():
     lib.oracle_full_backward.restype = None
     lib.oracle_linear_forward.argtypes = [vp, vp, vp, i64, i64, i64, vp]
     lib.oracle_linear_forward.restype = None
+    lib.oracle_attention_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
+    lib.oracle_attention_forward.restype = None
+    lib.oracle_attention_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp]
+    lib.oracle_attention_backward.restype = None
+    lib.oracle_attention_memory_ratio.argtypes = [ctypes.c_int, dbl, dbl, dbl]
+    lib.oracle_attention_memory_ratio.restype = dbl
     lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
     lib.oracle_set_num_threads.restype = None
     lib.oracle_num_threads.argtypes = []
@@ -165,3 +171,40 @@ def full_backward(X, dY, W, want=("dW", "db", "dX")):
     _load().oracle_full_backward(_ptr(X), _ptr(dY), _ptr(W), M, C_in, C_out,
                                  _ptr(dW), _ptr(db), _ptr(dX))
     return {k: v for k, v in (("dW", dW), ("db", db), ("dX", dX)) if v is not None}
+
+
+ATTN_DROP_QUERY = 0
+ATTN_DROP_QKV = 1
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def attention_forward(Q, K, V, q_rows, q_offs, k_rows, k_offs, heads):
+    """Attention output A [M, heads*d] in fp64 for queries in the q lists against keys in the k lists
+    (per-sample lists of global row ids with their offsets); rows outside the q lists are zero."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    M, C = Q.shape
+    d = C // heads
+    qr, qo, kr, ko = _i32(q_rows), _i32(q_offs), _i32(k_rows), _i32(k_offs)
+    A = np.empty((M, C))
+    _load().oracle_attention_forward(_ptr(Q), _ptr(K), _ptr(V), _ptr(qr), _ptr(qo), _ptr(kr), _ptr(ko),
+                                     len(qo) - 1, M, heads, d, _ptr(A))
+    return A
+
+
+def attention_backward(Q, K, V, dA, q_rows, q_offs, k_rows, k_offs, heads):
+    """(dQ, dK, dV), each [M, heads*d] in fp64, zero outside the chosen token lists."""
+    Q, K, V, dA = _f64(Q), _f64(K), _f64(V), _f64(dA)
+    M, C = Q.shape
+    d = C // heads
+    qr, qo, kr, ko = _i32(q_rows), _i32(q_offs), _i32(k_rows), _i32(k_offs)
+    dQ, dK, dV = np.empty((M, C)), np.empty((M, C)), np.empty((M, C))
+    _load().oracle_attention_backward(_ptr(Q), _ptr(K), _ptr(V), _ptr(dA), _ptr(qr), _ptr(qo), _ptr(kr), _ptr(ko),
+                                      len(qo) - 1, M, heads, d, _ptr(dQ), _ptr(dK), _ptr(dV))
+    return dQ, dK, dV
+
+
+def attention_memory_ratio(mode: int, d: float, n: float, r: float) -> float:
+    return float(_load().oracle_attention_memory_ratio(mode, float(d), float(n), float(r)))

@@ -15,6 +15,8 @@
  *   - dW, dX of a linear / point-wise layer under SBP:  Eq. 5 and the text after it
  *   - full backward for the invariants:                 Eq. 3
  *   - no gradient rescaling:                            Eq. 1
+ *   - attention with the gradient kept on token subsets: Sec. 4 ("How to apply SBP on MHSA?"), Supp.
+ *                                                       "Gradient Calculation of Attention Layers"
  * The paper names no random generator; the sampler uses Philox4x32-10
  * (Salmon, Moraes, Dror, Shaw: "Parallel Random Numbers: As Easy as 1, 2, 3",
  * SC'11), written here from that paper's definition of the round function.
@@ -22,7 +24,9 @@
  * Parity pins: every function here is pinned by tests that do not call it to
  * check itself (published Philox known answers, brute-force selection, hand
  * computed integer cases, reduction to library matrix products, enumeration
- * of all masks).  Nothing in this file is "parity unpinned".
+ * of all masks; for the attention functions: central differences of the forward,
+ * the full backward written as matrix products, the paper's exact-on-kept-rows
+ * statement and its printed memory ratios).  Nothing in this file is "parity unpinned".
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -417,4 +421,131 @@ int oracle_num_threads(void)
 #else
     return 1;
 #endif
+}
+
+/* ------------------------------------------------------------------ */
+/* SBP on multi-head self-attention (Sec. 4, "How to apply SBP on MHSA?";   */
+/* Supp. "Gradient Calculation of Attention Layers")                   */
+/* ------------------------------------------------------------------ */
+/*
+ * One head of one sample, with the gradient path restricted to a set Zq of query tokens and a set Zk
+ * of key / value tokens (both given as per-sample lists of global row ids, as the sampler writes them):
+ *
+ *   forward (the supplementary's attention equation on the chosen tokens):
+ *     M_ij = q_i . k_j / sqrt(d)      i in Zq, j in Zk
+ *     S_i: = softmax_j(M_i:)          over j in Zk
+ *     A_i  = sum_j S_ij v_j
+ *   backward (the supplementary's gradients of query, key and value, dQ = dM K / sqrt(d),
+ *   dK = Q^T dM / sqrt(d), dV = S^T dA, with the derivative of the row softmax between dS and dM):
+ *     dS_ij = dA_i . v_j
+ *     dM_ij = S_ij (dS_ij - sum_l S_il dS_il)
+ *     dQ_i  = sum_j dM_ij k_j / sqrt(d);  dK_j = sum_i dM_ij q_i / sqrt(d);  dV_j = sum_i S_ij dA_i
+ *   rows outside Zq (dQ) or Zk (dK, dV) receive +0.0: their gradient is dropped.
+ *
+ * Zq = kept tokens, Zk = all tokens is the paper's "Drop Query only" (its worked derivation: dM of the
+ * dropped queries is zero, dQ is exact on the kept rows, dK = Q_keep^T dM_keep / sqrt(d)); Zq = Zk = kept
+ * tokens is "Drop QKV", read as attention among the kept tokens (the reading of Algorithm 1 applied to the
+ * attention operation, whose cached maps are the r^2 n^2 ones of the paper's memory formula); Zq = Zk = all
+ * tokens is ordinary attention.  Matrices are [M, heads * d] row-major, head hh in columns [hh*d, (hh+1)*d).
+ */
+void oracle_attention_forward(const double* Q, const double* K, const double* V,
+                              const int32_t* q_rows, const int32_t* q_offs,
+                              const int32_t* k_rows, const int32_t* k_offs,
+                              int64_t B, int64_t M, int64_t heads, int64_t d, double* A)
+{
+    const int64_t C = heads * d;
+    const double scale = 1.0 / sqrt((double)d);
+    for (int64_t e = 0; e < M * C; ++e) A[e] = 0.0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t hh = 0; hh < heads; ++hh) {
+            const int64_t nk = k_offs[b + 1] - k_offs[b];
+            double* s = (double*)malloc(sizeof(double) * (size_t)(nk > 0 ? nk : 1));
+            for (int64_t a = q_offs[b]; a < q_offs[b + 1]; ++a) {
+                const double* q = Q + (int64_t)q_rows[a] * C + hh * d;
+                double mx = -INFINITY;
+                for (int64_t j = 0; j < nk; ++j) {
+                    const double* k = K + (int64_t)k_rows[k_offs[b] + j] * C + hh * d;
+                    double acc = 0.0;
+                    for (int64_t c = 0; c < d; ++c) acc += q[c] * k[c];
+                    s[j] = acc * scale;
+                    if (s[j] > mx) mx = s[j];
+                }
+                double sum = 0.0;
+                for (int64_t j = 0; j < nk; ++j) { s[j] = exp(s[j] - mx); sum += s[j]; }
+                double* out = A + (int64_t)q_rows[a] * C + hh * d;
+                for (int64_t j = 0; j < nk; ++j) {
+                    const double* v = V + (int64_t)k_rows[k_offs[b] + j] * C + hh * d;
+                    const double p = s[j] / sum;
+                    for (int64_t c = 0; c < d; ++c) out[c] += p * v[c];
+                }
+            }
+            free(s);
+        }
+}
+
+void oracle_attention_backward(const double* Q, const double* K, const double* V, const double* dA,
+                               const int32_t* q_rows, const int32_t* q_offs,
+                               const int32_t* k_rows, const int32_t* k_offs,
+                               int64_t B, int64_t M, int64_t heads, int64_t d,
+                               double* dQ, double* dK, double* dV)
+{
+    const int64_t C = heads * d;
+    const double scale = 1.0 / sqrt((double)d);
+    for (int64_t e = 0; e < M * C; ++e) { dQ[e] = 0.0; dK[e] = 0.0; dV[e] = 0.0; }
+    /* one (sample, head) pair touches only its own rows and columns: the pairs are independent */
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t hh = 0; hh < heads; ++hh) {
+            const int64_t nk = k_offs[b + 1] - k_offs[b];
+            double* p = (double*)malloc(sizeof(double) * (size_t)(nk > 0 ? nk : 1));
+            double* ds = (double*)malloc(sizeof(double) * (size_t)(nk > 0 ? nk : 1));
+            for (int64_t a = q_offs[b]; a < q_offs[b + 1]; ++a) {
+                const int64_t qi = (int64_t)q_rows[a] * C + hh * d;
+                double mx = -INFINITY;
+                for (int64_t j = 0; j < nk; ++j) {
+                    const double* k = K + (int64_t)k_rows[k_offs[b] + j] * C + hh * d;
+                    double acc = 0.0;
+                    for (int64_t c = 0; c < d; ++c) acc += Q[qi + c] * k[c];
+                    p[j] = acc * scale;
+                    if (p[j] > mx) mx = p[j];
+                }
+                double sum = 0.0;
+                for (int64_t j = 0; j < nk; ++j) { p[j] = exp(p[j] - mx); sum += p[j]; }
+                double delta = 0.0;
+                for (int64_t j = 0; j < nk; ++j) {
+                    const double* v = V + (int64_t)k_rows[k_offs[b] + j] * C + hh * d;
+                    p[j] /= sum;
+                    double acc = 0.0;
+                    for (int64_t c = 0; c < d; ++c) acc += dA[qi + c] * v[c];
+                    ds[j] = acc;
+                    delta += p[j] * acc;
+                }
+                for (int64_t j = 0; j < nk; ++j) {
+                    const int64_t kj = (int64_t)k_rows[k_offs[b] + j] * C + hh * d;
+                    const double dm = p[j] * (ds[j] - delta);
+                    for (int64_t c = 0; c < d; ++c) {
+                        dQ[qi + c] += dm * K[kj + c] * scale;
+                        dK[kj + c] += dm * Q[qi + c] * scale;
+                        dV[kj + c] += p[j] * dA[qi + c];
+                    }
+                }
+            }
+            free(p);
+            free(ds);
+        }
+}
+
+/*
+ * Cached activations of an attention layer under SBP relative to full backpropagation, counted term by term as
+ * the paper lists them (Sec. 4): QKV vectors h d n each, attention maps before and after the softmax h n n each.
+ *   mode 0, Drop Query only: K and V whole, Q and both maps at keep ratio r:  (2 + r) h d n + 2 r h n n
+ *   mode 1, Drop QKV:        Q, K, V at r, both maps at r^2:                   3 r h d n + 2 r^2 h n n
+ * over 3 h d n + 2 h n n.
+ */
+double oracle_attention_memory_ratio(int mode, double d, double n, double r)
+{
+    const double full = 3.0 * d * n + 2.0 * n * n;
+    if (mode == 0) return ((2.0 + r) * d * n + 2.0 * r * n * n) / full;
+    return (3.0 * r * d * n + 2.0 * r * r * n * n) / full;
 }

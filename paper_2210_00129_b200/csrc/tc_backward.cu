@@ -304,17 +304,16 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     // Narrow layers leave half of each accumulator slot unused, which makes room for the bias gradient as one more
     // output column of the dW tiles: db[j] = sum_m dY[m, j] * 1.  The "column of ones" is a constant 64 x 64 operand
     // block (MN-major, only its first column set) kept in the third staging buffer; a second, 16-wide MMA per k-step
-    // multiplies it with the same gathered rows of dY.
-    const uint32_t dw_bufs = (kNarrow && p.db_from_mma) ? kEpiBufs - 1 : kEpiBufs;   // staging buffers left to the dW epilogue
+    // multiplies it with the same gathered rows of dY.  Wide layers have no spare columns in a slot, but under the role
+    // split a dW block runs a single piece and never touches the second slot, so the column goes there.
+    const uint32_t dw_bufs = p.db_from_mma ? kEpiBufs - 1 : kEpiBufs;   // staging buffers left to the dW epilogue
     const uint32_t ones_off = (ring - raw_addr) + kRingBytes + 256 + kBiasSmemBytes + (kEpiBufs - 1) * kEpiBufBytes;
-    if constexpr (kNarrow) {
-        if (p.db_from_mma) {
-            for (uint32_t w = threadIdx.x; w < kBlock64Bytes / 4; w += kTcThreads) {
-                const uint32_t row = w >> 5, word = w & 31u;            // 128-byte rows of 32 words; column 0 sits in chunk (row & 7)
-                reinterpret_cast<uint32_t*>(smem_raw + ones_off)[w] = (word == ((row & 7u) << 2)) ? 0x00003F80u : 0u;
-            }
-            ptx::fence_async_proxy();                                    // read by the tensor core (async proxy)
+    if (p.db_from_mma) {
+        for (uint32_t w = threadIdx.x; w < kBlock64Bytes / 4; w += kTcThreads) {
+            const uint32_t row = w >> 5, word = w & 31u;            // 128-byte rows of 32 words; column 0 sits in chunk (row & 7)
+            reinterpret_cast<uint32_t*>(smem_raw + ones_off)[w] = (word == ((row & 7u) << 2)) ? 0x00003F80u : 0u;
         }
+        ptx::fence_async_proxy();                                    // read by the tensor core (async proxy)
     }
     if (warp == 5) ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
     ptx::tc_fence_before_sync();
@@ -381,6 +380,9 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                // where the bias column accumulates: the unused half of a narrow tile's slot; with wide tiles the other
+                // slot, which a block that runs a single dW piece (the role split) never uses
+                const uint32_t bias_tmem = kNarrow ? d_tmem + 128u : tmem_base + (acc ^ 1u) * kAccCols;
                 // K-major (dX): a 16-deep slice is 32 bytes along the swizzled row, 8-row groups 1024 B apart.
                 // MN-major (dW): a 16-deep slice is 16 rows (two atoms); 64-wide blocks of the MN extent 8 KB apart.
                 const uint32_t idesc = t.is_dw ? ptx::umma_idesc_bf16(kBM, BNW, true, true)
@@ -399,11 +401,9 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                         const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, kAtomBytes);
                         const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, kAtomBytes);
                         ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
-                        if constexpr (kNarrow) {
-                            if (t.is_dw && t.col_tile == 0 && p.db_from_mma) {   // the bias column: accumulator columns 128..143, column 128 is db
-                                const uint64_t d1 = ptx::umma_desc_sw128(raw_addr + ones_off + u * k_step, kBlock64Bytes, kAtomBytes);
-                                ptx::umma_bf16(d_tmem + 128u, da, d1, ptx::umma_idesc_bf16(kBM, 16, true, true), (k | u) != 0u);
-                            }
+                        if (t.is_dw && t.col_tile == 0 && p.db_from_mma) {   // the bias column: 16 more accumulator columns, the first is db
+                            const uint64_t d1 = ptx::umma_desc_sw128(raw_addr + ones_off + u * k_step, kBlock64Bytes, kAtomBytes);
+                            ptx::umma_bf16(bias_tmem, da, d1, ptx::umma_idesc_bf16(kBM, 16, true, true), (k | u) != 0u);
                         }
                     }
                     ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));      // stage reusable once these MMAs retire
@@ -510,7 +510,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         // db partial of this CTA's share of the kept rows
-        if (p.db_partial != nullptr && !(kNarrow && p.db_from_mma)) {
+        if (p.db_partial != nullptr && !p.db_from_mma) {
             float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kRingBytes + 256);
             const int t = threadIdx.x - kBiasWarp0 * 32;
             const int V = C_out >> 3;                                  // 16-byte column vectors per row
@@ -638,7 +638,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const int j = (int)(t.row_tile * kBM) + warp * 32 + lane;
                 const int i0 = (int)(t.col_tile * BNW);
                 float* out_col = p.dW_out + (int64_t)t.split * p.dw_split_stride + (int64_t)i0 * C_out + j;
-                const bool bias_col = kNarrow && p.db_from_mma && t.col_tile == 0;
+                const bool bias_col = p.db_from_mma && t.col_tile == 0;
                 if (t.num_kb == 0) {                                 // a piece without kept rows contributes zero
                     if (!p.dw_accumulate && j < C_out)
                         for (int c0 = 0; c0 < BNW && i0 + c0 < C_in; ++c0) out_col[(int64_t)c0 * C_out] = 0.f;
@@ -681,7 +681,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
                     if (bias_col) {                                  // accumulator column 128: this piece's share of db
                         float v[kEpiChunk];
-                        ptx::tmem_ld_32x16(taddr + 128u, v);
+                        ptx::tmem_ld_32x16(kNarrow ? taddr + 128u : tmem_base + (acc ^ 1u) * kAccCols + ((uint32_t)(warp * 32) << 16), v);
                         ptx::tmem_ld_wait();
                         if (j < C_out) p.db_partial[(int64_t)t.split * C_out + j] = v[0];
                     }
@@ -846,7 +846,9 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
                 const double target = bytes_w / (bytes_w + bytes_x) * (double)kNumSMs;
                 int64_t sp = (int64_t)(target / (double)w_tiles + 0.5);
                 const int64_t x_rtiles = (M_keep_cap + kBM - 1) / kBM;
-                if (sp >= 2 && w_kb / sp >= 8 && x_rtiles >= sp && w_tiles * sp <= kNumSMs - 16) {
+                // worth it only with enough dX tiles per dX block to balance (a short list leaves the groups uneven)
+                if (sp >= 2 && w_kb / sp >= 8 && x_rtiles >= sp && w_tiles * sp <= kNumSMs - 16 &&
+                    x_tiles >= 8 * (kNumSMs - w_tiles * sp)) {
                     pl.splits = (int)sp;
                     pl.dw_ctas = (int)(w_tiles * sp);
                     role_split = true;
@@ -958,8 +960,9 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
         map_dw = map_x;                                              // never used
     }
     prm.db_partial = (db != nullptr) ? db_workspace : nullptr;
-    // narrow layers (both tile kinds 128 wide): db is one more output column of the dW tiles, one partial row per split
-    const bool db_from_mma = db != nullptr && want_dw && pl.bnx <= 128 && pl.bnw <= 128;
+    // narrow layers (both tile kinds 128 wide), and wide ones under the role split (one dW piece per block, so the second
+    // accumulator slot is free): db is one more output column of the dW tiles, one partial row per split
+    const bool db_from_mma = db != nullptr && want_dw && ((pl.bnx <= 128 && pl.bnw <= 128) || pl.dw_ctas > 0);
     prm.db_from_mma = db_from_mma ? 1 : 0;
     const int db_rows = db_from_mma ? pl.splits : 0;                 // 0: one row per block (set below)
     prm.status_word = status_word;
