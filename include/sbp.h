@@ -12,6 +12,7 @@
  *   sbp_linear_forward   Y = X W + b, with that cache written by the same launch (Eq. 2)
  *   sbp_linear_backward  dW = X_keep^T dY_keep, db = sum dY_keep,
  *                        dX = scatter(dY_keep W^T), zeros elsewhere   (Eq. 5)
+ *   sbp_attention_backward  dQ, dK, dV of attention on the kept tokens (Sec. 4, Drop QKV / Drop Query only)
  *
  * Nothing is rescaled by 1/r: Eq. 1 keeps the plain 1/B factor.
  *
@@ -62,7 +63,8 @@ enum {
     SBP_FLAG_PLAIN_FMA = 8,   /* bf16 only: use the CUDA-core FMA kernels instead of the tensor-core ones */
     SBP_FLAG_DY_COMPACT = 16, /* dY holds only the kept rows, packed: [M_keep_cap, C_out] (chained layers, Sec. 3.3.1) */
     SBP_FLAG_DX_COMPACT = 32, /* dX receives only the kept rows, packed: [M_keep_cap, C_in]; no zero rows are written */
-    SBP_FLAG_W_OUT_IN = 64    /* W, and dW, are stored [C_out, C_in] (the usual layout of framework linear layers) */
+    SBP_FLAG_W_OUT_IN = 64,   /* W, and dW, are stored [C_out, C_in] (the usual layout of framework linear layers) */
+    SBP_FLAG_ATTN_ALL_KEYS = 128 /* sbp_attention_backward: keys and values are all tokens, only queries are dropped */
 };
 
 const char* sbp_status_string(sbp_status s);
@@ -229,6 +231,42 @@ sbp_status sbp_linear_backward(sbp_dtype dt,
 int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                      int64_t C_out, int want_dW, int want_db, int want_dX,
                                      uint32_t flags);
+
+/*
+ * SBP backward of multi-head scaled dot-product attention (Sec. 4, "How to apply SBP on MHSA?"; supplementary,
+ * "Gradient Calculation of Attention Layers": A = softmax(Q K^T / sqrt(d)) V per head, dQ = dM K / sqrt(d),
+ * dK = Q^T dM / sqrt(d), dV = S^T dA), with the gradient path restricted to token subsets.  Per sample b and head,
+ * with Zq the query tokens of the sample listed in q_rows and Zk its key / value tokens:
+ *   S_ij  = softmax over j in Zk of q_i . k_j / sqrt(d)                 i in Zq   (recomputed; no attention map is cached)
+ *   dS_ij = dA_i . v_j,   dM_ij = S_ij (dS_ij - sum_l S_il dS_il)
+ *   dQ_i  = sum_j dM_ij k_j / sqrt(d),  dK_j = sum_i dM_ij q_i / sqrt(d),  dV_j = sum_i S_ij dA_i
+ *   rows of dQ outside Zq and rows of dK, dV outside Zk = +0.0 (their gradient is dropped)
+ * Which subsets:
+ *   Drop QKV (what the paper applies to image transformers): kv_rows = NULL, flags = 0: Zk = Zq = the kept tokens;
+ *     the gradient path is attention among the kept tokens (the wrapped-operation reading of Algorithm 1; its maps
+ *     are the r^2 n^2 ones of the paper's memory formula).
+ *   Drop Query only (the supplementary's worked derivation): SBP_FLAG_ATTN_ALL_KEYS: Zk = all N tokens; dQ is the exact
+ *     gradient on the kept rows, dK = Q_keep^T dM_keep / sqrt(d), dV = S_keep^T dA_keep (dA is read on kept rows only:
+ *     inside a block that drops the same tokens everywhere its other rows are zero).
+ *   kv_rows / kv_offsets given: any other pair of subsets.  q_rows = NULL: every token is a query (with
+ *     SBP_FLAG_ATTN_ALL_KEYS this is ordinary attention backward, keep ratio 1).
+ * Layout: Q, K, V [B*N, ld_qkv] and dQ, dK, dV [B*N, ld_out] hold head hh in columns [hh*d, (hh+1)*d) from their
+ * own base pointers, so the three slices of a fused [B*N, 3*heads*d] projection output can be passed with
+ * ld = 3*heads*d; dA [B*N, ld_da] likewise.  q_rows / q_offsets (and kv_*) are lists as sbp_sample_keep writes them:
+ * ascending global row ids b*N + n and B + 1 offsets; max_kept = the largest per-sample count any list may hold
+ * (e.g. sbp_keep_count(...)), ignored when no list is given.
+ * This build: SBP_BF16 with d = 64, at most 256 tokens of a sample on either side (N <= 256 where a side takes all
+ * tokens), leading dimensions multiples of 8: otherwise SBP_ERR_UNSUPPORTED.  P = S and dM are rounded to bf16
+ * between the products, accumulation is fp32.  SBP_ERR_INVALID_ARG for null / misaligned pointers and bad sizes.
+ * status_word as for sbp_linear_backward.  Deterministic.
+ */
+sbp_status sbp_attention_backward(sbp_dtype dt, const void* Q /* dev */, const void* K /* dev */, const void* V /* dev */,
+                                  int64_t ld_qkv, const void* dA /* dev */, int64_t ld_da,
+                                  const int32_t* q_rows /* dev, nullable */, const int32_t* q_offsets /* dev, nullable */,
+                                  const int32_t* kv_rows /* dev, nullable */, const int32_t* kv_offsets /* dev, nullable */,
+                                  int64_t B, int64_t N, int64_t heads, int64_t head_dim, int64_t max_kept,
+                                  void* dQ /* dev */, void* dK /* dev */, void* dV /* dev */, int64_t ld_out,
+                                  uint32_t flags, int32_t* status_word /* dev, nullable */, void* stream);
 
 /*
  * Diagnostic (pure host function; no counterpart in the paper): how many times this process has

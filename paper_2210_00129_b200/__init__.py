@@ -22,11 +22,11 @@ SBP_ERR_CUDA, SBP_ERR_TIMEOUT, SBP_ERR_BAD_INDICES = 4, 5, 6
 SBP_F32, SBP_BF16 = 0, 1
 SBP_MASK_RANDOM, SBP_MASK_GRID, SBP_MASK_TEMPORAL, SBP_MASK_TEMPORAL_GRID = 0, 1, 2, 3
 SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
-SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT, SBP_FLAG_W_OUT_IN = 16, 32, 64
+SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT, SBP_FLAG_W_OUT_IN, SBP_FLAG_ATTN_ALL_KEYS = 16, 32, 64, 128
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
-           "sbp_plan_search_count", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
+           "sbp_plan_search_count", "sbp_attention_backward", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
            "sbp_selftest_bounded_wait")
 
 _lib = None
@@ -67,6 +67,9 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_linear_backward.restype = ci
     lib.sbp_linear_backward_kernel_count.argtypes = [ci, i64, i64, i64, i64, ci, ci, ci, u32]
     lib.sbp_linear_backward_kernel_count.restype = ci
+    lib.sbp_attention_backward.argtypes = [ci, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, i64, i64, i64, i64, i64, vp, vp, vp, i64,
+                                           u32, vp, vp]
+    lib.sbp_attention_backward.restype = ci
     lib.sbp_plan_search_count.argtypes = []
     lib.sbp_plan_search_count.restype = i64
     lib.sbp_step_host_arena_bytes.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl]
@@ -158,6 +161,18 @@ def sbp_linear_backward_kernel_count(dt, M, M_keep_cap, C_in, C_out, want_dW=Tru
                                      flags=0) -> int:
     return int(load_library().sbp_linear_backward_kernel_count(dt, M, M_keep_cap, C_in, C_out, int(want_dW),
                                                                int(want_db), int(want_dX), flags))
+
+
+def sbp_attention_backward(dt, Q, K, V, ld_qkv, dA, ld_da, q_rows, q_offsets, kv_rows, kv_offsets, B, N, heads, head_dim,
+                           max_kept, dQ, dK, dV, ld_out, flags=0, status_word=None, stream=None, check=True) -> int:
+    """dQ, dK, dV of attention restricted to the listed query and key / value tokens (Drop QKV / Drop Query only)."""
+    s = load_library().sbp_attention_backward(dt, _ptr(Q), _ptr(K), _ptr(V), ld_qkv, _ptr(dA), ld_da, _ptr(q_rows),
+                                              _ptr(q_offsets), _ptr(kv_rows), _ptr(kv_offsets), B, N, heads, head_dim,
+                                              max_kept, _ptr(dQ), _ptr(dK), _ptr(dV), ld_out, flags, _ptr(status_word),
+                                              _stream(stream))
+    if check:
+        _check(s, "sbp_attention_backward")
+    return s
 
 
 def sbp_plan_search_count() -> int:

@@ -1,0 +1,375 @@
+// SBP backward of scaled dot-product attention on token subsets (Sec. 4, "How to apply SBP on MHSA?"; supplementary,
+// "Gradient Calculation of Attention Layers"), bf16 on the tensor cores (tcgen05 / TMEM), head dimension 64.
+//
+// One (sample, head) problem at a time per block (persistent blocks, one per SM).  With Zq the kept query tokens and Zk
+// the kept key / value tokens of the sample (at most 256 each):
+//     S  = softmax_j(q_i . k_j / sqrt(d))  over j in Zk          (recomputed here: no n x n map is cached at all)
+//     dS = dA V^T,   dM = S * (dS - rowsum(S * dS)) / sqrt(d)
+//     dV = S^T dA,   dK = dM^T Q,   dQ = dM K
+// All five products run as tcgen05.mma on operands staged once in shared memory (128-byte swizzle): a row-major
+// [tokens x 64] tile serves as the K-major operand of Q K^T / dA V^T and, unchanged, as the MN-major operand of the
+// three gradient products.  A first pass over the query tiles finds each row's softmax statistics (maximum, sum,
+// rowsum(S * dS)) from S and dS in tensor memory; the second pass recomputes 128 x 128 blocks of S and dS, turns them
+// into bf16 blocks of S and dM in shared memory, and accumulates dV, dK (per key tile) and dQ (per query tile) in
+// tensor memory: 128 + 128 + 64 + 64 + 2 * 64 = 512 columns.  Rows of the outputs outside the token sets are zeroed
+// by a small kernel of their own.  Every wait is bounded and reports through the status word.
+#include "tc_ptx.cuh"
+
+namespace sbp {
+namespace {
+
+constexpr int kAttnThreads = 256;
+constexpr int kD = 64;                          // head dimension (one 128-byte swizzle row of bf16)
+constexpr int kMaxTok = 256;                    // most kept tokens of a sample on either side
+constexpr uint32_t kRowB = 128;
+constexpr uint32_t kTokBytes = kMaxTok * kRowB;             // 32 KB: one [256 x 64] operand
+constexpr uint32_t kBlkBytes = 128 * kRowB;                 // 16 KB: [128 rows x 64 columns]
+constexpr uint32_t kAttnSmem = 4 * kTokBytes + 2 * 2 * kBlkBytes + 1024;   // Q, K, V, dA + S block + dM block (+ alignment slack)
+static_assert(kAttnSmem <= 227 * 1024, "shared memory per block");
+
+// tensor-memory columns
+constexpr uint32_t kColS = 0, kColDS = 128, kColDV = 256, kColDK = 320, kColDQ = 384;   // second pass
+constexpr uint32_t kColS1 = 0, kColDS1 = 256;                                            // first pass: up to 256 keys each
+
+struct AttnParams {
+    const __nv_bfloat16 *Q, *K, *V, *dA;
+    int64_t ld_qkv, ld_da, ld_out;
+    const int32_t *q_rows, *q_offs, *k_rows, *k_offs;     // null rows = every token of the sample
+    int B, N, heads;
+    __nv_bfloat16 *dQ, *dK, *dV;
+    float scale;
+    int32_t* status_word;
+};
+
+struct AttnShared {
+    uint64_t bar_s, bar_o;
+    uint32_t tmem_slot;
+    int abort_flag;
+    float part[2][128][3];        // per column half: running maximum, sum, sum of e^(s-m) * dS
+    float stat[kMaxTok][3];       // per query row: maximum (scaled, base 2), 1 / sum, rowsum(S * dS)
+};
+
+__device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk) { return row * kRowB + ((chunk ^ (row & 7u)) << 4); }
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// gather `tiles * 128` rows of 64 bf16 (head slice) into a swizzled operand; rows past `count` become zeros
+__device__ __forceinline__ void load_rows(uint32_t dst, const __nv_bfloat16* src, int64_t ld, const int32_t* rows, int64_t first,
+                                          int64_t base_row, int count, int tiles, int col0) {
+    const uint32_t chunk = threadIdx.x & 7u;
+    for (int r = threadIdx.x >> 3; r < tiles * 128; r += kAttnThreads / 8) {
+        const bool live = r < count;
+        const int64_t g = live ? (rows != nullptr ? (int64_t)__ldg(rows + first + r) : base_row + r) : 0;
+        ptx::cp_async_16(dst + swz((uint32_t)r, chunk), src + (live ? g * ld + col0 + chunk * 8 : 0), live ? 16u : 0u);
+    }
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ AttnShared sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* gen = smem_raw + (base - raw);                 // generic pointer to the same place
+    const uint32_t sQ = base, sK = base + kTokBytes, sV = base + 2 * kTokBytes, sDA = base + 3 * kTokBytes;
+    const uint32_t sP = base + 4 * kTokBytes, sDM = sP + 2 * kBlkBytes;     // [2 blocks of 64 keys][128 query rows][128 B]
+    uint8_t* gP = gen + 4 * kTokBytes;
+    uint8_t* gDM = gP + 2 * kBlkBytes;
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&sh.bar_s), 1);
+        ptx::mbar_init(ptx::smem_addr(&sh.bar_o), 1);
+        sh.abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 0) ptx::tmem_alloc(ptx::smem_addr(&sh.tmem_slot), 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_slot);
+    volatile int* abort_flag = &sh.abort_flag;
+    pdl_wait();
+    const bool skip_all = p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0;
+
+    const int q4 = warp & 3, half = warp >> 2;              // TMEM lane quadrant of this warp; which half of the columns it takes
+    const int row = q4 * 32 + lane;                         // accumulator row (query row, or key row in the dV / dK epilogue)
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const float sl2 = p.scale * 1.4426950408889634f;        // scores are kept in base 2: e^(x) = 2^(x log2 e)
+    uint32_t n_s = 0, n_o = 0;                              // completed uses of the two barriers
+    bool ok = !skip_all;
+
+    for (int prob = blockIdx.x; ok && prob < p.B * p.heads; prob += gridDim.x) {
+        const int b = prob / p.heads, hh = prob % p.heads;
+        const int64_t q0 = p.q_rows ? __ldg(p.q_offs + b) : 0, k0 = p.k_rows ? __ldg(p.k_offs + b) : 0;
+        const int nq = p.q_rows ? (int)(__ldg(p.q_offs + b + 1) - q0) : p.N;
+        const int nk = p.k_rows ? (int)(__ldg(p.k_offs + b + 1) - k0) : p.N;
+        if (nq <= 0 || nk <= 0) continue;
+        const int QT = (nq + 127) >> 7, KT = (nk + 127) >> 7;
+        const int col0 = hh * kD;
+        const int64_t base_row = (int64_t)b * p.N;
+        // ---- stage the four operands ----
+        load_rows(sQ, p.Q, p.ld_qkv, p.q_rows, q0, base_row, nq, QT, col0);
+        load_rows(sDA, p.dA, p.ld_da, p.q_rows, q0, base_row, nq, QT, col0);
+        load_rows(sK, p.K, p.ld_qkv, p.k_rows, k0, base_row, nk, KT, col0);
+        load_rows(sV, p.V, p.ld_qkv, p.k_rows, k0, base_row, nk, KT, col0);
+        ptx::cp_async_wait_all();
+        ptx::fence_async_proxy();
+        __syncthreads();
+
+        // ---- first pass: softmax statistics of every query row ----
+        for (int qt = 0; qt < QT && ok; ++qt) {
+            if (threadIdx.x == 0) {
+                ptx::tc_fence_after_sync();
+                const uint32_t idesc = ptx::umma_idesc_bf16(128, KT * 128, false, false);
+#pragma unroll
+                for (uint32_t u = 0; u < 4; ++u) {
+                    const uint64_t dq = ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 32, 16, 1024);
+                    const uint64_t dk = ptx::umma_desc_sw128(sK + u * 32, 16, 1024);
+                    ptx::umma_bf16(tmem + kColS1, dq, dk, idesc, u != 0);
+                }
+#pragma unroll
+                for (uint32_t u = 0; u < 4; ++u) {
+                    const uint64_t da = ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 32, 16, 1024);
+                    const uint64_t dv = ptx::umma_desc_sw128(sV + u * 32, 16, 1024);
+                    ptx::umma_bf16(tmem + kColDS1, da, dv, idesc, u != 0);
+                }
+                ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
+            }
+            ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_s), n_s & 1u, abort_flag, p.status_word);
+            ++n_s;
+            ok = !__syncthreads_or(!ok);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            // this thread: row `row`, columns [half * KT * 64, (half + 1) * KT * 64)
+            float m = -INFINITY, l = 0.f, u_acc = 0.f;
+            const int cbeg = half * KT * 64, cend = cbeg + KT * 64;
+            for (int c = cbeg; c < cend; c += 32) {
+                float s[32], ds[32];
+                ptx::tmem_ld_32x32(tmem + kColS1 + (uint32_t)c + lane_off, s);
+                ptx::tmem_ld_32x32(tmem + kColDS1 + (uint32_t)c + lane_off, ds);
+                ptx::tmem_ld_wait();
+                float cm = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    s[j] = (c + j < nk) ? s[j] * sl2 : -INFINITY;
+                    cm = fmaxf(cm, s[j]);
+                }
+                if (cm > m) {                                // rescale what has been summed so far
+                    const float f = exp2f(m - cm);           // 0 on the first chunk (m = -inf)
+                    l *= f; u_acc *= f; m = cm;
+                }
+                if (m > -INFINITY) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float e = exp2f(s[j] - m);     // 0 for masked columns
+                        l += e;
+                        u_acc += e * ds[j];
+                    }
+                }
+            }
+            sh.part[half][row][0] = m; sh.part[half][row][1] = l; sh.part[half][row][2] = u_acc;
+            ptx::tc_fence_before_sync();
+            __syncthreads();
+            if (half == 0) {
+                const float m0 = sh.part[0][row][0], m1 = sh.part[1][row][0];
+                const float mm = fmaxf(m0, m1);
+                const float f0 = (m0 > -INFINITY) ? exp2f(m0 - mm) : 0.f, f1 = (m1 > -INFINITY) ? exp2f(m1 - mm) : 0.f;
+                const float ll = sh.part[0][row][1] * f0 + sh.part[1][row][1] * f1;
+                const float uu = sh.part[0][row][2] * f0 + sh.part[1][row][2] * f1;
+                sh.stat[qt * 128 + row][0] = mm;
+                sh.stat[qt * 128 + row][1] = 1.f / ll;
+                sh.stat[qt * 128 + row][2] = uu / ll;
+            }
+            __syncthreads();
+        }
+        if (!ok) break;
+
+        // ---- second pass: blocks of S and dM, and the three gradient products ----
+        for (int kt = 0; kt < KT && ok; ++kt) {
+            for (int qt = 0; qt < QT && ok; ++qt) {
+                if (threadIdx.x == 0) {
+                    ptx::tc_fence_after_sync();
+                    const uint32_t idesc = ptx::umma_idesc_bf16(128, 128, false, false);
+#pragma unroll
+                    for (uint32_t u = 0; u < 4; ++u) {
+                        const uint64_t dq = ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 32, 16, 1024);
+                        const uint64_t dk = ptx::umma_desc_sw128(sK + kt * kBlkBytes + u * 32, 16, 1024);
+                        ptx::umma_bf16(tmem + kColS, dq, dk, idesc, u != 0);
+                    }
+#pragma unroll
+                    for (uint32_t u = 0; u < 4; ++u) {
+                        const uint64_t da = ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 32, 16, 1024);
+                        const uint64_t dv = ptx::umma_desc_sw128(sV + kt * kBlkBytes + u * 32, 16, 1024);
+                        ptx::umma_bf16(tmem + kColDS, da, dv, idesc, u != 0);
+                    }
+                    ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
+                }
+                ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_s), n_s & 1u, abort_flag, p.status_word);
+                ++n_s;
+                // the products of the previous block have read the S / dM blocks in shared memory by now (they were
+                // issued before the MMAs just waited for, and the tensor pipe runs in order)
+                ok = !__syncthreads_or(!ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const float mx = sh.stat[qt * 128 + row][0], inv_l = sh.stat[qt * 128 + row][1], delta = sh.stat[qt * 128 + row][2];
+#pragma unroll
+                for (int c = 0; c < 64; c += 32) {
+                    float s[32], ds[32];
+                    ptx::tmem_ld_32x32(tmem + kColS + (uint32_t)(half * 64 + c) + lane_off, s);
+                    ptx::tmem_ld_32x32(tmem + kColDS + (uint32_t)(half * 64 + c) + lane_off, ds);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const bool live = kt * 128 + half * 64 + c + j < nk;
+                        const float pj = live ? exp2f(s[j] * sl2 - mx) * inv_l : 0.f;
+                        s[j] = pj;
+                        ds[j] = pj * (ds[j] - delta) * p.scale;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t off = swz((uint32_t)row, (uint32_t)(c / 8 + q));
+                        *reinterpret_cast<uint4*>(gP + half * kBlkBytes + off) =
+                            make_uint4(pack2(s[q * 8], s[q * 8 + 1]), pack2(s[q * 8 + 2], s[q * 8 + 3]), pack2(s[q * 8 + 4], s[q * 8 + 5]), pack2(s[q * 8 + 6], s[q * 8 + 7]));
+                        *reinterpret_cast<uint4*>(gDM + half * kBlkBytes + off) =
+                            make_uint4(pack2(ds[q * 8], ds[q * 8 + 1]), pack2(ds[q * 8 + 2], ds[q * 8 + 3]), pack2(ds[q * 8 + 4], ds[q * 8 + 5]), pack2(ds[q * 8 + 6], ds[q * 8 + 7]));
+                    }
+                }
+                ptx::fence_async_proxy();                    // the blocks are read by the tensor core
+                ptx::tc_fence_before_sync();
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    ptx::tc_fence_after_sync();
+                    const uint32_t id_t = ptx::umma_idesc_bf16(128, 64, true, true);     // dV, dK: both operands MN-major
+                    const uint32_t id_q = ptx::umma_idesc_bf16(128, 64, false, true);    // dQ: dM K-major, K MN-major
+#pragma unroll
+                    for (uint32_t u = 0; u < 8; ++u) {           // reduction over the 128 query rows of the tile, 16 at a time
+                        const uint64_t dp = ptx::umma_desc_sw128(sP + u * 2048, kBlkBytes, 1024);
+                        const uint64_t dda = ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 2048, kBlkBytes, 1024);
+                        ptx::umma_bf16(tmem + kColDV, dp, dda, id_t, (qt | (int)u) != 0);
+                        const uint64_t ddm = ptx::umma_desc_sw128(sDM + u * 2048, kBlkBytes, 1024);
+                        const uint64_t dq = ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 2048, kBlkBytes, 1024);
+                        ptx::umma_bf16(tmem + kColDK, ddm, dq, id_t, (qt | (int)u) != 0);
+                    }
+#pragma unroll
+                    for (uint32_t u = 0; u < 8; ++u) {           // reduction over the 128 keys of the tile: two 64-key blocks x four steps
+                        const uint64_t ddm = ptx::umma_desc_sw128(sDM + (u >> 2) * kBlkBytes + (u & 3u) * 32, 16, 1024);
+                        const uint64_t dk = ptx::umma_desc_sw128(sK + kt * kBlkBytes + u * 2048, kBlkBytes, 1024);
+                        ptx::umma_bf16(tmem + kColDQ + (uint32_t)qt * 64u, ddm, dk, id_q, (kt | (int)u) != 0);
+                    }
+                    ptx::umma_commit(ptx::smem_addr(&sh.bar_o));
+                }
+                ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_o), n_o & 1u, abort_flag, p.status_word);
+                ++n_o;
+                ok = !__syncthreads_or(!ok);
+            }
+            if (!ok) break;
+            // ---- dV and dK of this key tile: accumulator row = key, 64 columns; this thread takes 32 of them ----
+            ptx::tc_fence_after_sync();
+            const int key = kt * 128 + row;
+#pragma unroll
+            for (int which = 0; which < 2; ++which) {
+                float v[32];
+                ptx::tmem_ld_32x32(tmem + (which ? kColDK : kColDV) + (uint32_t)(half * 32) + lane_off, v);
+                ptx::tmem_ld_wait();
+                if (key < nk) {
+                    const int64_t g = p.k_rows ? (int64_t)__ldg(p.k_rows + k0 + key) : base_row + key;
+                    __nv_bfloat16* out = (which ? p.dK : p.dV) + g * p.ld_out + col0 + half * 32;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        ptx::st_global_v4(out + q * 8, pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]),
+                                          pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncthreads();
+        }
+        if (!ok) break;
+        // ---- dQ of every query tile ----
+        ptx::tc_fence_after_sync();
+        for (int qt = 0; qt < QT; ++qt) {
+            float v[32];
+            ptx::tmem_ld_32x32(tmem + kColDQ + (uint32_t)(qt * 64 + half * 32) + lane_off, v);
+            ptx::tmem_ld_wait();
+            const int qi = qt * 128 + row;
+            if (qi < nq) {
+                const int64_t g = p.q_rows ? (int64_t)__ldg(p.q_rows + q0 + qi) : base_row + qi;
+                __nv_bfloat16* out = p.dQ + g * p.ld_out + col0 + half * 32;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    ptx::st_global_v4(out + q * 8, pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]),
+                                      pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
+            }
+        }
+        ptx::tc_fence_before_sync();
+        __syncthreads();                                     // operands and accumulators are free for the next problem
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, 512);
+    }
+}
+
+// rows of `out` [M, ld] (columns [0, cols)) that are not in the ascending list `rows[0 .. *total)` become +0.0:
+// entry m of the list owns the gap in front of it, one extra worker the tail
+__global__ void zero_rows_outside_kernel(__nv_bfloat16* out, int64_t M, int64_t ld, int cols, const int32_t* rows,
+                                         const int32_t* total_dev, const int32_t* status_word) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (status_word != nullptr && *reinterpret_cast<const volatile int32_t*>(status_word) != 0) return;
+    const int64_t total = __ldg(total_dev);
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t m = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); m <= total; m += warps) {
+        const int64_t lo = m > 0 ? (int64_t)__ldg(rows + m - 1) + 1 : 0;
+        const int64_t hi = m < total ? (int64_t)__ldg(rows + m) : M;
+        for (int64_t r = lo; r < hi; ++r)
+            for (int c = lane * 8; c < cols; c += 256) ptx::st_global_v4(out + r * ld + c, 0u, 0u, 0u, 0u);
+    }
+}
+
+}  // namespace
+
+bool attention_supported(sbp_dtype dt, int64_t head_dim) { return dt == SBP_BF16 && head_dim == kD; }
+int64_t attention_max_tokens() { return kMaxTok; }
+
+cudaError_t launch_attention_backward(const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA, int64_t ld_da,
+                                      const int32_t* q_rows, const int32_t* q_offs, const int32_t* k_rows, const int32_t* k_offs,
+                                      int64_t B, int64_t N, int64_t heads, void* dQ, void* dK, void* dV, int64_t ld_out,
+                                      int32_t* status_word, cudaStream_t stream) {
+    const cudaError_t opt = opt_in_dynamic_smem<attention_bwd_kernel>((int)kAttnSmem);
+    if (opt != cudaSuccess) return opt;
+    AttnParams prm;
+    prm.Q = static_cast<const __nv_bfloat16*>(Q); prm.K = static_cast<const __nv_bfloat16*>(K);
+    prm.V = static_cast<const __nv_bfloat16*>(V); prm.dA = static_cast<const __nv_bfloat16*>(dA);
+    prm.ld_qkv = ld_qkv; prm.ld_da = ld_da; prm.ld_out = ld_out;
+    prm.q_rows = q_rows; prm.q_offs = q_offs; prm.k_rows = k_rows; prm.k_offs = k_offs;
+    prm.B = (int)B; prm.N = (int)N; prm.heads = (int)heads;
+    prm.dQ = static_cast<__nv_bfloat16*>(dQ); prm.dK = static_cast<__nv_bfloat16*>(dK); prm.dV = static_cast<__nv_bfloat16*>(dV);
+    prm.scale = 1.0f / sqrtf((float)kD);
+    prm.status_word = status_word;
+    const int64_t problems = B * heads;
+    const dim3 grid((unsigned)(problems < kNumSMs ? problems : kNumSMs));
+    cudaError_t e = cudaSuccess;
+    const int cols = (int)(heads * kD);
+    // the zeros first: they touch only rows outside the lists, the products only rows inside them
+    if (q_rows != nullptr)
+        e = launch_pdl(zero_rows_outside_kernel, dim3(2 * kNumSMs), dim3(256), 0, stream, prm.dQ, B * N, ld_out, cols, q_rows,
+                       q_offs + B, (const int32_t*)status_word);
+    if (e == cudaSuccess && k_rows != nullptr) {
+        e = launch_pdl(zero_rows_outside_kernel, dim3(2 * kNumSMs), dim3(256), 0, stream, prm.dK, B * N, ld_out, cols, k_rows,
+                       k_offs + B, (const int32_t*)status_word);
+        if (e == cudaSuccess)
+            e = launch_pdl(zero_rows_outside_kernel, dim3(2 * kNumSMs), dim3(256), 0, stream, prm.dV, B * N, ld_out, cols, k_rows,
+                           k_offs + B, (const int32_t*)status_word);
+    }
+    if (e != cudaSuccess) return e;
+    return launch_pdl(attention_bwd_kernel, grid, dim3(kAttnThreads), kAttnSmem, stream, prm);
+}
+
+}  // namespace sbp

@@ -331,6 +331,42 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
 
 int64_t sbp_plan_search_count(void) { return tc_plan_searches(); }
 
+sbp_status sbp_attention_backward(sbp_dtype dt, const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA,
+                                  int64_t ld_da, const int32_t* q_rows, const int32_t* q_offsets, const int32_t* kv_rows,
+                                  const int32_t* kv_offsets, int64_t B, int64_t N, int64_t heads, int64_t head_dim,
+                                  int64_t max_kept, void* dQ, void* dK, void* dV, int64_t ld_out, uint32_t flags,
+                                  int32_t* status_word, void* stream) {
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (Q == nullptr || K == nullptr || V == nullptr || dA == nullptr || dQ == nullptr || dK == nullptr || dV == nullptr)
+        return SBP_ERR_INVALID_ARG;
+    if (B <= 0 || N <= 0 || heads <= 0 || head_dim <= 0 || B * N >= (1ll << 31) || heads * head_dim >= (1ll << 24))
+        return SBP_ERR_INVALID_ARG;
+    if ((q_rows == nullptr) != (q_offsets == nullptr) || (kv_rows == nullptr) != (kv_offsets == nullptr))
+        return SBP_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)SBP_FLAG_ATTN_ALL_KEYS) return SBP_ERR_INVALID_ARG;
+    if ((flags & SBP_FLAG_ATTN_ALL_KEYS) && kv_rows != nullptr) return SBP_ERR_INVALID_ARG;
+    const int64_t C = heads * head_dim;
+    if (ld_qkv < C || ld_da < C || ld_out < C) return SBP_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dA) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) ||
+        (reinterpret_cast<uintptr_t>(q_rows) & 3u) || (reinterpret_cast<uintptr_t>(q_offsets) & 3u) ||
+        (reinterpret_cast<uintptr_t>(kv_rows) & 3u) || (reinterpret_cast<uintptr_t>(kv_offsets) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    if (!attention_supported(dt, head_dim)) return SBP_ERR_UNSUPPORTED;
+    if (ld_qkv % 8 != 0 || ld_da % 8 != 0 || ld_out % 8 != 0) return SBP_ERR_UNSUPPORTED;
+    // keys and values: their own lists, else all tokens when asked for, else the query lists (Drop QKV)
+    const int32_t* k_rows = kv_rows != nullptr ? kv_rows : ((flags & SBP_FLAG_ATTN_ALL_KEYS) ? nullptr : q_rows);
+    const int32_t* k_offs = kv_rows != nullptr ? kv_offsets : ((flags & SBP_FLAG_ATTN_ALL_KEYS) ? nullptr : q_offsets);
+    // most tokens a sample can bring to either side: N where a side takes all tokens, else the caller's bound on its lists
+    const bool any_all = q_rows == nullptr || k_rows == nullptr;
+    const bool any_list = q_rows != nullptr || k_rows != nullptr;
+    if (any_list && (max_kept <= 0 || max_kept > N)) return SBP_ERR_INVALID_ARG;
+    const int64_t most = any_all ? N : max_kept;
+    if (most > attention_max_tokens()) return SBP_ERR_UNSUPPORTED;
+    const cudaError_t e = launch_attention_backward(Q, K, V, ld_qkv, dA, ld_da, q_rows, q_offsets, k_rows, k_offs, B, N, heads, dQ,
+                                                    dK, dV, ld_out, status_word, (cudaStream_t)stream);
+    return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
 namespace {
 struct StepArena {
     size_t X, dY, W, rows, offs, Xk, dW, db, dX, status, ws, ws_bytes, total;

@@ -187,6 +187,15 @@ sbp_status launch_tc_forward(const void* X, const void* W, bool w_out_in, const 
                              void* Y, const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap,
                              void* X_keep, int32_t* status_word, cudaStream_t stream);
 
+// SBP attention backward on token subsets (bf16, head dimension 64, at most attention_max_tokens() kept tokens per sample
+// and side); null row lists mean every token of the sample
+bool    attention_supported(sbp_dtype dt, int64_t head_dim);
+int64_t attention_max_tokens();
+cudaError_t launch_attention_backward(const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA, int64_t ld_da,
+                                      const int32_t* q_rows, const int32_t* q_offs, const int32_t* k_rows, const int32_t* k_offs,
+                                      int64_t B, int64_t N, int64_t heads, void* dQ, void* dK, void* dV, int64_t ld_out,
+                                      int32_t* status_word, cudaStream_t stream);
+
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
