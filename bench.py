@@ -9,7 +9,7 @@ keep-ratio sweep {0.25, 0.5, 0.75, 1.0} reported beside the headline; `--workloa
 the single fc1 layer at B=64.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
-    python bench.py --sweep all|vit|convnext|detection|forward|blocks|sampler [--iters 24]
+    python bench.py --sweep all|vit|convnext|detection|forward|blocks|attention|sampler [--iters 24]
 
 Prints one JSON line (rank 0).  ``value`` counts the backward FLOPs of the kept rows
 (4 * M_keep * C_in * C_out per layer, step and GPU) over device time, with inputs resident in HBM;
@@ -828,6 +828,48 @@ def forward_layers(bench, pk):
     return rows
 
 
+def attention_layers(bench, pk):
+    """sbp_attention_backward on ViT-B/16 heads (12 heads of 64, 196 tokens, B = 128): Drop QKV at three keep ratios,
+    Drop Query only, and ordinary attention backward (keep ratio 1.0) through the same kernel."""
+    B, H, W_, heads, d = 128, 14, 14, 12, 64
+    N, M, C = H * W_, B * H * W_, heads * d
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    n_sets = 3
+    sets = [dict(qkv=torch.randn(M, 3 * C, device="cuda", generator=gen).bfloat16(),
+                 dA=(torch.randn(M, C, device="cuda", generator=gen) * 0.01).bfloat16(),
+                 out=torch.zeros(M, 3 * C, device="cuda", dtype=torch.bfloat16),
+                 rows=torch.zeros(M, dtype=torch.int32, device="cuda"), offs=torch.zeros(B + 1, dtype=torch.int32, device="cuda"))
+            for _ in range(n_sets)]
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out_rows = []
+    for name, r, flags, lists in (("Drop QKV r=0.25", 0.25, 0, True), ("Drop QKV r=0.5", 0.5, 0, True), ("Drop QKV r=0.75", 0.75, 0, True),
+                                  ("Drop Query only r=0.5", 0.5, sbp.SBP_FLAG_ATTN_ALL_KEYS, True),
+                                  ("all tokens (keep ratio 1.0)", 1.0, sbp.SBP_FLAG_ATTN_ALL_KEYS, False)):
+        cap = sbp.sbp_keep_count(0, H, W_, r)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(bench.stream):
+            for s_ in sets:
+                sbp.sbp_sample_keep(0, B, H, W_, r, 0, 0, 0, 0, s_["rows"], s_["offs"], stream=bench.sid)
+        bench.stream.synchronize()
+
+        def call(k, i):
+            s_ = sets[k]
+            q, o = s_["qkv"], s_["out"]
+            sbp.sbp_attention_backward(sbp.SBP_BF16, q[:, :C], q[:, C:2 * C], q[:, 2 * C:], 3 * C, s_["dA"], C,
+                                       s_["rows"] if lists else None, s_["offs"] if lists else None, None, None, B, N, heads, d,
+                                       cap if lists else 0, o[:, :C], o[:, C:2 * C], o[:, 2 * C:], 3 * C, flags, st, stream=bench.sid)
+        us = bench.time_us(call, n_sets)
+        nq = cap if lists else N
+        nk = N if (flags & sbp.SBP_FLAG_ATTN_ALL_KEYS) else cap
+        flop = 10.0 * nq * nk * d * B * heads
+        # kept rows of Q and dA, of K and V read; kept rows of dQ, dK, dV written, zeros in all their other rows
+        by = (2.0 * nq + 2.0 * nk) * B * C * 2 + 3.0 * M * C * 2
+        tmin = max(flop / (pk["bf16_tflops_sustained"] * 1e12), by / (pk["hbm_gbs"] * 1e9)) * 1e6
+        out_rows.append((name, nq, nk, us, tmin, flop / us / 1e6, by / us / 1e3))
+    assert int(st.item()) == 0
+    return out_rows
+
+
 def sampler_stress(bench, pk):
     """Sampler alone on a shape whose index stream is large enough to read as bandwidth."""
     rows = []
@@ -855,7 +897,7 @@ def run_sweep(args):
     args.group = args.sweep
     print(f"peaks ({kind}): bf16 {pk['bf16_tflops_sustained']:.0f} TFLOP/s sustained, HBM {pk['hbm_gbs']:.0f} GB/s; "
           f"{args.iters} graph-replayed launches per figure, rotating buffer sets larger than L2\n")
-    if args.group not in ("sampler", "blocks", "forward"):
+    if args.group not in ("sampler", "blocks", "forward", "attention"):
         if args.compact:
             print("us (t_min / t) per call; bound of the whole backward in the last column\n")
             print("| layer | M_keep | sample | cache | db | dW | dX | dW+dX (one launch) | backward (dW+db+dX) | TFLOP/s | bound |")
@@ -909,6 +951,14 @@ def run_sweep(args):
         for nm, B, H, W_, d, r in blocks:
             cap, ts, tp, flop = mlp_block(bench, B, H, W_, d, 4 * d, r)
             print(f"| {nm} | {cap} | {ts:.1f} | {tp:.1f} | {ts / tp:.2f} | {flop / tp / 1e6:.0f} |")
+    if args.group in ("attention", "all"):
+        print("\n| sbp_attention_backward, ViT-B/16 heads (B=128, 12 x 64, 196 tokens) | queries | keys | us | t_min us | t_min/t | TFLOP/s | GB/s |")
+        print("|---|---|---|---|---|---|---|---|")
+        rows = attention_layers(bench, pk)
+        for name, nq, nk, us, tmin, tf, gbs in rows:
+            print(f"| {name} | {nq} | {nk} | {us:.1f} | {tmin:.1f} | {tmin / us:.2f} | {tf:.0f} | {gbs:.0f} |")
+        full = rows[-1][3]
+        print("\nspeed-up against keep ratio 1.0: " + ", ".join(f"{name}: {full / us:.2f}x" for name, _, _, us, _, _, _ in rows[:-1]))
     if args.group in ("sampler", "all"):
         print("\n| sampler shape | kept ids | us | index stream GB/s | positions per ns |")
         print("|---|---|---|---|---|")
@@ -928,7 +978,7 @@ def main():
                     help="timed steps: replay of captured steps (default) or direct C-ABI calls from Python")
     ap.add_argument("--allreduce", action="store_true",
                     help="also time the steps followed by the all-reduce of dW / db when started under a launcher with one rank")
-    ap.add_argument("--sweep", default=None, choices=["vit", "convnext", "detection", "forward", "blocks", "sampler", "all"],
+    ap.add_argument("--sweep", default=None, choices=["vit", "convnext", "detection", "forward", "blocks", "attention", "sampler", "all"],
                     help="print per-call timing tables of every layer shape of a group instead of the JSON line")
     ap.add_argument("--iters", type=int, default=24, help="--sweep: launches per figure")
     ap.add_argument("--compact", action="store_true", help="--sweep: one table row per layer, us (t_min / t) per call")

@@ -315,14 +315,305 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
     }
 }
 
-// rows of `out` [M, ld] (columns [0, cols)) that are not in the ascending list `rows[0 .. *total)` become +0.0:
-// entry m of the list owns the gap in front of it, one extra worker the tail
-__global__ void zero_rows_outside_kernel(__nv_bfloat16* out, int64_t M, int64_t ld, int cols, const int32_t* rows,
-                                         const int32_t* total_dev, const int32_t* status_word) {
+
+// ---------------------------------------------------------------------------------------------
+// At most 128 kept tokens on both sides (keep ratios up to 0.5 on 14 x 14 maps, the paper's setting): one 128 x 128
+// tile per problem, so S and dS are computed once, the statistics and the blocks come from the same accumulators, and
+// the block is small enough for two per SM (96 KB of operands, 256 tensor-memory columns, 128 threads): while one block
+// waits for its loads or its products, the other computes.  Each thread owns one query row: it keeps the row's dM as
+// packed bf16 in registers while the S block feeds dV, then writes dM over the S block for dK and dQ.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSmallThreads = 128;
+constexpr uint32_t kSmallSmem = 4 * kBlkBytes + 2 * kBlkBytes + 1024;      // Q, K, V, dA + one S / dM block (+ alignment slack)
+
+struct SmallShared {
+    uint64_t bar_s, bar_o;
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+// What a thread needs to know about a problem before it can start its copies: the token counts, the global rows
+// (t / 8 + 16 i) whose 16-byte chunk t % 8 it copies on the query and on the key side, and the rows whose results it
+// stores.  Fetched one problem ahead, so that these dependent index loads never sit in front of the copies.
+struct SmallMeta {
+    int nq, nk;
+    int32_t qid[8], kid[8];       // -1: no such token (the row is zero-filled)
+    int32_t q_out, k_out;         // global row of query / key number threadIdx.x, -1 if there is none
+};
+__device__ __forceinline__ SmallMeta fetch_meta(const AttnParams& p, int prob) {
+    SmallMeta mt;
+    mt.nq = mt.nk = 0;
+    if (prob >= p.B * p.heads) return mt;
+    const int b = prob / p.heads;
+    const int base_row = b * p.N;
+    const int q0 = p.q_rows ? __ldg(p.q_offs + b) : 0, k0 = p.k_rows ? __ldg(p.k_offs + b) : 0;
+    mt.nq = p.q_rows ? __ldg(p.q_offs + b + 1) - q0 : p.N;
+    mt.nk = p.k_rows ? __ldg(p.k_offs + b + 1) - k0 : p.N;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = (threadIdx.x >> 3) + 16 * i;
+        mt.qid[i] = r < mt.nq ? (p.q_rows ? __ldg(p.q_rows + q0 + r) : base_row + r) : -1;
+        mt.kid[i] = r < mt.nk ? (p.k_rows ? __ldg(p.k_rows + k0 + r) : base_row + r) : -1;
+    }
+    const int r = threadIdx.x;
+    mt.q_out = r < mt.nq ? (p.q_rows ? __ldg(p.q_rows + q0 + r) : base_row + r) : -1;
+    mt.k_out = r < mt.nk ? (p.k_rows ? __ldg(p.k_rows + k0 + r) : base_row + r) : -1;
+    return mt;
+}
+// rows past `count` (up to the next multiple of 16, which is as far as the products step) become zeros
+__device__ __forceinline__ void load_rows_small(uint32_t dst, const __nv_bfloat16* src, int64_t ld, const int32_t (&id)[8], int count, int col0) {
+    const uint32_t chunk = threadIdx.x & 7u;
+    const int padded = (count + 15) & ~15;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = (threadIdx.x >> 3) + 16 * i;
+        if (r < padded)
+            ptx::cp_async_16(dst + swz((uint32_t)r, chunk), src + (id[i] >= 0 ? (int64_t)id[i] * ld + col0 + chunk * 8 : 0), id[i] >= 0 ? 16u : 0u);
+    }
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(const AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ SmallShared sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* gen = smem_raw + (base - raw);
+    const uint32_t sQ = base, sK = base + kBlkBytes, sV = base + 2 * kBlkBytes, sDA = base + 3 * kBlkBytes;
+    const uint32_t sP = base + 4 * kBlkBytes;              // [2 blocks of 64 keys][128 query rows][128 B]: S, later dM
+    uint8_t* gP = gen + 4 * kBlkBytes;
+    uint8_t* gV = gen + 2 * kBlkBytes;
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&sh.bar_s), 1);
+        ptx::mbar_init(ptx::smem_addr(&sh.bar_o), 1);
+        sh.abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 0) ptx::tmem_alloc(ptx::smem_addr(&sh.tmem_slot), 256);
+    // operand rows that a problem does not fill are still read by the products (they only reach accumulator rows nobody
+    // stores), so they must hold finite numbers: clear everything once
+    for (uint32_t w = threadIdx.x; w < 6 * kBlkBytes / 16; w += kSmallThreads) reinterpret_cast<uint4*>(gen)[w] = make_uint4(0u, 0u, 0u, 0u);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_slot);
+    volatile int* abort_flag = &sh.abort_flag;
+    pdl_wait();
+    const bool skip_all = p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0;
+
+    const int row = threadIdx.x;                            // accumulator row of this thread: a query, or a key in the dV / dK read-out
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const float sl2 = p.scale * 1.4426950408889634f;        // scores in base 2: e^x = 2^(x log2 e)
+    uint32_t n_s = 0, n_o = 0;
+    bool ok = !skip_all;
+    SmallMeta cur = fetch_meta(p, ok ? (int)blockIdx.x : p.B * p.heads);
+
+    for (int prob = blockIdx.x; ok && prob < p.B * p.heads; prob += gridDim.x) {
+        const int nq = cur.nq, nk = cur.nk;
+        const int col0 = (prob % p.heads) * kD;
+        const int32_t q_out = cur.q_out, k_out = cur.k_out;
+        if (nq > 0 && nk > 0) {
+            load_rows_small(sQ, p.Q, p.ld_qkv, cur.qid, nq, col0);
+            load_rows_small(sK, p.K, p.ld_qkv, cur.kid, nk, col0);
+            load_rows_small(sDA, p.dA, p.ld_da, cur.qid, nq, col0);
+            load_rows_small(sV, p.V, p.ld_qkv, cur.kid, nk, col0);
+        }
+        cur = fetch_meta(p, prob + (int)gridDim.x);          // the next problem's indices travel while this one computes
+        if (nq <= 0 || nk <= 0) continue;
+        const uint32_t q_steps = (uint32_t)(nq + 15) >> 4, k_steps = (uint32_t)(nk + 15) >> 4;   // 16-row steps that hold tokens
+        const uint32_t n_keys = k_steps * 16u;              // accumulator columns computed (a multiple of 16)
+        ptx::cp_async_wait_all();
+        ptx::fence_async_proxy();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            ptx::tc_fence_after_sync();
+            const uint32_t idesc = ptx::umma_idesc_bf16(128, (int)n_keys, false, false);
+#pragma unroll
+            for (uint32_t u = 0; u < 4; ++u) {              // the two products alternate: they fill different accumulators
+                ptx::umma_bf16(tmem, ptx::umma_desc_sw128(sQ + u * 32, 16, 1024), ptx::umma_desc_sw128(sK + u * 32, 16, 1024), idesc, u != 0);
+                ptx::umma_bf16(tmem + 128u, ptx::umma_desc_sw128(sDA + u * 32, 16, 1024), ptx::umma_desc_sw128(sV + u * 32, 16, 1024), idesc, u != 0);
+            }
+            ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
+        }
+        ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_s), n_s & 1u, abort_flag, p.status_word);
+        ++n_s;
+        ok = !__syncthreads_or(!ok);
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        // ---- this thread's row of S and dS, three sweeps over the accumulators: the maximum; the sum and
+        //      rowsum(e^(s - m) dS); then the S block to shared memory with dM kept in registers.  Columns from nk on
+        //      (padding keys, stale columns past n_keys) are masked; only the chunk holding column nk pays for it. ----
+        float mx = -INFINITY;
+        for (uint32_t c = 0; c < n_keys; c += 32) {
+            float s[32];
+            ptx::tmem_ld_32x32(tmem + c + lane_off, s);
+            ptx::tmem_ld_wait();
+            if ((int)c + 32 <= nk) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, s[j]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, ((int)c + j < nk) ? s[j] : -INFINITY);
+            }
+        }
+        const float nm = -mx * sl2;
+        float l = 0.f, u_acc = 0.f;
+        for (uint32_t c = 0; c < n_keys; c += 32) {
+            float s[32], ds[32];
+            ptx::tmem_ld_32x32(tmem + c + lane_off, s);
+            ptx::tmem_ld_32x32(tmem + 128u + c + lane_off, ds);
+            ptx::tmem_ld_wait();
+            const bool whole = (int)c + 32 <= nk;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                float e = ex2(fmaf(s[j], sl2, nm)), g = ds[j];
+                if (!whole) {                                // a stale column may hold anything, NaN included
+                    e = ((int)c + j < nk) ? e : 0.f;
+                    g = ((int)c + j < nk) ? g : 0.f;
+                }
+                l += e;
+                u_acc = fmaf(e, g, u_acc);
+            }
+        }
+        const float inv_l = 1.f / l;
+        const float nds = -u_acc * inv_l * p.scale;         // -rowsum(S dS) / sqrt(d)
+        uint32_t dm[64];
+#pragma unroll
+        for (uint32_t c = 0; c < 128; c += 32) {
+            if (c < n_keys) {
+                float s[32], ds[32];
+                ptx::tmem_ld_32x32(tmem + c + lane_off, s);
+                ptx::tmem_ld_32x32(tmem + 128u + c + lane_off, ds);
+                ptx::tmem_ld_wait();
+                const bool whole = (int)c + 32 <= nk;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float e = ex2(fmaf(s[j], sl2, nm)), g = ds[j];
+                    if (!whole) {
+                        e = ((int)c + j < nk) ? e : 0.f;
+                        g = ((int)c + j < nk) ? g : 0.f;
+                    }
+                    const float pj = e * inv_l;
+                    s[j] = pj;
+                    ds[j] = pj * fmaf(g, p.scale, nds);      // dM / sqrt(d)
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    *reinterpret_cast<uint4*>(gP + (c >> 6) * kBlkBytes + swz((uint32_t)row, ((c & 63u) >> 3) + q)) =
+                        make_uint4(pack2(s[q * 8], s[q * 8 + 1]), pack2(s[q * 8 + 2], s[q * 8 + 3]), pack2(s[q * 8 + 4], s[q * 8 + 5]), pack2(s[q * 8 + 6], s[q * 8 + 7]));
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) dm[(c >> 1) + q * 4 + e] = pack2(ds[q * 8 + 2 * e], ds[q * 8 + 2 * e + 1]);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) dm[(c >> 1) + e] = 0u;
+            }
+        }
+        ptx::fence_async_proxy();
+        ptx::tc_fence_before_sync();
+        __syncthreads();                                     // S and dS in tensor memory are dead from here on
+        if (threadIdx.x == 0) {
+            ptx::tc_fence_after_sync();
+            const uint32_t id_t = ptx::umma_idesc_bf16(128, 64, true, true);
+            for (uint32_t u = 0; u < q_steps; ++u)           // dV = S^T dA over the query rows
+                ptx::umma_bf16(tmem, ptx::umma_desc_sw128(sP + u * 2048, kBlkBytes, 1024), ptx::umma_desc_sw128(sDA + u * 2048, kBlkBytes, 1024), id_t, u != 0);
+            ptx::umma_commit(ptx::smem_addr(&sh.bar_o));
+        }
+        ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_o), n_o & 1u, abort_flag, p.status_word);
+        ++n_o;
+        ok = !__syncthreads_or(!ok);
+        if (!ok) break;
+        // ---- dM over the S block ----
+#pragma unroll
+        for (uint32_t c = 0; c < 128; c += 8)
+            if (c < n_keys)
+                *reinterpret_cast<uint4*>(gP + (c >> 6) * kBlkBytes + swz((uint32_t)row, (c & 63u) >> 3)) =
+                    make_uint4(dm[c >> 1], dm[(c >> 1) + 1], dm[(c >> 1) + 2], dm[(c >> 1) + 3]);
+        ptx::fence_async_proxy();
+        ptx::tc_fence_before_sync();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            ptx::tc_fence_after_sync();
+            const uint32_t id_t = ptx::umma_idesc_bf16(128, 64, true, true), id_q = ptx::umma_idesc_bf16(128, 64, false, true);
+            const uint32_t steps = q_steps > k_steps ? q_steps : k_steps;
+            for (uint32_t u = 0; u < steps; ++u) {           // dK = dM^T Q over the query rows, dQ = dM K over the keys, alternating
+                if (u < q_steps)
+                    ptx::umma_bf16(tmem + 64u, ptx::umma_desc_sw128(sP + u * 2048, kBlkBytes, 1024), ptx::umma_desc_sw128(sQ + u * 2048, kBlkBytes, 1024), id_t, u != 0);
+                if (u < k_steps)
+                    ptx::umma_bf16(tmem + 128u, ptx::umma_desc_sw128(sP + (u >> 2) * kBlkBytes + (u & 3u) * 32, 16, 1024),
+                                   ptx::umma_desc_sw128(sK + u * 2048, kBlkBytes, 1024), id_q, u != 0);
+            }
+            ptx::umma_commit(ptx::smem_addr(&sh.bar_o));
+        }
+        ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_o), n_o & 1u, abort_flag, p.status_word);
+        ++n_o;
+        ok = !__syncthreads_or(!ok);
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        // ---- read-out.  A thread holds one accumulator row (a key for dV and dK, a query for dQ), but a store that
+        //      touches 32 rows costs 32 transactions: each warp passes its 32 rows through shared memory (the S block's
+        //      two halves and the V operand are free by now) and writes four whole 128-byte rows per instruction. ----
+#pragma unroll
+        for (int which = 0; which < 3; ++which) {
+            uint8_t* stage = which == 0 ? gP : which == 1 ? gP + kBlkBytes : gV;
+#pragma unroll
+            for (int c = 0; c < 64; c += 32) {
+                float v[32];
+                ptx::tmem_ld_32x32(tmem + (uint32_t)(which * 64 + c) + lane_off, v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4*>(stage + swz((uint32_t)row, (uint32_t)(c / 8 + q))) =
+                        make_uint4(pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]), pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int which = 0; which < 3; ++which) {
+            const uint8_t* stage = which == 0 ? gP : which == 1 ? gP + kBlkBytes : gV;
+            __nv_bfloat16* out = (which == 0 ? p.dV : which == 1 ? p.dK : p.dQ) + col0 + (lane & 7) * 8;
+            const int32_t mine = which == 2 ? q_out : k_out;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = i * 4 + (lane >> 3);                                   // row within this warp's 32
+                const int32_t g = __shfl_sync(0xffffffffu, mine, r);
+                const uint4 pk = *reinterpret_cast<const uint4*>(stage + swz((uint32_t)(warp * 32 + r), (uint32_t)(lane & 7)));
+                if (g >= 0) ptx::st_global_v4(out + (int64_t)g * p.ld_out, pk.x, pk.y, pk.z, pk.w);
+            }
+        }
+        ptx::tc_fence_before_sync();
+        __syncthreads();                                     // operands, stages and accumulators are free for the next problem
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, 256);
+    }
+}
+
+// rows of an output [M, ld] (columns [0, cols)) that are not in its ascending list rows[0 .. *total) become +0.0:
+// entry m of the list owns the gap in front of it, one extra worker the tail; blockIdx.y picks the output
+struct ZeroJob {
+    __nv_bfloat16* out[3];
+    const int32_t* rows[3];
+    const int32_t* total[3];
+};
+__global__ void zero_rows_outside_kernel(const ZeroJob job, int64_t M, int64_t ld, int cols, const int32_t* status_word) {
     pdl_launch_dependents();
     pdl_wait();
     if (status_word != nullptr && *reinterpret_cast<const volatile int32_t*>(status_word) != 0) return;
-    const int64_t total = __ldg(total_dev);
+    const int32_t* rows = job.rows[blockIdx.y];
+    if (rows == nullptr) return;
+    __nv_bfloat16* out = job.out[blockIdx.y];
+    const int64_t total = __ldg(job.total[blockIdx.y]);
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     for (int64_t m = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); m <= total; m += warps) {
@@ -340,10 +631,8 @@ int64_t attention_max_tokens() { return kMaxTok; }
 
 cudaError_t launch_attention_backward(const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA, int64_t ld_da,
                                       const int32_t* q_rows, const int32_t* q_offs, const int32_t* k_rows, const int32_t* k_offs,
-                                      int64_t B, int64_t N, int64_t heads, void* dQ, void* dK, void* dV, int64_t ld_out,
-                                      int32_t* status_word, cudaStream_t stream) {
-    const cudaError_t opt = opt_in_dynamic_smem<attention_bwd_kernel>((int)kAttnSmem);
-    if (opt != cudaSuccess) return opt;
+                                      int64_t B, int64_t N, int64_t heads, int64_t most_tokens, void* dQ, void* dK, void* dV,
+                                      int64_t ld_out, int32_t* status_word, cudaStream_t stream) {
     AttnParams prm;
     prm.Q = static_cast<const __nv_bfloat16*>(Q); prm.K = static_cast<const __nv_bfloat16*>(K);
     prm.V = static_cast<const __nv_bfloat16*>(V); prm.dA = static_cast<const __nv_bfloat16*>(dA);
@@ -354,21 +643,25 @@ cudaError_t launch_attention_backward(const void* Q, const void* K, const void* 
     prm.scale = 1.0f / sqrtf((float)kD);
     prm.status_word = status_word;
     const int64_t problems = B * heads;
-    const dim3 grid((unsigned)(problems < kNumSMs ? problems : kNumSMs));
-    cudaError_t e = cudaSuccess;
-    const int cols = (int)(heads * kD);
     // the zeros first: they touch only rows outside the lists, the products only rows inside them
-    if (q_rows != nullptr)
-        e = launch_pdl(zero_rows_outside_kernel, dim3(2 * kNumSMs), dim3(256), 0, stream, prm.dQ, B * N, ld_out, cols, q_rows,
-                       q_offs + B, (const int32_t*)status_word);
-    if (e == cudaSuccess && k_rows != nullptr) {
-        e = launch_pdl(zero_rows_outside_kernel, dim3(2 * kNumSMs), dim3(256), 0, stream, prm.dK, B * N, ld_out, cols, k_rows,
-                       k_offs + B, (const int32_t*)status_word);
-        if (e == cudaSuccess)
-            e = launch_pdl(zero_rows_outside_kernel, dim3(2 * kNumSMs), dim3(256), 0, stream, prm.dV, B * N, ld_out, cols, k_rows,
-                           k_offs + B, (const int32_t*)status_word);
+    if (q_rows != nullptr || k_rows != nullptr) {
+        ZeroJob job;
+        job.out[0] = prm.dQ; job.rows[0] = q_rows; job.total[0] = q_rows ? q_offs + B : nullptr;
+        job.out[1] = prm.dK; job.rows[1] = k_rows; job.total[1] = k_rows ? k_offs + B : nullptr;
+        job.out[2] = prm.dV; job.rows[2] = k_rows; job.total[2] = k_rows ? k_offs + B : nullptr;
+        const cudaError_t e = launch_pdl(zero_rows_outside_kernel, dim3(kNumSMs, 3), dim3(256), 0, stream, job, B * N, ld_out,
+                                         (int)(heads * kD), (const int32_t*)status_word);
+        if (e != cudaSuccess) return e;
     }
-    if (e != cudaSuccess) return e;
+    if (most_tokens <= 128) {
+        const cudaError_t opt = opt_in_dynamic_smem<attention_bwd_small_kernel>((int)kSmallSmem);
+        if (opt != cudaSuccess) return opt;
+        const dim3 grid((unsigned)(problems < 2 * kNumSMs ? problems : 2 * kNumSMs));
+        return launch_pdl(attention_bwd_small_kernel, grid, dim3(kSmallThreads), kSmallSmem, stream, prm);
+    }
+    const cudaError_t opt = opt_in_dynamic_smem<attention_bwd_kernel>((int)kAttnSmem);
+    if (opt != cudaSuccess) return opt;
+    const dim3 grid((unsigned)(problems < kNumSMs ? problems : kNumSMs));
     return launch_pdl(attention_bwd_kernel, grid, dim3(kAttnThreads), kAttnSmem, stream, prm);
 }
 

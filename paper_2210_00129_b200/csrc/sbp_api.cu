@@ -362,8 +362,8 @@ sbp_status sbp_attention_backward(sbp_dtype dt, const void* Q, const void* K, co
     if (any_list && (max_kept <= 0 || max_kept > N)) return SBP_ERR_INVALID_ARG;
     const int64_t most = any_all ? N : max_kept;
     if (most > attention_max_tokens()) return SBP_ERR_UNSUPPORTED;
-    const cudaError_t e = launch_attention_backward(Q, K, V, ld_qkv, dA, ld_da, q_rows, q_offsets, k_rows, k_offs, B, N, heads, dQ,
-                                                    dK, dV, ld_out, status_word, (cudaStream_t)stream);
+    const cudaError_t e = launch_attention_backward(Q, K, V, ld_qkv, dA, ld_da, q_rows, q_offsets, k_rows, k_offs, B, N, heads, most,
+                                                    dQ, dK, dV, ld_out, status_word, (cudaStream_t)stream);
     return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
 }
 
