@@ -13,6 +13,7 @@
  *   sbp_linear_backward  dW = X_keep^T dY_keep, db = sum dY_keep,
  *                        dX = scatter(dY_keep W^T), zeros elsewhere   (Eq. 5)
  *   sbp_attention_backward  dQ, dK, dV of attention on the kept tokens (Sec. 4, Drop QKV / Drop Query only)
+ *   sbp_patch_cache / sbp_patch_scatter  stride >= kernel convolutions as linear layers on patch rows (Sec. 3.2.2)
  *
  * Nothing is rescaled by 1/r: Eq. 1 keeps the plain 1/B factor.
  *
@@ -231,6 +232,37 @@ sbp_status sbp_linear_backward(sbp_dtype dt,
 int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                      int64_t C_out, int want_dW, int want_db, int want_dX,
                                      uint32_t flags);
+
+/*
+ * Convolutions with stride >= kernel size as SBP layers (Sec. 3.2.2, the text after Eq. 6: with s >= k the
+ * neighbour effect disappears and the layer behaves like a point-wise one; ConvNeXt's 2 x 2 / stride 2
+ * down-sampling layers, Sec. 5).  Channels-last X [B, H, W, C], weights [k, k, C, C_out] = a [k*k*C, C_out]
+ * matrix, output grid Ho = (H - k) / stride + 1, Wo = (W - k) / stride + 1 (no padding); keep_rows are kept
+ * OUTPUT positions (b*Ho + ho)*Wo + wo, as sbp_sample_keep draws them on an Ho x Wo map.  Each output position
+ * reads its own k x k patch, so the layer is a linear layer on patch rows of k*k*C values (ordered dh, dw, c):
+ *
+ *   sbp_patch_cache     X_keep[m, (dh, dw, c)] = X[b, stride*ho + dh, stride*wo + dw, c]  for kept m = (b, ho, wo);
+ *                       [M_keep_cap, k*k*C], rows past M_keep zeroed: the forward cache (Algorithm 1)
+ *   sbp_linear_backward with C_in = k*k*C on X_keep, dY [B*Ho*Wo, C_out] and SBP_FLAG_DX_COMPACT: dW, db and the
+ *                       packed input gradient dX_patches [M_keep_cap, k*k*C]
+ *   sbp_patch_scatter   dX[b, stride*ho + dh, stride*wo + dw, c] = dX_patches[m, (dh, dw, c)] for kept m; every
+ *                       other input position (dropped patches, positions no patch covers) = +0.0.  Every element
+ *                       of dX is written exactly once.  workspace: sbp_patch_scatter_workspace_bytes(...) bytes,
+ *                       256-byte aligned (one int32 per output position).
+ * C * sizeof(element) must be a multiple of 16 (else SBP_ERR_UNSUPPORTED); stride < k, k larger than the map and
+ * other bad sizes or pointers give SBP_ERR_INVALID_ARG; a short workspace SBP_ERR_WORKSPACE.  M_keep is
+ * *M_keep_dev when given, else M_keep_cap.  Bit-exact copies; deterministic.
+ */
+sbp_status sbp_patch_cache(sbp_dtype dt, const void* X /* dev */, int64_t B, int64_t H, int64_t W, int64_t C,
+                           int64_t k, int64_t stride, const int32_t* keep_rows /* dev */,
+                           const int32_t* M_keep_dev /* dev, nullable */, int64_t M_keep_cap, void* X_keep /* dev */,
+                           void* stream);
+size_t sbp_patch_scatter_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t k, int64_t stride);
+sbp_status sbp_patch_scatter(sbp_dtype dt, const void* dX_patches /* dev */, int64_t B, int64_t H, int64_t W, int64_t C,
+                             int64_t k, int64_t stride, const int32_t* keep_rows /* dev */,
+                             const int32_t* M_keep_dev /* dev, nullable */, int64_t M_keep_cap, void* dX /* dev */,
+                             void* workspace /* dev */, size_t workspace_bytes, int32_t* status_word /* dev, nullable */,
+                             void* stream);
 
 /*
  * SBP backward of multi-head scaled dot-product attention (Sec. 4, "How to apply SBP on MHSA?"; supplementary,

@@ -67,6 +67,10 @@ def _load():
     lib.oracle_attention_backward.restype = None
     lib.oracle_attention_memory_ratio.argtypes = [ctypes.c_int, dbl, dbl, dbl]
     lib.oracle_attention_memory_ratio.restype = dbl
+    lib.oracle_patch_conv_forward.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, vp]
+    lib.oracle_patch_conv_forward.restype = None
+    lib.oracle_patch_conv_backward.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp, vp, vp]
+    lib.oracle_patch_conv_backward.restype = None
     lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
     lib.oracle_set_num_threads.restype = None
     lib.oracle_num_threads.argtypes = []
@@ -208,3 +212,30 @@ def attention_backward(Q, K, V, dA, q_rows, q_offs, k_rows, k_offs, heads):
 
 def attention_memory_ratio(mode: int, d: float, n: float, r: float) -> float:
     return float(_load().oracle_attention_memory_ratio(mode, float(d), float(n), float(r)))
+
+
+def patch_conv_forward(X, Wt, bias, k, stride):
+    """Y [B, Ho, Wo, Co] of a k x k convolution with stride >= k, channels last, no padding (fp64)."""
+    X, Wt = _f64(X), _f64(Wt)
+    B, H, W, C = X.shape
+    Co = Wt.shape[3]
+    assert Wt.shape == (k, k, C, Co) and stride >= k
+    b = _f64(bias) if bias is not None else None
+    Y = np.empty((B, (H - k) // stride + 1, (W - k) // stride + 1, Co))
+    _load().oracle_patch_conv_forward(_ptr(X), _ptr(Wt), _ptr(b), B, H, W, C, Co, k, stride, _ptr(Y))
+    return Y
+
+
+def patch_conv_backward(X, dY, Wt, keep_rows, k, stride, want=("dW", "db", "dX")):
+    """SBP backward of that layer with dY kept on the listed output positions (ids (b*Ho + ho)*Wo + wo)."""
+    X, dY, Wt = _f64(X), _f64(dY), _f64(Wt)
+    B, H, W, C = X.shape
+    Co = Wt.shape[3]
+    rows = np.ascontiguousarray(keep_rows, dtype=np.int32)
+    assert dY.shape == (B, (H - k) // stride + 1, (W - k) // stride + 1, Co) and stride >= k
+    dW = np.empty((k, k, C, Co)) if "dW" in want else None
+    db = np.empty(Co) if "db" in want else None
+    dX = np.empty((B, H, W, C)) if "dX" in want else None
+    _load().oracle_patch_conv_backward(_ptr(X), _ptr(dY), _ptr(Wt), _ptr(rows), rows.shape[0], B, H, W, C, Co, k, stride,
+                                       _ptr(dW), _ptr(db), _ptr(dX))
+    return {n: v for n, v in (("dW", dW), ("db", db), ("dX", dX)) if v is not None}

@@ -549,3 +549,69 @@ double oracle_attention_memory_ratio(int mode, double d, double n, double r)
     if (mode == 0) return ((2.0 + r) * d * n + 2.0 * r * n * n) / full;
     return (3.0 * r * d * n + 2.0 * r * r * n * n) / full;
 }
+
+/* ------------------------------------------------------------------ */
+/* Convolution with stride >= kernel size under SBP (Sec. 3.2.2, the   */
+/* text after Eq. 6: with s >= k the neighbour effect disappears and   */
+/* the layer behaves like a point-wise one; ConvNeXt's 2 x 2 / stride 2 */
+/* down-sampling layers, Sec. 5)                                        */
+/* ------------------------------------------------------------------ */
+/*
+ * Channels-last tensors: X [B, H, W, C], weights Wt [k, k, C, Co], Y and dY [B, Ho, Wo, Co] with
+ * Ho = (H - k) / s + 1, Wo = (W - k) / s + 1 (no padding), s >= k:
+ *   Y[b, ho, wo, j] = sum_{dh, dw, c} X[b, s ho + dh, s wo + dw, c] Wt[dh, dw, c, j] (+ bias[j])
+ * Every output position reads its own k x k patch; patches of different output positions do not overlap.
+ * Backward (Eq. 6 written out for this case) with dY dropped outside the kept output positions
+ * (keep_rows: ascending global ids (b Ho + ho) Wo + wo):
+ *   dW[dh, dw, c, j] = sum_{kept m} X[patch of m at (dh, dw), c] dY[m, j]
+ *   db[j]            = sum_{kept m} dY[m, j]
+ *   dX[patch of m at (dh, dw), c] = sum_j dY[m, j] Wt[dh, dw, c, j]   for kept m; every other input position +0.0
+ */
+void oracle_patch_conv_forward(const double* X, const double* Wt, const double* bias, int64_t B, int64_t H,
+                               int64_t W, int64_t C, int64_t Co, int64_t k, int64_t s, double* Y)
+{
+    const int64_t Ho = (H - k) / s + 1, Wo = (W - k) / s + 1;
+#pragma omp parallel for collapse(2)
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t ho = 0; ho < Ho; ++ho)
+            for (int64_t wo = 0; wo < Wo; ++wo) {
+                double* y = Y + ((b * Ho + ho) * Wo + wo) * Co;
+                for (int64_t j = 0; j < Co; ++j) y[j] = bias ? bias[j] : 0.0;
+                for (int64_t dh = 0; dh < k; ++dh)
+                    for (int64_t dw = 0; dw < k; ++dw) {
+                        const double* x = X + ((b * H + s * ho + dh) * W + s * wo + dw) * C;
+                        const double* w = Wt + (dh * k + dw) * C * Co;
+                        for (int64_t c = 0; c < C; ++c)
+                            for (int64_t j = 0; j < Co; ++j) y[j] += x[c] * w[c * Co + j];
+                    }
+            }
+}
+
+void oracle_patch_conv_backward(const double* X, const double* dY, const double* Wt, const int32_t* keep_rows,
+                                int64_t M_keep, int64_t B, int64_t H, int64_t W, int64_t C, int64_t Co,
+                                int64_t k, int64_t s, double* dW, double* db, double* dX)
+{
+    const int64_t Ho = (H - k) / s + 1, Wo = (W - k) / s + 1;
+    if (dW) for (int64_t e = 0; e < k * k * C * Co; ++e) dW[e] = 0.0;
+    if (db) for (int64_t j = 0; j < Co; ++j) db[j] = 0.0;
+    if (dX) for (int64_t e = 0; e < B * H * W * C; ++e) dX[e] = 0.0;
+    for (int64_t m = 0; m < M_keep; ++m) {
+        const int64_t g = keep_rows[m];
+        const int64_t b = g / (Ho * Wo), ho = (g / Wo) % Ho, wo = g % Wo;
+        const double* dy = dY + g * Co;
+        if (db) for (int64_t j = 0; j < Co; ++j) db[j] += dy[j];
+        for (int64_t dh = 0; dh < k; ++dh)
+            for (int64_t dw = 0; dw < k; ++dw) {
+                const int64_t pix = (b * H + s * ho + dh) * W + s * wo + dw;
+                const double* w = Wt + (dh * k + dw) * C * Co;
+                for (int64_t c = 0; c < C; ++c) {
+                    if (dW) for (int64_t j = 0; j < Co; ++j) dW[((dh * k + dw) * C + c) * Co + j] += X[pix * C + c] * dy[j];
+                    if (dX) {
+                        double acc = 0.0;
+                        for (int64_t j = 0; j < Co; ++j) acc += dy[j] * w[c * Co + j];
+                        dX[pix * C + c] = acc;
+                    }
+                }
+            }
+    }
+}

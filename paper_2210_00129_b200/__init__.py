@@ -26,7 +26,8 @@ SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT, SBP_FLAG_W_OUT_IN, SBP_FLAG_ATTN_ALL_K
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
-           "sbp_plan_search_count", "sbp_attention_backward", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
+           "sbp_plan_search_count", "sbp_attention_backward", "sbp_patch_cache", "sbp_patch_scatter_workspace_bytes",
+           "sbp_patch_scatter", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
            "sbp_selftest_bounded_wait")
 
 _lib = None
@@ -70,6 +71,12 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_attention_backward.argtypes = [ci, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, i64, i64, i64, i64, i64, vp, vp, vp, i64,
                                            u32, vp, vp]
     lib.sbp_attention_backward.restype = ci
+    lib.sbp_patch_cache.argtypes = [ci, vp, i64, i64, i64, i64, i64, i64, vp, vp, i64, vp, vp]
+    lib.sbp_patch_cache.restype = ci
+    lib.sbp_patch_scatter_workspace_bytes.argtypes = [i64, i64, i64, i64, i64]
+    lib.sbp_patch_scatter_workspace_bytes.restype = sz
+    lib.sbp_patch_scatter.argtypes = [ci, vp, i64, i64, i64, i64, i64, i64, vp, vp, i64, vp, vp, sz, vp, vp]
+    lib.sbp_patch_scatter.restype = ci
     lib.sbp_plan_search_count.argtypes = []
     lib.sbp_plan_search_count.restype = i64
     lib.sbp_step_host_arena_bytes.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl]
@@ -172,6 +179,30 @@ def sbp_attention_backward(dt, Q, K, V, ld_qkv, dA, ld_da, q_rows, q_offsets, kv
                                               _stream(stream))
     if check:
         _check(s, "sbp_attention_backward")
+    return s
+
+
+def sbp_patch_cache(dt, X, B, H, W, C, k, stride, keep_rows, M_keep_dev, M_keep_cap, X_keep, stream=None, check=True) -> int:
+    """Forward cache of a stride >= kernel convolution: the kept output positions' k x k patches as rows of k*k*C values."""
+    s = load_library().sbp_patch_cache(dt, _ptr(X), B, H, W, C, k, stride, _ptr(keep_rows), _ptr(M_keep_dev), M_keep_cap,
+                                       _ptr(X_keep), _stream(stream))
+    if check:
+        _check(s, "sbp_patch_cache")
+    return s
+
+
+def sbp_patch_scatter_workspace_bytes(B, H, W, k, stride) -> int:
+    return int(load_library().sbp_patch_scatter_workspace_bytes(B, H, W, k, stride))
+
+
+def sbp_patch_scatter(dt, dX_patches, B, H, W, C, k, stride, keep_rows, M_keep_dev, M_keep_cap, dX, workspace, workspace_bytes,
+                      status_word=None, stream=None, check=True) -> int:
+    """Packed patch gradients [M_keep_cap, k*k*C] back into dX [B, H, W, C], zeros everywhere else."""
+    s = load_library().sbp_patch_scatter(dt, _ptr(dX_patches), B, H, W, C, k, stride, _ptr(keep_rows), _ptr(M_keep_dev),
+                                         M_keep_cap, _ptr(dX), _ptr(workspace), workspace_bytes, _ptr(status_word),
+                                         _stream(stream))
+    if check:
+        _check(s, "sbp_patch_scatter")
     return s
 
 

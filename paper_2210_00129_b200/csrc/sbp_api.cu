@@ -331,6 +331,56 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
 
 int64_t sbp_plan_search_count(void) { return tc_plan_searches(); }
 
+namespace {
+// shared argument checks of the two patch calls; returns SBP_OK and the output grid when the geometry is usable
+sbp_status patch_geometry(sbp_dtype dt, int64_t B, int64_t H, int64_t W, int64_t C, int64_t k, int64_t stride, int64_t M_keep_cap,
+                          int64_t* Ho, int64_t* Wo) {
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || k <= 0 || stride < k || k > H || k > W) return SBP_ERR_INVALID_ARG;
+    if (B * H * W >= (1ll << 31) || C >= (1ll << 24) || k > 64) return SBP_ERR_INVALID_ARG;
+    *Ho = (H - k) / stride + 1;
+    *Wo = (W - k) / stride + 1;
+    if (M_keep_cap < 0 || M_keep_cap > B * *Ho * *Wo) return SBP_ERR_INVALID_ARG;
+    if ((C * (dt == SBP_BF16 ? 2 : 4)) % 16 != 0) return SBP_ERR_UNSUPPORTED;
+    return SBP_OK;
+}
+}  // namespace
+
+sbp_status sbp_patch_cache(sbp_dtype dt, const void* X, int64_t B, int64_t H, int64_t W, int64_t C, int64_t k, int64_t stride,
+                           const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap, void* X_keep, void* stream) {
+    int64_t Ho = 0, Wo = 0;
+    const sbp_status g = patch_geometry(dt, B, H, W, C, k, stride, M_keep_cap, &Ho, &Wo);
+    if (g != SBP_OK) return g;
+    if (X == nullptr || X_keep == nullptr || keep_rows == nullptr || !aligned16(X) || !aligned16(X_keep) ||
+        (reinterpret_cast<uintptr_t>(keep_rows) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    const cudaError_t e = launch_patch_gather(X, H, W, C * (dt == SBP_BF16 ? 2 : 4), k, stride, keep_rows, M_keep_dev, M_keep_cap,
+                                              X_keep, (cudaStream_t)stream);
+    return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
+size_t sbp_patch_scatter_workspace_bytes(int64_t B, int64_t H, int64_t W, int64_t k, int64_t stride) {
+    if (B <= 0 || H <= 0 || W <= 0 || k <= 0 || stride < k || k > H || k > W) return 256;
+    return align_up((size_t)(B * ((H - k) / stride + 1) * ((W - k) / stride + 1)) * sizeof(int32_t), 256);
+}
+
+sbp_status sbp_patch_scatter(sbp_dtype dt, const void* dX_patches, int64_t B, int64_t H, int64_t W, int64_t C, int64_t k,
+                             int64_t stride, const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap, void* dX,
+                             void* workspace, size_t workspace_bytes, int32_t* status_word, void* stream) {
+    int64_t Ho = 0, Wo = 0;
+    const sbp_status g = patch_geometry(dt, B, H, W, C, k, stride, M_keep_cap, &Ho, &Wo);
+    if (g != SBP_OK) return g;
+    if (dX_patches == nullptr || dX == nullptr || keep_rows == nullptr || !aligned16(dX_patches) || !aligned16(dX) ||
+        (reinterpret_cast<uintptr_t>(keep_rows) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < sbp_patch_scatter_workspace_bytes(B, H, W, k, stride))
+        return SBP_ERR_WORKSPACE;
+    const cudaError_t e = launch_patch_scatter(dX_patches, B, H, W, C * (dt == SBP_BF16 ? 2 : 4), k, stride, keep_rows, M_keep_dev,
+                                               M_keep_cap, dX, static_cast<int32_t*>(workspace), status_word, (cudaStream_t)stream);
+    return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
 sbp_status sbp_attention_backward(sbp_dtype dt, const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA,
                                   int64_t ld_da, const int32_t* q_rows, const int32_t* q_offsets, const int32_t* kv_rows,
                                   const int32_t* kv_offsets, int64_t B, int64_t N, int64_t heads, int64_t head_dim,

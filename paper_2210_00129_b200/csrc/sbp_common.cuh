@@ -187,6 +187,14 @@ sbp_status launch_tc_forward(const void* X, const void* W, bool w_out_in, const 
                              void* Y, const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap,
                              void* X_keep, int32_t* status_word, cudaStream_t stream);
 
+// stride >= kernel convolutions as linear layers on patch rows: gather of the kept patches, scatter of their gradients
+cudaError_t launch_patch_gather(const void* X, int64_t H, int64_t W, int64_t pos_bytes, int64_t k, int64_t s,
+                                const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap, void* X_keep,
+                                cudaStream_t stream);
+cudaError_t launch_patch_scatter(const void* dXp, int64_t B, int64_t H, int64_t W, int64_t pos_bytes, int64_t k, int64_t s,
+                                 const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap, void* dX,
+                                 int32_t* slot, const int32_t* status_word, cudaStream_t stream);
+
 // SBP attention backward on token subsets (bf16, head dimension 64, at most attention_max_tokens() kept tokens per sample
 // and side); null row lists mean every token of the sample
 bool    attention_supported(sbp_dtype dt, int64_t head_dim);
