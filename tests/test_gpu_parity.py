@@ -300,3 +300,19 @@ def test_bounded_wait_gives_up_reports_and_leaves_the_stream_usable():
     assert np.array_equal(host(offs), want_offs) and np.array_equal(host(rows)[:len(want_rows)], want_rows)
     assert sbp.sbp_selftest_bounded_wait(0.0, status, completed, check=False) == sbp.SBP_ERR_INVALID_ARG
     assert sbp.sbp_selftest_bounded_wait(5000.0, status, completed, check=False) == sbp.SBP_ERR_INVALID_ARG
+
+
+@pytest.mark.skipif(torch.cuda.device_count() < 2, reason="needs two GPUs in one process")
+def test_one_process_drives_two_devices():
+    # the opt-in for large dynamic shared memory belongs to the (kernel, device) pair: a tensor-core backward on
+    # device 0 and then on device 1 from the same process must both launch (no peer memory, no collective)
+    M, X, Wt, dY, keep = _case("bf16", 4, 14, 14, 256, 384, 0.5)
+    want = oracle.linear_backward(synth.to_f64(oracle.forward_cache(X, keep), "bf16"), synth.to_f64(dY, "bf16"),
+                                  synth.to_f64(Wt, "bf16"), keep)
+    for d in (0, 1):
+        with torch.cuda.device(d):
+            rows_d = torch.from_numpy(keep).cuda()
+            Xk_d = run_forward_cache("bf16", dev(X, "bf16"), rows_d, len(keep))
+            got = run_backward("bf16", Xk_d, dev(dY, "bf16"), dev(Wt, "bf16"), rows_d, len(keep))
+            assert got["status"] == 0
+            assert relerr(host(got["dW"]), want["dW"]) <= 5e-3 and relerr(synth.to_f64(host(got["dX"]), "bf16"), want["dX"]) <= 5e-3
