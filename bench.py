@@ -10,6 +10,7 @@ the single fc1 layer at B=64.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
     python bench.py --sweep all|vit|convnext|detection|forward|blocks|attention|sampler [--iters 24]
+    python bench.py --probe
 
 Prints one JSON line (rank 0).  ``value`` counts the backward FLOPs of the kept rows
 (4 * M_keep * C_in * C_out per layer, step and GPU) over device time, with inputs resident in HBM;
@@ -967,6 +968,56 @@ def run_sweep(args):
 
 
 
+def run_probes(args):
+    """Tables of the two diagnostic probes of the library: what the cp.async gather path sustains, and what a
+    tcgen05.mma of a given width costs."""
+    import torch
+    import paper_2210_00129_b200 as sbp
+    from paper_2210_00129_b200 import build as sbp_build
+    sbp_build.build()
+    sbp.load_library()
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def time_us(fn, reps=5):
+        best = 1e30
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1) * 1e3)
+        return best
+
+    print("| gather of random rows (every other row kept) | source | rows x bytes | blocks | copy threads | ring | us | GB/s | GB/s per SM |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    for source, M, rb, reps in (("DRAM (205 MB)", 200704, 1024, 1), ("DRAM (51 MB of 256-byte rows)", 200704, 256, 1), ("L2 (24 MB)", 24576, 1024, 8)):
+        src = torch.ones(M * rb, dtype=torch.uint8, device="cuda")
+        lists = [torch.nonzero(torch.rand(M, device="cuda", generator=gen) < 0.5).flatten().to(torch.int32) for _ in range(reps)]
+        rows = torch.cat(lists).contiguous()
+        n = int(rows.numel())
+        for blocks in (148, 74, 37):
+            for threads, stages in ((64, 6), (128, 6), (256, 12)):
+                us = time_us(lambda: sbp.sbp_probe_gather_ring(src, rb, rows, n, threads, stages, blocks, st))
+                gbs = n * rb / us / 1e3
+                print(f"| | {source} | {n} x {rb} | {blocks} | {threads} | {stages} x 16 KB | {us:.1f} | {gbs:.0f} | {gbs / blocks:.1f} |")
+        del src
+    print("\n| tcgen05.mma, M = 128, K = 16, bf16 | operands | N | accumulators | clocks per instruction | clocks per 64-deep k-block | ideal (4096 MAC/clk) | fraction |")
+    print("|---|---|---|---|---|---|---|---|")
+    cyc = torch.zeros(1, dtype=torch.int64, device="cuda")
+    iters = 2000
+    for blocks in (1, 148):
+        for mn in (0, 1):
+            for acc in (1, 2):
+                for N in (16, 32, 64, 128, 192, 256):
+                    sbp.sbp_probe_mma_rate(N, mn, acc, iters, blocks, cyc, st)
+                    sbp.sbp_probe_mma_rate(N, mn, acc, iters, blocks, cyc, st)
+                    torch.cuda.synchronize()
+                    c = int(cyc.item())
+                    per_kb = c / iters / acc                      # per accumulator chain and k-block
+                    ideal = 128.0 * N * 64 / 4096.0
+                    print(f"| {blocks} block(s) | {'MN-major' if mn else 'K-major'} | {N} | {acc} | {c / (iters * 4 * acc):.1f} | {per_kb:.0f} | {ideal:.0f} | {ideal / per_kb:.2f} |")
+    assert int(st.item()) == 0, "device status word set by a probe"
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -982,7 +1033,11 @@ def main():
                     help="print per-call timing tables of every layer shape of a group instead of the JSON line")
     ap.add_argument("--iters", type=int, default=24, help="--sweep: launches per figure")
     ap.add_argument("--compact", action="store_true", help="--sweep: one table row per layer, us (t_min / t) per call")
+    ap.add_argument("--probe", action="store_true", help="print the tables of the library's diagnostic probes (gather ring, tcgen05.mma rate)")
     args = ap.parse_args()
+    if args.probe:
+        run_probes(args)
+        return
     if args.sweep:
         run_sweep(args)
         return

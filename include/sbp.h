@@ -369,6 +369,26 @@ sbp_status sbp_bias_grad_static(sbp_dtype dt, const void* dY /* dev */, const in
 sbp_status sbp_selftest_bounded_wait(double limit_ms, int32_t* status_word /* dev */,
                                      int32_t* completed /* dev */, void* stream);
 
+/*
+ * Diagnostic probes (no counterpart in the paper): micro-measurements of the machinery the tensor-core kernels are
+ * built from; `python bench.py --probe` prints their tables.  The caller times the calls with events.
+ *
+ * sbp_probe_gather_ring: copies the rows `rows[0 .. n_rows)` (each an index of a row of `row_bytes` bytes in `src`,
+ *   row_bytes a multiple of 128; the indices must lie inside src) with 16-byte cp.async into a ring of `stages`
+ *   (2..12) 16 KB shared-memory stages per block, `threads` (64, 128 or 256) copying threads and `blocks` blocks, the
+ *   way the backward kernel gathers the kept rows of dY; a consumer frees each stage as it lands.  Nothing is written
+ *   to global memory.
+ * sbp_probe_mma_rate: one thread per block issues 4 * iters tcgen05.mma (M = 128, K = 16, bf16, width N a multiple of
+ *   16 up to 256, operands K-major or MN-major) into one accumulator, or alternating between two accumulators 256
+ *   columns apart (accumulators = 2: 8 * iters instructions); cycles_out[0] (dev) receives the SM clocks from the
+ *   first issue to the completion of the last instruction on block 0, or -1 if the bounded wait ran out.
+ * SBP_ERR_INVALID_ARG for sizes outside these ranges and null / misaligned pointers.
+ */
+sbp_status sbp_probe_gather_ring(const void* src /* dev */, int64_t row_bytes, const int32_t* rows /* dev */, int64_t n_rows,
+                                 int threads, int stages, int blocks, int32_t* status_word /* dev, nullable */, void* stream);
+sbp_status sbp_probe_mma_rate(int N, int mn_major, int accumulators, int iters, int blocks, int64_t* cycles_out /* dev */,
+                              int32_t* status_word /* dev, nullable */, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

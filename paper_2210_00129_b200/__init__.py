@@ -28,7 +28,7 @@ EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forwar
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
            "sbp_plan_search_count", "sbp_attention_backward", "sbp_patch_cache", "sbp_patch_scatter_workspace_bytes",
            "sbp_patch_scatter", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
-           "sbp_selftest_bounded_wait")
+           "sbp_selftest_bounded_wait", "sbp_probe_gather_ring", "sbp_probe_mma_rate")
 
 _lib = None
 
@@ -77,6 +77,10 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_patch_scatter_workspace_bytes.restype = sz
     lib.sbp_patch_scatter.argtypes = [ci, vp, i64, i64, i64, i64, i64, i64, vp, vp, i64, vp, vp, sz, vp, vp]
     lib.sbp_patch_scatter.restype = ci
+    lib.sbp_probe_gather_ring.argtypes = [vp, i64, vp, i64, ci, ci, ci, vp, vp]
+    lib.sbp_probe_gather_ring.restype = ci
+    lib.sbp_probe_mma_rate.argtypes = [ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.sbp_probe_mma_rate.restype = ci
     lib.sbp_plan_search_count.argtypes = []
     lib.sbp_plan_search_count.restype = i64
     lib.sbp_step_host_arena_bytes.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl]
@@ -234,6 +238,24 @@ def sbp_bias_grad_static(dt, dY, keep_rows, M_keep_dev, M, M_keep_cap, C_out, db
                                             _ptr(db), flags, _stream(stream))
     if check:
         _check(s, "sbp_bias_grad_static")
+    return s
+
+
+def sbp_probe_gather_ring(src, row_bytes, rows, n_rows, threads, stages, blocks, status_word=None, stream=None, check=True) -> int:
+    """Diagnostic: gather rows through a shared-memory ring as the tensor-core kernels do; time it with events."""
+    s = load_library().sbp_probe_gather_ring(_ptr(src), row_bytes, _ptr(rows), n_rows, threads, stages, blocks, _ptr(status_word),
+                                             _stream(stream))
+    if check:
+        _check(s, "sbp_probe_gather_ring")
+    return s
+
+
+def sbp_probe_mma_rate(N, mn_major, accumulators, iters, blocks, cycles_out, status_word=None, stream=None, check=True) -> int:
+    """Diagnostic: clocks of a stream of tcgen05.mma instructions of width N (int64 CUDA tensor receives the count)."""
+    s = load_library().sbp_probe_mma_rate(N, int(mn_major), accumulators, iters, blocks, _ptr(cycles_out), _ptr(status_word),
+                                          _stream(stream))
+    if check:
+        _check(s, "sbp_probe_mma_rate")
     return s
 
 

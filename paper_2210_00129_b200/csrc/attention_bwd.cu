@@ -46,7 +46,8 @@ struct AttnShared {
     uint32_t tmem_slot;
     int abort_flag;
     float part[2][128][3];        // per column half: running maximum, sum, sum of e^(s-m) * dS
-    float stat[kMaxTok][3];       // per query row: maximum (scaled, base 2), 1 / sum, rowsum(S * dS)
+    float stat[kMaxTok][3];       // per query row: -maximum (base 2, scaled), 1 / sum, -rowsum(S * dS) / sqrt(d)
+    int32_t q_glob[kMaxTok], k_glob[kMaxTok];   // global row of every query / key of the problem (-1: none)
 };
 
 __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk) { return row * kRowB + ((chunk ^ (row & 7u)) << 4); }
@@ -56,14 +57,50 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// gather `tiles * 128` rows of 64 bf16 (head slice) into a swizzled operand; rows past `count` become zeros
-__device__ __forceinline__ void load_rows(uint32_t dst, const __nv_bfloat16* src, int64_t ld, const int32_t* rows, int64_t first,
-                                          int64_t base_row, int count, int tiles, int col0) {
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// What a thread needs to know about a problem before it can start its copies: the token counts, the global rows
+// (t / 8 + 32 i) whose 16-byte chunk t % 8 it copies on the query and on the key side, and the global rows of query
+// and key number t (for the read-out).  Fetched one problem ahead, so that these dependent index loads never sit in
+// front of the copies.
+struct BigMeta {
+    int nq, nk;
+    int32_t qid[8], kid[8];       // -1: no such token (the row is zero-filled)
+    int32_t q_glob, k_glob;
+};
+__device__ __forceinline__ BigMeta fetch_big_meta(const AttnParams& p, int prob) {
+    BigMeta mt;
+    mt.nq = mt.nk = 0;
+    if (prob >= p.B * p.heads) return mt;
+    const int b = prob / p.heads;
+    const int base_row = b * p.N;
+    const int q0 = p.q_rows ? __ldg(p.q_offs + b) : 0, k0 = p.k_rows ? __ldg(p.k_offs + b) : 0;
+    mt.nq = p.q_rows ? __ldg(p.q_offs + b + 1) - q0 : p.N;
+    mt.nk = p.k_rows ? __ldg(p.k_offs + b + 1) - k0 : p.N;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = (threadIdx.x >> 3) + 32 * i;
+        mt.qid[i] = r < mt.nq ? (p.q_rows ? __ldg(p.q_rows + q0 + r) : base_row + r) : -1;
+        mt.kid[i] = r < mt.nk ? (p.k_rows ? __ldg(p.k_rows + k0 + r) : base_row + r) : -1;
+    }
+    const int r = threadIdx.x;
+    mt.q_glob = r < mt.nq ? (p.q_rows ? __ldg(p.q_rows + q0 + r) : base_row + r) : -1;
+    mt.k_glob = r < mt.nk ? (p.k_rows ? __ldg(p.k_rows + k0 + r) : base_row + r) : -1;
+    return mt;
+}
+// rows past `count` (up to the next multiple of 16, which is as far as the products step) become zeros
+__device__ __forceinline__ void load_rows_big(uint32_t dst, const __nv_bfloat16* src, int64_t ld, const int32_t (&id)[8], int count, int col0) {
     const uint32_t chunk = threadIdx.x & 7u;
-    for (int r = threadIdx.x >> 3; r < tiles * 128; r += kAttnThreads / 8) {
-        const bool live = r < count;
-        const int64_t g = live ? (rows != nullptr ? (int64_t)__ldg(rows + first + r) : base_row + r) : 0;
-        ptx::cp_async_16(dst + swz((uint32_t)r, chunk), src + (live ? g * ld + col0 + chunk * 8 : 0), live ? 16u : 0u);
+    const int padded = (count + 15) & ~15;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = (threadIdx.x >> 3) + 32 * i;
+        if (r < padded)
+            ptx::cp_async_16(dst + swz((uint32_t)r, chunk), src + (id[i] >= 0 ? (int64_t)id[i] * ld + col0 + chunk * 8 : 0), id[i] >= 0 ? 16u : 0u);
     }
 }
 
@@ -87,6 +124,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
         ptx::fence_mbar_init();
     }
     if (warp == 0) ptx::tmem_alloc(ptx::smem_addr(&sh.tmem_slot), 512);
+    // operand rows a problem does not fill are still read by the products (they only reach accumulator rows nobody
+    // stores), so they must hold finite numbers: clear everything once
+    for (uint32_t w = threadIdx.x; w < (4 * kTokBytes + 4 * kBlkBytes) / 16; w += kAttnThreads) reinterpret_cast<uint4*>(gen)[w] = make_uint4(0u, 0u, 0u, 0u);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
@@ -96,46 +136,43 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
     const bool skip_all = p.status_word != nullptr && *reinterpret_cast<volatile int32_t*>(p.status_word) != 0;
 
     const int q4 = warp & 3, half = warp >> 2;              // TMEM lane quadrant of this warp; which half of the columns it takes
-    const int row = q4 * 32 + lane;                         // accumulator row (query row, or key row in the dV / dK epilogue)
+    const int row = q4 * 32 + lane;                         // accumulator row (query row, or key row in the dV / dK read-out)
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const float sl2 = p.scale * 1.4426950408889634f;        // scores are kept in base 2: e^(x) = 2^(x log2 e)
     uint32_t n_s = 0, n_o = 0;                              // completed uses of the two barriers
     bool ok = !skip_all;
+    BigMeta cur = fetch_big_meta(p, ok ? (int)blockIdx.x : p.B * p.heads);
 
     for (int prob = blockIdx.x; ok && prob < p.B * p.heads; prob += gridDim.x) {
-        const int b = prob / p.heads, hh = prob % p.heads;
-        const int64_t q0 = p.q_rows ? __ldg(p.q_offs + b) : 0, k0 = p.k_rows ? __ldg(p.k_offs + b) : 0;
-        const int nq = p.q_rows ? (int)(__ldg(p.q_offs + b + 1) - q0) : p.N;
-        const int nk = p.k_rows ? (int)(__ldg(p.k_offs + b + 1) - k0) : p.N;
+        const int nq = cur.nq, nk = cur.nk;
+        const int col0 = (prob % p.heads) * kD;
+        if (nq > 0 && nk > 0) {
+            load_rows_big(sQ, p.Q, p.ld_qkv, cur.qid, nq, col0);
+            load_rows_big(sK, p.K, p.ld_qkv, cur.kid, nk, col0);
+            load_rows_big(sDA, p.dA, p.ld_da, cur.qid, nq, col0);
+            load_rows_big(sV, p.V, p.ld_qkv, cur.kid, nk, col0);
+            sh.q_glob[threadIdx.x] = cur.q_glob;
+            sh.k_glob[threadIdx.x] = cur.k_glob;
+        }
+        cur = fetch_big_meta(p, prob + (int)gridDim.x);      // the next problem's indices travel while this one computes
         if (nq <= 0 || nk <= 0) continue;
         const int QT = (nq + 127) >> 7, KT = (nk + 127) >> 7;
-        const int col0 = hh * kD;
-        const int64_t base_row = (int64_t)b * p.N;
-        // ---- stage the four operands ----
-        load_rows(sQ, p.Q, p.ld_qkv, p.q_rows, q0, base_row, nq, QT, col0);
-        load_rows(sDA, p.dA, p.ld_da, p.q_rows, q0, base_row, nq, QT, col0);
-        load_rows(sK, p.K, p.ld_qkv, p.k_rows, k0, base_row, nk, KT, col0);
-        load_rows(sV, p.V, p.ld_qkv, p.k_rows, k0, base_row, nk, KT, col0);
+        const int keys_pad = (nk + 15) & ~15;               // accumulator columns of the first pass (a multiple of 16)
         ptx::cp_async_wait_all();
         ptx::fence_async_proxy();
         __syncthreads();
 
-        // ---- first pass: softmax statistics of every query row ----
+        // ---- first pass: softmax statistics of every query row (S and dS over all keys: up to 256 columns each) ----
         for (int qt = 0; qt < QT && ok; ++qt) {
             if (threadIdx.x == 0) {
                 ptx::tc_fence_after_sync();
-                const uint32_t idesc = ptx::umma_idesc_bf16(128, KT * 128, false, false);
+                const uint32_t idesc = ptx::umma_idesc_bf16(128, keys_pad, false, false);
 #pragma unroll
-                for (uint32_t u = 0; u < 4; ++u) {
-                    const uint64_t dq = ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 32, 16, 1024);
-                    const uint64_t dk = ptx::umma_desc_sw128(sK + u * 32, 16, 1024);
-                    ptx::umma_bf16(tmem + kColS1, dq, dk, idesc, u != 0);
-                }
-#pragma unroll
-                for (uint32_t u = 0; u < 4; ++u) {
-                    const uint64_t da = ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 32, 16, 1024);
-                    const uint64_t dv = ptx::umma_desc_sw128(sV + u * 32, 16, 1024);
-                    ptx::umma_bf16(tmem + kColDS1, da, dv, idesc, u != 0);
+                for (uint32_t u = 0; u < 4; ++u) {          // the two products alternate: they fill different accumulators
+                    ptx::umma_bf16(tmem + kColS1, ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 32, 16, 1024),
+                                   ptx::umma_desc_sw128(sK + u * 32, 16, 1024), idesc, u != 0);
+                    ptx::umma_bf16(tmem + kColDS1, ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 32, 16, 1024),
+                                   ptx::umma_desc_sw128(sV + u * 32, 16, 1024), idesc, u != 0);
                 }
                 ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
             }
@@ -144,98 +181,113 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
             ok = !__syncthreads_or(!ok);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            // this thread: row `row`, columns [half * KT * 64, (half + 1) * KT * 64)
-            float m = -INFINITY, l = 0.f, u_acc = 0.f;
-            const int cbeg = half * KT * 64, cend = cbeg + KT * 64;
+            // this thread: row `row`, columns [128 half, 128 half + 128) below keys_pad; two sweeps (maximum; sums)
+            const int cbeg = half * 128, cend = keys_pad < cbeg + 128 ? keys_pad : cbeg + 128;
+            float mx = -INFINITY;
             for (int c = cbeg; c < cend; c += 32) {
-                float s[32], ds[32];
+                float s[32];
                 ptx::tmem_ld_32x32(tmem + kColS1 + (uint32_t)c + lane_off, s);
-                ptx::tmem_ld_32x32(tmem + kColDS1 + (uint32_t)c + lane_off, ds);
                 ptx::tmem_ld_wait();
-                float cm = -INFINITY;
+                if (c + 32 <= nk) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    s[j] = (c + j < nk) ? s[j] * sl2 : -INFINITY;
-                    cm = fmaxf(cm, s[j]);
+                    for (int j = 0; j < 32; ++j) mx = fmaxf(mx, s[j]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) mx = fmaxf(mx, (c + j < nk) ? s[j] : -INFINITY);
                 }
-                if (cm > m) {                                // rescale what has been summed so far
-                    const float f = exp2f(m - cm);           // 0 on the first chunk (m = -inf)
-                    l *= f; u_acc *= f; m = cm;
-                }
-                if (m > -INFINITY) {
+            }
+            float l = 0.f, u_acc = 0.f;
+            if (mx > -INFINITY) {
+                const float nm = -mx * sl2;
+                for (int c = cbeg; c < cend; c += 32) {
+                    float s[32], ds[32];
+                    ptx::tmem_ld_32x32(tmem + kColS1 + (uint32_t)c + lane_off, s);
+                    ptx::tmem_ld_32x32(tmem + kColDS1 + (uint32_t)c + lane_off, ds);
+                    ptx::tmem_ld_wait();
+                    const bool whole = c + 32 <= nk;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const float e = exp2f(s[j] - m);     // 0 for masked columns
+                        float e = ex2(fmaf(s[j], sl2, nm)), g = ds[j];
+                        if (!whole) {                        // a stale column may hold anything, NaN included
+                            e = (c + j < nk) ? e : 0.f;
+                            g = (c + j < nk) ? g : 0.f;
+                        }
                         l += e;
-                        u_acc += e * ds[j];
+                        u_acc = fmaf(e, g, u_acc);
                     }
                 }
             }
-            sh.part[half][row][0] = m; sh.part[half][row][1] = l; sh.part[half][row][2] = u_acc;
+            sh.part[half][row][0] = mx; sh.part[half][row][1] = l; sh.part[half][row][2] = u_acc;
             ptx::tc_fence_before_sync();
             __syncthreads();
-            if (half == 0) {
+            if (half == 0) {                                 // the two halves of a row, rescaled to their common maximum
                 const float m0 = sh.part[0][row][0], m1 = sh.part[1][row][0];
                 const float mm = fmaxf(m0, m1);
-                const float f0 = (m0 > -INFINITY) ? exp2f(m0 - mm) : 0.f, f1 = (m1 > -INFINITY) ? exp2f(m1 - mm) : 0.f;
+                const float f0 = (m0 > -INFINITY) ? ex2((m0 - mm) * sl2) : 0.f, f1 = (m1 > -INFINITY) ? ex2((m1 - mm) * sl2) : 0.f;
                 const float ll = sh.part[0][row][1] * f0 + sh.part[1][row][1] * f1;
                 const float uu = sh.part[0][row][2] * f0 + sh.part[1][row][2] * f1;
-                sh.stat[qt * 128 + row][0] = mm;
-                sh.stat[qt * 128 + row][1] = 1.f / ll;
-                sh.stat[qt * 128 + row][2] = uu / ll;
+                const float inv_l = 1.f / ll;
+                sh.stat[qt * 128 + row][0] = -mm * sl2;
+                sh.stat[qt * 128 + row][1] = inv_l;
+                sh.stat[qt * 128 + row][2] = -uu * inv_l * p.scale;      // -rowsum(S dS) / sqrt(d)
             }
             __syncthreads();
         }
         if (!ok) break;
 
-        // ---- second pass: blocks of S and dM, and the three gradient products ----
+        // ---- second pass: 128 x 128 blocks of S and dM, and the three gradient products ----
         for (int kt = 0; kt < KT && ok; ++kt) {
+            const int kb = keys_pad - kt * 128 < 128 ? keys_pad - kt * 128 : 128;      // key columns of this tile (a multiple of 16)
+            const uint32_t k_steps = (uint32_t)kb >> 4;
             for (int qt = 0; qt < QT && ok; ++qt) {
+                const int q_rows_here = nq - qt * 128 < 128 ? nq - qt * 128 : 128;
+                const uint32_t q_steps = (uint32_t)(q_rows_here + 15) >> 4;
                 if (threadIdx.x == 0) {
                     ptx::tc_fence_after_sync();
-                    const uint32_t idesc = ptx::umma_idesc_bf16(128, 128, false, false);
+                    const uint32_t idesc = ptx::umma_idesc_bf16(128, kb, false, false);
 #pragma unroll
                     for (uint32_t u = 0; u < 4; ++u) {
-                        const uint64_t dq = ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 32, 16, 1024);
-                        const uint64_t dk = ptx::umma_desc_sw128(sK + kt * kBlkBytes + u * 32, 16, 1024);
-                        ptx::umma_bf16(tmem + kColS, dq, dk, idesc, u != 0);
-                    }
-#pragma unroll
-                    for (uint32_t u = 0; u < 4; ++u) {
-                        const uint64_t da = ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 32, 16, 1024);
-                        const uint64_t dv = ptx::umma_desc_sw128(sV + kt * kBlkBytes + u * 32, 16, 1024);
-                        ptx::umma_bf16(tmem + kColDS, da, dv, idesc, u != 0);
+                        ptx::umma_bf16(tmem + kColS, ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 32, 16, 1024),
+                                       ptx::umma_desc_sw128(sK + kt * kBlkBytes + u * 32, 16, 1024), idesc, u != 0);
+                        ptx::umma_bf16(tmem + kColDS, ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 32, 16, 1024),
+                                       ptx::umma_desc_sw128(sV + kt * kBlkBytes + u * 32, 16, 1024), idesc, u != 0);
                     }
                     ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
                 }
                 ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_s), n_s & 1u, abort_flag, p.status_word);
                 ++n_s;
-                // the products of the previous block have read the S / dM blocks in shared memory by now (they were
-                // issued before the MMAs just waited for, and the tensor pipe runs in order)
                 ok = !__syncthreads_or(!ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const float mx = sh.stat[qt * 128 + row][0], inv_l = sh.stat[qt * 128 + row][1], delta = sh.stat[qt * 128 + row][2];
+                const float nm = sh.stat[qt * 128 + row][0], inv_l = sh.stat[qt * 128 + row][1], nds = sh.stat[qt * 128 + row][2];
 #pragma unroll
                 for (int c = 0; c < 64; c += 32) {
-                    float s[32], ds[32];
-                    ptx::tmem_ld_32x32(tmem + kColS + (uint32_t)(half * 64 + c) + lane_off, s);
-                    ptx::tmem_ld_32x32(tmem + kColDS + (uint32_t)(half * 64 + c) + lane_off, ds);
-                    ptx::tmem_ld_wait();
+                    const int cc = half * 64 + c;           // column within the tile
+                    if (cc < kb) {
+                        float s[32], ds[32];
+                        ptx::tmem_ld_32x32(tmem + kColS + (uint32_t)cc + lane_off, s);
+                        ptx::tmem_ld_32x32(tmem + kColDS + (uint32_t)cc + lane_off, ds);
+                        ptx::tmem_ld_wait();
+                        const bool whole = kt * 128 + cc + 32 <= nk;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const bool live = kt * 128 + half * 64 + c + j < nk;
-                        const float pj = live ? exp2f(s[j] * sl2 - mx) * inv_l : 0.f;
-                        s[j] = pj;
-                        ds[j] = pj * (ds[j] - delta) * p.scale;
-                    }
+                        for (int j = 0; j < 32; ++j) {
+                            float e = ex2(fmaf(s[j], sl2, nm)), g = ds[j];
+                            if (!whole) {
+                                e = (kt * 128 + cc + j < nk) ? e : 0.f;
+                                g = (kt * 128 + cc + j < nk) ? g : 0.f;
+                            }
+                            const float pj = e * inv_l;
+                            s[j] = pj;
+                            ds[j] = pj * fmaf(g, p.scale, nds);      // dM / sqrt(d)
+                        }
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t off = swz((uint32_t)row, (uint32_t)(c / 8 + q));
-                        *reinterpret_cast<uint4*>(gP + half * kBlkBytes + off) =
-                            make_uint4(pack2(s[q * 8], s[q * 8 + 1]), pack2(s[q * 8 + 2], s[q * 8 + 3]), pack2(s[q * 8 + 4], s[q * 8 + 5]), pack2(s[q * 8 + 6], s[q * 8 + 7]));
-                        *reinterpret_cast<uint4*>(gDM + half * kBlkBytes + off) =
-                            make_uint4(pack2(ds[q * 8], ds[q * 8 + 1]), pack2(ds[q * 8 + 2], ds[q * 8 + 3]), pack2(ds[q * 8 + 4], ds[q * 8 + 5]), pack2(ds[q * 8 + 6], ds[q * 8 + 7]));
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t off = (uint32_t)half * kBlkBytes + swz((uint32_t)row, (uint32_t)(c / 8 + q));
+                            *reinterpret_cast<uint4*>(gP + off) =
+                                make_uint4(pack2(s[q * 8], s[q * 8 + 1]), pack2(s[q * 8 + 2], s[q * 8 + 3]), pack2(s[q * 8 + 4], s[q * 8 + 5]), pack2(s[q * 8 + 6], s[q * 8 + 7]));
+                            *reinterpret_cast<uint4*>(gDM + off) =
+                                make_uint4(pack2(ds[q * 8], ds[q * 8 + 1]), pack2(ds[q * 8 + 2], ds[q * 8 + 3]), pack2(ds[q * 8 + 4], ds[q * 8 + 5]), pack2(ds[q * 8 + 6], ds[q * 8 + 7]));
+                        }
                     }
                 }
                 ptx::fence_async_proxy();                    // the blocks are read by the tensor core
@@ -245,20 +297,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
                     ptx::tc_fence_after_sync();
                     const uint32_t id_t = ptx::umma_idesc_bf16(128, 64, true, true);     // dV, dK: both operands MN-major
                     const uint32_t id_q = ptx::umma_idesc_bf16(128, 64, false, true);    // dQ: dM K-major, K MN-major
-#pragma unroll
-                    for (uint32_t u = 0; u < 8; ++u) {           // reduction over the 128 query rows of the tile, 16 at a time
-                        const uint64_t dp = ptx::umma_desc_sw128(sP + u * 2048, kBlkBytes, 1024);
-                        const uint64_t dda = ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 2048, kBlkBytes, 1024);
-                        ptx::umma_bf16(tmem + kColDV, dp, dda, id_t, (qt | (int)u) != 0);
-                        const uint64_t ddm = ptx::umma_desc_sw128(sDM + u * 2048, kBlkBytes, 1024);
-                        const uint64_t dq = ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 2048, kBlkBytes, 1024);
-                        ptx::umma_bf16(tmem + kColDK, ddm, dq, id_t, (qt | (int)u) != 0);
-                    }
-#pragma unroll
-                    for (uint32_t u = 0; u < 8; ++u) {           // reduction over the 128 keys of the tile: two 64-key blocks x four steps
-                        const uint64_t ddm = ptx::umma_desc_sw128(sDM + (u >> 2) * kBlkBytes + (u & 3u) * 32, 16, 1024);
-                        const uint64_t dk = ptx::umma_desc_sw128(sK + kt * kBlkBytes + u * 2048, kBlkBytes, 1024);
-                        ptx::umma_bf16(tmem + kColDQ + (uint32_t)qt * 64u, ddm, dk, id_q, (kt | (int)u) != 0);
+                    const uint32_t steps = q_steps > k_steps ? q_steps : k_steps;
+                    for (uint32_t u = 0; u < steps; ++u) {   // three accumulators take turns; only the 16-row steps that hold tokens run
+                        if (u < q_steps) {                   // reductions over the query rows of the tile
+                            ptx::umma_bf16(tmem + kColDV, ptx::umma_desc_sw128(sP + u * 2048, kBlkBytes, 1024),
+                                           ptx::umma_desc_sw128(sDA + qt * kBlkBytes + u * 2048, kBlkBytes, 1024), id_t, (qt | (int)u) != 0);
+                            ptx::umma_bf16(tmem + kColDK, ptx::umma_desc_sw128(sDM + u * 2048, kBlkBytes, 1024),
+                                           ptx::umma_desc_sw128(sQ + qt * kBlkBytes + u * 2048, kBlkBytes, 1024), id_t, (qt | (int)u) != 0);
+                        }
+                        if (u < k_steps)                     // reduction over the keys of the tile: two 64-key blocks x four steps
+                            ptx::umma_bf16(tmem + kColDQ + (uint32_t)qt * 64u, ptx::umma_desc_sw128(sDM + (u >> 2) * kBlkBytes + (u & 3u) * 32, 16, 1024),
+                                           ptx::umma_desc_sw128(sK + kt * kBlkBytes + u * 2048, kBlkBytes, 1024), id_q, (kt | (int)u) != 0);
                     }
                     ptx::umma_commit(ptx::smem_addr(&sh.bar_o));
                 }
@@ -267,25 +316,33 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
                 ok = !__syncthreads_or(!ok);
             }
             if (!ok) break;
-            // ---- dV and dK of this key tile: accumulator row = key, 64 columns; this thread takes 32 of them ----
+            // ---- dV and dK of this key tile: accumulator row = key; through shared memory (the S and dM blocks are free)
+            //      so that every store instruction writes whole 128-byte rows ----
             ptx::tc_fence_after_sync();
-            const int key = kt * 128 + row;
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 float v[32];
                 ptx::tmem_ld_32x32(tmem + (which ? kColDK : kColDV) + (uint32_t)(half * 32) + lane_off, v);
                 ptx::tmem_ld_wait();
-                if (key < nk) {
-                    const int64_t g = p.k_rows ? (int64_t)__ldg(p.k_rows + k0 + key) : base_row + key;
-                    __nv_bfloat16* out = (which ? p.dK : p.dV) + g * p.ld_out + col0 + half * 32;
+                uint8_t* stage = which ? gDM : gP;
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        ptx::st_global_v4(out + q * 8, pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]),
-                                          pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
-                }
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4*>(stage + swz((uint32_t)row, (uint32_t)(half * 4 + q))) =
+                        make_uint4(pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]), pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
             }
             ptx::tc_fence_before_sync();
             __syncthreads();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int idx = threadIdx.x + kAttnThreads * i;          // 2 outputs x 128 rows x 8 chunks
+                const int which = idx >> 10, r = (idx >> 3) & 127, ch = idx & 7;
+                const int32_t g = sh.k_glob[kt * 128 + r];
+                if (kt * 128 + r < nk && g >= 0) {
+                    const uint4 pk = *reinterpret_cast<const uint4*>((which ? gDM : gP) + swz((uint32_t)r, (uint32_t)ch));
+                    ptx::st_global_v4((which ? p.dK : p.dV) + (int64_t)g * p.ld_out + col0 + ch * 8, pk.x, pk.y, pk.z, pk.w);
+                }
+            }
+            __syncthreads();                                 // the stages become S / dM blocks again
         }
         if (!ok) break;
         // ---- dQ of every query tile ----
@@ -294,18 +351,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
             float v[32];
             ptx::tmem_ld_32x32(tmem + kColDQ + (uint32_t)(qt * 64 + half * 32) + lane_off, v);
             ptx::tmem_ld_wait();
-            const int qi = qt * 128 + row;
-            if (qi < nq) {
-                const int64_t g = p.q_rows ? (int64_t)__ldg(p.q_rows + q0 + qi) : base_row + qi;
-                __nv_bfloat16* out = p.dQ + g * p.ld_out + col0 + half * 32;
+            uint8_t* stage = qt ? gDM : gP;
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    ptx::st_global_v4(out + q * 8, pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]),
-                                      pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
+            for (int q = 0; q < 4; ++q)
+                *reinterpret_cast<uint4*>(stage + swz((uint32_t)row, (uint32_t)(half * 4 + q))) =
+                    make_uint4(pack2(v[q * 8], v[q * 8 + 1]), pack2(v[q * 8 + 2], v[q * 8 + 3]), pack2(v[q * 8 + 4], v[q * 8 + 5]), pack2(v[q * 8 + 6], v[q * 8 + 7]));
+        }
+        ptx::tc_fence_before_sync();
+        __syncthreads();
+        for (int i = 0; i < 4 * QT; ++i) {
+            const int idx = threadIdx.x + kAttnThreads * i;              // QT tiles x 128 rows x 8 chunks
+            const int qt = idx >> 10, r = (idx >> 3) & 127, ch = idx & 7;
+            const int32_t g = sh.q_glob[qt * 128 + r];
+            if (qt * 128 + r < nq && g >= 0) {
+                const uint4 pk = *reinterpret_cast<const uint4*>((qt ? gDM : gP) + swz((uint32_t)r, (uint32_t)ch));
+                ptx::st_global_v4(p.dQ + (int64_t)g * p.ld_out + col0 + ch * 8, pk.x, pk.y, pk.z, pk.w);
             }
         }
         ptx::tc_fence_before_sync();
-        __syncthreads();                                     // operands and accumulators are free for the next problem
+        __syncthreads();                                     // operands, stages and accumulators are free for the next problem
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -314,7 +378,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
         ptx::tmem_dealloc(tmem, 512);
     }
 }
-
 
 // ---------------------------------------------------------------------------------------------
 // At most 128 kept tokens on both sides (keep ratios up to 0.5 on 14 x 14 maps, the paper's setting): one 128 x 128
@@ -371,12 +434,6 @@ __device__ __forceinline__ void load_rows_small(uint32_t dst, const __nv_bfloat1
             ptx::cp_async_16(dst + swz((uint32_t)r, chunk), src + (id[i] >= 0 ? (int64_t)id[i] * ld + col0 + chunk * 8 : 0), id[i] >= 0 ? 16u : 0u);
     }
 }
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 __global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(const AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ SmallShared sh;

@@ -1,0 +1,175 @@
+// Diagnostic probes (no counterpart in the paper): two micro-measurements of the machinery the tensor-core kernels are
+// built from, kept in the library so that the figures the design quotes can be re-taken with one command
+// (`python bench.py --probe`).
+//   gather ring: rows picked by an index list are copied with 16-byte cp.async into a ring of 16 KB shared-memory
+//                stages (128 rows x 128 bytes, 128-byte swizzle) behind full / empty mbarriers, exactly as the backward
+//                kernel gathers the kept rows of dY; a consumer thread frees each stage as soon as it has landed.
+//                Nothing is computed: the time is what the gather path alone can sustain.
+//   mma rate:    one thread per block issues a stream of tcgen05.mma (M = 128, K = 16, bf16) of a given width on
+//                constant operands and reports the clocks from the first issue to the completion of the last.
+#include "tc_ptx.cuh"
+
+namespace sbp {
+namespace {
+
+struct ProbeShared {
+    uint64_t full[12], empty[12], done;
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS + 32, 1)
+probe_gather_kernel(const uint8_t* __restrict__ src, const int32_t* __restrict__ rows, int n_rows, int row_bytes, int stages,
+                    int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ ProbeShared sh;
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;
+    constexpr uint32_t kStage = 128 * 128;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&sh.full[s]), THREADS);
+            ptx::mbar_init(ptx::smem_addr(&sh.empty[s]), 1);
+        }
+        sh.abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    volatile int* abort_flag = &sh.abort_flag;
+    const int ntiles = (n_rows + 127) / 128;
+    const int kb_per_tile = row_bytes / 128;
+    if (threadIdx.x >= THREADS) {                           // consumer warp: one lane frees the stages as they fill
+        if (threadIdx.x == THREADS) {
+            uint32_t it = 0;
+            for (int t = blockIdx.x; t < ntiles; t += gridDim.x)
+                for (int k = 0; k < kb_per_tile; ++k, ++it) {
+                    const int s = it % stages;
+                    if (!ptx::mbar_wait(ptx::smem_addr(&sh.full[s]), (it / stages) & 1u, abort_flag, status_word)) return;
+                    ptx::mbar_arrive(ptx::smem_addr(&sh.empty[s]));
+                }
+        }
+        return;
+    }
+    constexpr int RPI = THREADS / 8;                        // rows one wave of all copying threads covers
+    constexpr int NI = 128 / RPI;
+    const uint32_t chunk = threadIdx.x & 7u, sub = threadIdx.x >> 3;
+    uint32_t it = 0;
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        const uint8_t* p[NI];
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+            int m = t * 128 + i * RPI + (int)sub;
+            if (m >= n_rows) m = n_rows - 1;
+            p[i] = src + (size_t)__ldg(rows + m) * row_bytes + chunk * 16;
+        }
+        for (int k = 0; k < kb_per_tile; ++k, ++it) {
+            const int s = it % stages;
+            bool ok = ptx::mbar_wait(ptx::smem_addr(&sh.empty[s]), ((it / stages) & 1u) ^ 1u, abort_flag, status_word);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { ptx::cp_async_wait_all(); return; }
+            const uint32_t dst = ring + s * kStage;
+#pragma unroll
+            for (int i = 0; i < NI; ++i) {
+                const uint32_t r = i * RPI + sub;
+                ptx::cp_async_16(dst + r * 128 + ((chunk ^ (r & 7u)) << 4), p[i] + k * 128, 16u);
+            }
+            ptx::cp_async_arrive_noinc(ptx::smem_addr(&sh.full[s]));
+        }
+    }
+    ptx::cp_async_wait_all();
+}
+
+__global__ void __launch_bounds__(128, 1)
+probe_mma_kernel(int N, int mn_major, int accumulators, int iters, long long* cycles_out, int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ ProbeShared sh;
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    // operands: A = 128 x 64 (16 KB) at base, B = up to 256 x 64 (32 KB) behind it; all ones (bf16 1.0)
+    for (uint32_t i = threadIdx.x; i < 48 * 1024 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3F803F80u;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&sh.done), 1);
+        sh.abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    ptx::fence_async_proxy();
+    if (threadIdx.x < 32) ptx::tmem_alloc(ptx::smem_addr(&sh.tmem_slot), 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_slot);
+    if (threadIdx.x == 0) {
+        const uint32_t a_addr = base, b_addr = base + 16 * 1024;
+        const uint32_t idesc = ptx::umma_idesc_bf16(128, N, mn_major != 0, mn_major != 0);
+        const uint32_t k_step = mn_major ? 16u * 128u : 32u;          // as in the backward kernel's two operand layouts
+        const uint32_t lbo = mn_major ? 64u * 128u : 16u;
+        const long long c0 = clock64();
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (uint32_t u = 0; u < 4; ++u) {
+                const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, 1024);
+                const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, 1024);
+                ptx::umma_bf16(tmem, da, db, idesc, (it | (int)u) != 0);
+                if (accumulators == 2) ptx::umma_bf16(tmem + 256u, da, db, idesc, (it | (int)u) != 0);
+            }
+        }
+        ptx::umma_commit(ptx::smem_addr(&sh.done));
+        const bool ok = ptx::mbar_wait(ptx::smem_addr(&sh.done), 0, &sh.abort_flag, status_word);
+        const long long c1 = clock64();
+        if (blockIdx.x == 0) cycles_out[0] = ok ? c1 - c0 : -1;
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, 512);
+    }
+}
+
+}  // namespace
+}  // namespace sbp
+
+extern "C" {
+
+sbp_status sbp_probe_gather_ring(const void* src, int64_t row_bytes, const int32_t* rows, int64_t n_rows, int threads, int stages,
+                                 int blocks, int32_t* status_word, void* stream) {
+    using namespace sbp;
+    if (src == nullptr || rows == nullptr || (reinterpret_cast<uintptr_t>(src) & 15u) || (reinterpret_cast<uintptr_t>(rows) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    if (row_bytes < 128 || row_bytes % 128 != 0 || row_bytes > (1 << 20) || n_rows <= 0 || n_rows >= (1ll << 31)) return SBP_ERR_INVALID_ARG;
+    if (stages < 2 || stages > 12 || blocks < 1 || blocks > 4 * kNumSMs) return SBP_ERR_INVALID_ARG;
+    const size_t smem = (size_t)stages * 16384 + 1024;
+    cudaError_t e;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (threads == 64) {
+        e = opt_in_dynamic_smem<probe_gather_kernel<64>>(197 * 1024);
+        if (e == cudaSuccess) probe_gather_kernel<64><<<blocks, 96, smem, st>>>((const uint8_t*)src, rows, (int)n_rows, (int)row_bytes, stages, status_word);
+    } else if (threads == 128) {
+        e = opt_in_dynamic_smem<probe_gather_kernel<128>>(197 * 1024);
+        if (e == cudaSuccess) probe_gather_kernel<128><<<blocks, 160, smem, st>>>((const uint8_t*)src, rows, (int)n_rows, (int)row_bytes, stages, status_word);
+    } else if (threads == 256) {
+        e = opt_in_dynamic_smem<probe_gather_kernel<256>>(197 * 1024);
+        if (e == cudaSuccess) probe_gather_kernel<256><<<blocks, 288, smem, st>>>((const uint8_t*)src, rows, (int)n_rows, (int)row_bytes, stages, status_word);
+    } else {
+        return SBP_ERR_INVALID_ARG;
+    }
+    if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return SBP_ERR_CUDA;
+    return SBP_OK;
+}
+
+sbp_status sbp_probe_mma_rate(int N, int mn_major, int accumulators, int iters, int blocks, int64_t* cycles_out, int32_t* status_word,
+                              void* stream) {
+    using namespace sbp;
+    if (cycles_out == nullptr || (reinterpret_cast<uintptr_t>(cycles_out) & 7u)) return SBP_ERR_INVALID_ARG;
+    if (N < 16 || N > 256 || N % 16 != 0 || (accumulators != 1 && accumulators != 2) || iters < 1 || iters > 100000 || blocks < 1 ||
+        blocks > kNumSMs)
+        return SBP_ERR_INVALID_ARG;
+    const cudaError_t e = opt_in_dynamic_smem<probe_mma_kernel>(50 * 1024);
+    if (e != cudaSuccess) return SBP_ERR_CUDA;
+    probe_mma_kernel<<<blocks, 128, 50 * 1024, (cudaStream_t)stream>>>(N, mn_major, accumulators, iters, reinterpret_cast<long long*>(cycles_out),
+                                                                       status_word);
+    return cudaGetLastError() == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -323,7 +323,8 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
     if ((flags & SBP_FLAG_W_OUT_IN) && (want_dW || want_dX)) n += (want_dX ? 1 : 0) + (want_dW ? 1 : 0);   // transposes
     const bool db_rides = tc && want_db && (want_dW || want_dX);
     if (want_db && !db_rides) n += 2;                      // strip partials + fixed-order reduce
-    if (tc) return n + tc_backward_kernel_count(M_keep_cap, C_in, C_out, want_dW != 0, want_dX != 0, db_rides);
+    if (tc) return n + tc_backward_kernel_count(M_keep_cap, C_in, C_out, want_dW != 0, want_dX != 0, db_rides,
+                                                (flags & SBP_FLAG_DY_COMPACT) != 0);
     if (want_dW) n += simt_dw_kernel_count(M_keep_cap, C_in, C_out);
     if (want_dX) n += 1;
     return n;

@@ -209,7 +209,7 @@ bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t 
 size_t tc_dw_workspace_bytes(int64_t M_keep_cap, int64_t C_in, int64_t C_out);
 int64_t tc_plan_searches();              // split-plan searches run so far in this process
 int    tc_backward_kernel_count(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bool want_dx,
-                                bool want_db);
+                                bool want_db, bool dy_packed);
 // dW (nullable) and dX (nullable) of one layer in a single persistent kernel (+ the split reduce); when db is
 // given its column sums ride along in the same kernel (db_workspace: kNumSMs * C_out floats) + one reduce
 // (dy_rows / dx_rows as for launch_simt_dx)
