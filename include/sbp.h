@@ -13,6 +13,7 @@
  *   sbp_linear_backward  dW = X_keep^T dY_keep, db = sum dY_keep,
  *                        dX = scatter(dY_keep W^T), zeros elsewhere   (Eq. 5)
  *   sbp_attention_backward  dQ, dK, dV of attention on the kept tokens (Sec. 4, Drop QKV / Drop Query only)
+ *   sbp_act_backward     dZ = dH * gelu'(Z_keep) on packed rows between two layers of a block (Sec. 3.3.1)
  *   sbp_patch_cache / sbp_patch_scatter  stride >= kernel convolutions as linear layers on patch rows (Sec. 3.2.2)
  *
  * Nothing is rescaled by 1/r: Eq. 1 keeps the plain 1/B factor.
@@ -52,6 +53,9 @@ typedef enum {
 } sbp_status;
 
 typedef enum { SBP_F32 = 0, SBP_BF16 = 1 } sbp_dtype;
+
+/* position-wise activations sbp_act_backward knows */
+typedef enum { SBP_ACT_GELU = 0 /* exact form: z Phi(z) */ } sbp_activation;
 
 /* Sec. 4, "How to sample the gradient keep mask?": uniformly random positions,
  * or a structured periodic ("grid-wise") mask. */
@@ -232,6 +236,22 @@ sbp_status sbp_linear_backward(sbp_dtype dt,
 int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap, int64_t C_in,
                                      int64_t C_out, int want_dW, int want_db, int want_dX,
                                      uint32_t flags);
+
+/*
+ * Backward of a position-wise activation between two SBP layers that share a keep set (Sec. 3.3.1 and the
+ * supplementary's chain rule for transformer blocks: kept positions stay kept and dropped ones stay dropped through
+ * position-wise operations, so inside an MLP block - linear, GELU, linear - the gradient can stay packed):
+ *   dZ[m, c] = dH[m, c] * act'(Z_keep[m, c])   for m < M_keep;  rows [M_keep, M_keep_cap) of dZ = 0
+ * Z_keep [M_keep_cap, C]: the cached pre-activation rows of the kept positions (what sbp_forward_cache or
+ * sbp_linear_forward's cache holds for the layer behind the activation); dH [M_keep_cap, C]: the packed gradient of
+ * the activation's output (the SBP_FLAG_DX_COMPACT output of the layer above); dZ [M_keep_cap, C]: the packed gradient
+ * of its input (the SBP_FLAG_DY_COMPACT input of the layer below); dZ may alias dH.  SBP_ACT_GELU:
+ * gelu'(z) = (1 + erf(z / sqrt 2)) / 2 + z exp(-z^2 / 2) / sqrt(2 pi).  Arithmetic in fp32, one rounding to dt.
+ * C * sizeof(element) must be a multiple of 16 (else SBP_ERR_UNSUPPORTED); other activations SBP_ERR_UNSUPPORTED.
+ */
+sbp_status sbp_act_backward(sbp_dtype dt, sbp_activation act, const void* Z_keep /* dev */, const void* dH /* dev */,
+                            const int32_t* M_keep_dev /* dev, nullable */, int64_t M_keep_cap, int64_t C,
+                            void* dZ /* dev */, int32_t* status_word /* dev, nullable */, void* stream);
 
 /*
  * Convolutions with stride >= kernel size as SBP layers (Sec. 3.2.2, the text after Eq. 6: with s >= k the

@@ -71,6 +71,10 @@ def _load():
     lib.oracle_patch_conv_forward.restype = None
     lib.oracle_patch_conv_backward.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp, vp, vp]
     lib.oracle_patch_conv_backward.restype = None
+    lib.oracle_gelu.argtypes = [vp, i64, vp]
+    lib.oracle_gelu.restype = None
+    lib.oracle_act_backward_gelu.argtypes = [vp, vp, i64, vp]
+    lib.oracle_act_backward_gelu.restype = None
     lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
     lib.oracle_set_num_threads.restype = None
     lib.oracle_num_threads.argtypes = []
@@ -239,3 +243,20 @@ def patch_conv_backward(X, dY, Wt, keep_rows, k, stride, want=("dW", "db", "dX")
     _load().oracle_patch_conv_backward(_ptr(X), _ptr(dY), _ptr(Wt), _ptr(rows), rows.shape[0], B, H, W, C, Co, k, stride,
                                        _ptr(dW), _ptr(db), _ptr(dX))
     return {n: v for n, v in (("dW", dW), ("db", db), ("dX", dX)) if v is not None}
+
+
+def gelu(z):
+    """Exact GELU, z Phi(z), in fp64."""
+    z = _f64(z)
+    out = np.empty_like(z)
+    _load().oracle_gelu(_ptr(z), z.size, _ptr(out))
+    return out
+
+
+def act_backward_gelu(z, dh):
+    """dz = dh * gelu'(z) in fp64 (element-wise; the caller passes the kept rows)."""
+    z, dh = _f64(z), _f64(dh)
+    assert z.shape == dh.shape
+    out = np.empty_like(z)
+    _load().oracle_act_backward_gelu(_ptr(z), _ptr(dh), z.size, _ptr(out))
+    return out

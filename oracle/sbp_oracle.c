@@ -615,3 +615,24 @@ void oracle_patch_conv_backward(const double* X, const double* dY, const double*
             }
     }
 }
+
+/* ------------------------------------------------------------------ */
+/* Position-wise activation between two SBP layers of a block (Sec. 3.3.1; */
+/* the supplementary's chain rule for transformer blocks): element-wise,   */
+/* so it acts on the kept rows alone.  GELU in its exact form,             */
+/* gelu(z) = z Phi(z),  gelu'(z) = Phi(z) + z phi(z).                      */
+/* ------------------------------------------------------------------ */
+void oracle_gelu(const double* z, int64_t n, double* out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = 0.5 * z[i] * (1.0 + erf(z[i] / sqrt(2.0)));
+}
+
+void oracle_act_backward_gelu(const double* z, const double* dh, int64_t n, double* dz)
+{
+    const double inv_sqrt_2pi = 1.0 / sqrt(2.0 * acos(-1.0));
+    for (int64_t i = 0; i < n; ++i) {
+        const double Phi = 0.5 * (1.0 + erf(z[i] / sqrt(2.0)));
+        const double phi = inv_sqrt_2pi * exp(-0.5 * z[i] * z[i]);
+        dz[i] = dh[i] * (Phi + z[i] * phi);
+    }
+}

@@ -20,13 +20,14 @@ LIB_PATH = os.path.join(_HERE, "libsbp_b200.so")
 SBP_OK, SBP_ERR_INVALID_ARG, SBP_ERR_UNSUPPORTED, SBP_ERR_WORKSPACE = 0, 1, 2, 3
 SBP_ERR_CUDA, SBP_ERR_TIMEOUT, SBP_ERR_BAD_INDICES = 4, 5, 6
 SBP_F32, SBP_BF16 = 0, 1
+SBP_ACT_GELU = 0
 SBP_MASK_RANDOM, SBP_MASK_GRID, SBP_MASK_TEMPORAL, SBP_MASK_TEMPORAL_GRID = 0, 1, 2, 3
 SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
 SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT, SBP_FLAG_W_OUT_IN, SBP_FLAG_ATTN_ALL_KEYS = 16, 32, 64, 128
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
-           "sbp_plan_search_count", "sbp_attention_backward", "sbp_patch_cache", "sbp_patch_scatter_workspace_bytes",
+           "sbp_plan_search_count", "sbp_act_backward", "sbp_attention_backward", "sbp_patch_cache", "sbp_patch_scatter_workspace_bytes",
            "sbp_patch_scatter", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
            "sbp_selftest_bounded_wait", "sbp_probe_gather_ring", "sbp_probe_mma_rate")
 
@@ -81,6 +82,8 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_probe_gather_ring.restype = ci
     lib.sbp_probe_mma_rate.argtypes = [ci, ci, ci, ci, ci, vp, vp, vp]
     lib.sbp_probe_mma_rate.restype = ci
+    lib.sbp_act_backward.argtypes = [ci, ci, vp, vp, vp, i64, i64, vp, vp, vp]
+    lib.sbp_act_backward.restype = ci
     lib.sbp_plan_search_count.argtypes = []
     lib.sbp_plan_search_count.restype = i64
     lib.sbp_step_host_arena_bytes.argtypes = [ci, ci, i64, i64, i64, i64, i64, dbl]
@@ -207,6 +210,15 @@ def sbp_patch_scatter(dt, dX_patches, B, H, W, C, k, stride, keep_rows, M_keep_d
                                          _stream(stream))
     if check:
         _check(s, "sbp_patch_scatter")
+    return s
+
+
+def sbp_act_backward(dt, act, Z_keep, dH, M_keep_dev, M_keep_cap, C, dZ, status_word=None, stream=None, check=True) -> int:
+    """dZ = dH * act'(Z_keep) on packed kept rows (the activation between two layers of a packed block)."""
+    s = load_library().sbp_act_backward(dt, act, _ptr(Z_keep), _ptr(dH), _ptr(M_keep_dev), M_keep_cap, C, _ptr(dZ),
+                                        _ptr(status_word), _stream(stream))
+    if check:
+        _check(s, "sbp_act_backward")
     return s
 
 

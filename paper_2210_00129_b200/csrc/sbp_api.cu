@@ -332,6 +332,19 @@ int sbp_linear_backward_kernel_count(sbp_dtype dt, int64_t M, int64_t M_keep_cap
 
 int64_t sbp_plan_search_count(void) { return tc_plan_searches(); }
 
+sbp_status sbp_act_backward(sbp_dtype dt, sbp_activation act, const void* Z_keep, const void* dH, const int32_t* M_keep_dev,
+                            int64_t M_keep_cap, int64_t C, void* dZ, int32_t* status_word, void* stream) {
+    if (dt != SBP_F32 && dt != SBP_BF16) return SBP_ERR_INVALID_ARG;
+    if (act != SBP_ACT_GELU) return SBP_ERR_UNSUPPORTED;
+    if (Z_keep == nullptr || dH == nullptr || dZ == nullptr || !aligned16(Z_keep) || !aligned16(dH) || !aligned16(dZ))
+        return SBP_ERR_INVALID_ARG;
+    if (M_keep_cap < 0 || M_keep_cap >= (1ll << 31) || C <= 0 || C >= (1ll << 24)) return SBP_ERR_INVALID_ARG;
+    const int64_t row_bytes = C * (dt == SBP_BF16 ? 2 : 4);
+    if (row_bytes % 16 != 0) return SBP_ERR_UNSUPPORTED;
+    const cudaError_t e = launch_act_backward(dt, Z_keep, dH, dZ, row_bytes, M_keep_dev, M_keep_cap, status_word, (cudaStream_t)stream);
+    return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
 namespace {
 // shared argument checks of the two patch calls; returns SBP_OK and the output grid when the geometry is usable
 sbp_status patch_geometry(sbp_dtype dt, int64_t B, int64_t H, int64_t W, int64_t C, int64_t k, int64_t stride, int64_t M_keep_cap,

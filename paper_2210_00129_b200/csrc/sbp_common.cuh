@@ -187,6 +187,10 @@ sbp_status launch_tc_forward(const void* X, const void* W, bool w_out_in, const 
                              void* Y, const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap,
                              void* X_keep, int32_t* status_word, cudaStream_t stream);
 
+// dZ = dH * gelu'(Z_keep) on packed kept rows (element-wise)
+cudaError_t launch_act_backward(sbp_dtype dt, const void* Z, const void* dH, void* dZ, int64_t row_bytes, const int32_t* M_keep_dev,
+                                int64_t M_keep_cap, const int32_t* status_word, cudaStream_t stream);
+
 // stride >= kernel convolutions as linear layers on patch rows: gather of the kept patches, scatter of their gradients
 cudaError_t launch_patch_gather(const void* X, int64_t H, int64_t W, int64_t pos_bytes, int64_t k, int64_t s,
                                 const int32_t* keep_rows, const int32_t* M_keep_dev, int64_t M_keep_cap, void* X_keep,
