@@ -320,16 +320,51 @@ class Job:
         for (_, ci, co), L in zip(self.layers, s["layers"]):
             rc |= lib.sbp_forward_cache(code, L["p"]["X"], M, ci, a["rows"], a["cnt"], capk, L["p"]["Xk"], sid)
         for li in range(len(self.layers) - 1, -1, -1):
-            _, ci, co = self.layers[li]
-            q = s["layers"][li]["p"]
             if events is not None:
                 events[li][0].record(self.stream)
-            rc |= lib.sbp_linear_backward(code, q["Xk"], q["dY"], q["W"], a["rows"], a["cnt"], M, capk, ci, co, q["dW"], q["db"],
-                                          q["dX"], 0, self.ws.data_ptr(), self.ws_bytes, self.status.data_ptr(), sid)
+            rc |= self.backward_call(i, li, r, sid)
             if events is not None:
                 events[li][1].record(self.stream)
         if rc != 0:
             raise RuntimeError(f"sbp call failed with status {rc}")
+
+    def backward_call(self, i, li, r, sid):
+        """sbp_linear_backward of layer li on buffer set i (its keep set and cache must have been made at ratio r)."""
+        s = self.sets[i % self.n_sets]
+        _, ci, co = self.layers[li]
+        q, a = s["layers"][li]["p"], s["p"]
+        return self.lib.sbp_linear_backward(self.code, q["Xk"], q["dY"], q["W"], a["rows"], a["cnt"], self.M, self.cap[r], ci, co,
+                                            q["dW"], q["db"], q["dX"], 0, self.ws.data_ptr(), self.ws_bytes, self.status.data_ptr(), sid)
+
+    def timed_backward_graphs(self, r, reps):
+        """Device time of every layer's backward call at keep ratio r, without the host in the loop: per layer one CUDA
+        graph holding that call once per buffer set, replayed `reps` times between two events on the launch stream.
+        Returns (per-layer ms per call, seconds of the timed replays)."""
+        torch = self.torch
+        for k in range(self.n_sets):                       # keep sets and caches of every buffer set at this ratio
+            self.step(k, r)
+        self.barrier()
+        cap_stream = torch.cuda.Stream()
+        cap_stream.wait_stream(self.stream)
+        per_layer, total_s = [], 0.0
+        for li in range(len(self.layers)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap_stream):
+                for k in range(self.n_sets):
+                    if self.backward_call(k, li, r, cap_stream.cuda_stream) != 0:
+                        raise RuntimeError("sbp_linear_backward failed during capture")
+            g.replay()
+            self.barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(self.stream)
+            self.barrier()
+            ms = max_over_ranks(e0.elapsed_time(e1), "cuda")
+            per_layer.append(ms / (reps * self.n_sets))
+            total_s += ms * 1e-3
+        return per_layer, total_s
 
     def barrier(self):
         import torch.distributed as dist
@@ -467,11 +502,12 @@ def run_cuda(args, w, name):
     if sampler:
         sampler.start()
         time.sleep(0.3)
-    # The headline region carries no events between its calls (an event record between two kernels keeps the second
-    # from starting its launch early); the same K steps are then repeated as direct calls with every backward call
-    # bracketed, which gives the launch durations the roofline figure uses.
+    # The headline region replays whole captured steps.  The launch durations the roofline figure uses come from a
+    # second set of replays that hold only the backward calls, layer by layer (events between the calls of a step
+    # would keep a kernel from starting its launch early, and direct calls would put the host's pace into the figure).
     total_ms = job.timed_graphs(args.steps) if args.launch == "graph" else job.timed_calls(args.steps, inner_events=False)[0]
-    calls_ms, layer_ms = job.timed_calls(args.steps)
+    reps = max(1, -(-args.steps // job.n_sets))                    # about K launches of every layer's backward call
+    layer_ms, layer_s = job.timed_backward_graphs(w["keep_ratio"], reps)
     clocks = sampler.stop() if sampler else None
     assert int(job.status.item()) == 0, "device status word set during the timed steps"
     flops_step = flops_of(w, M_keep)
@@ -491,14 +527,16 @@ def run_cuda(args, w, name):
                           "launch": "direct C-ABI calls"}
 
     # ---- the same kernels over the keep-ratio sweep: backward time, speed-up against keep ratio 1.0, saved activations ----
-    sweep_steps = max(3, args.steps // 4)
+    sweep_reps = max(2, reps // 4)
     sweep = {}
     for r in sorted(set(w["sweep"]) | {1.0}):
-        for i in range(3):
-            job.step(i, r)
-        step_ms, per_layer = job.timed_calls(sweep_steps, r=r)
+        per_layer = layer_ms if r == w["keep_ratio"] else job.timed_backward_graphs(r, sweep_reps)[0]
+        if r == w["keep_ratio"]:
+            for k in range(job.n_sets):
+                job.step(k, r)
+            job.barrier()
         mk = job.m_keep()
-        sweep[r] = dict(M_keep=mk, ms_per_step=step_ms / sweep_steps, bwd_ms=per_layer, bwd_ms_total=sum(per_layer),
+        sweep[r] = dict(M_keep=mk, bwd_ms=per_layer, bwd_ms_total=sum(per_layer),
                         tflops_bwd=flops_of(w, mk) / (sum(per_layer) * 1e-3) / 1e12)
     for r, s in sweep.items():
         s["bwd_speedup_vs_keep1"] = sweep[1.0]["bwd_ms_total"] / s["bwd_ms_total"]
@@ -514,7 +552,7 @@ def run_cuda(args, w, name):
 
     if rank == 0:
         print(json.dumps(json_line(args, w, name, job, world, dict(
-            total_ms=total_ms, calls_ms=calls_ms, layer_ms=layer_ms, clocks=clocks, value=value, M_keep=M_keep,
+            total_ms=total_ms, calls_ms=layer_s * 1e3, layer_ms=layer_ms, clocks=clocks, value=value, M_keep=M_keep,
             with_allreduce=with_allreduce, sweep=sweep, e2e_ms=e2e_ms, e2e_steps=e2e_steps, e2e_value=e2e_value, h2d=h2d, d2h=d2h,
             warmup=warmup))))
     if dist.is_initialized():
@@ -844,6 +882,7 @@ def attention_layers(bench, pk):
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     out_rows = []
     for name, r, flags, lists in (("Drop QKV r=0.25", 0.25, 0, True), ("Drop QKV r=0.5", 0.5, 0, True), ("Drop QKV r=0.75", 0.75, 0, True),
+                                  ("Drop QKV r=0.5, kept rows only (no zero rows written)", 0.5, sbp.SBP_FLAG_ATTN_KEPT_ROWS_ONLY, True),
                                   ("Drop Query only r=0.5", 0.5, sbp.SBP_FLAG_ATTN_ALL_KEYS, True),
                                   ("all tokens (keep ratio 1.0)", 1.0, sbp.SBP_FLAG_ATTN_ALL_KEYS, False)):
         cap = sbp.sbp_keep_count(0, H, W_, r)
@@ -864,7 +903,7 @@ def attention_layers(bench, pk):
         nk = N if (flags & sbp.SBP_FLAG_ATTN_ALL_KEYS) else cap
         flop = 10.0 * nq * nk * d * B * heads
         # kept rows of Q and dA, of K and V read; kept rows of dQ, dK, dV written, zeros in all their other rows
-        by = (2.0 * nq + 2.0 * nk) * B * C * 2 + 3.0 * M * C * 2
+        by = (2.0 * nq + 2.0 * nk) * B * C * 2 + (3.0 * M * C * 2 if not (flags & sbp.SBP_FLAG_ATTN_KEPT_ROWS_ONLY) else (nq + 2.0 * nk) * B * C * 2)
         tmin = max(flop / (pk["bf16_tflops_sustained"] * 1e12), by / (pk["hbm_gbs"] * 1e9)) * 1e6
         out_rows.append((name, nq, nk, us, tmin, flop / us / 1e6, by / us / 1e3))
     assert int(st.item()) == 0

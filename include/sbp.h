@@ -69,7 +69,8 @@ enum {
     SBP_FLAG_DY_COMPACT = 16, /* dY holds only the kept rows, packed: [M_keep_cap, C_out] (chained layers, Sec. 3.3.1) */
     SBP_FLAG_DX_COMPACT = 32, /* dX receives only the kept rows, packed: [M_keep_cap, C_in]; no zero rows are written */
     SBP_FLAG_W_OUT_IN = 64,   /* W, and dW, are stored [C_out, C_in] (the usual layout of framework linear layers) */
-    SBP_FLAG_ATTN_ALL_KEYS = 128 /* sbp_attention_backward: keys and values are all tokens, only queries are dropped */
+    SBP_FLAG_ATTN_ALL_KEYS = 128, /* sbp_attention_backward: keys and values are all tokens, only queries are dropped */
+    SBP_FLAG_ATTN_KEPT_ROWS_ONLY = 256 /* sbp_attention_backward: write only the rows in the token lists, leave every other row alone */
 };
 
 const char* sbp_status_string(sbp_status s);
@@ -292,7 +293,9 @@ sbp_status sbp_patch_scatter(sbp_dtype dt, const void* dX_patches /* dev */, int
  *   S_ij  = softmax over j in Zk of q_i . k_j / sqrt(d)                 i in Zq   (recomputed; no attention map is cached)
  *   dS_ij = dA_i . v_j,   dM_ij = S_ij (dS_ij - sum_l S_il dS_il)
  *   dQ_i  = sum_j dM_ij k_j / sqrt(d),  dK_j = sum_i dM_ij q_i / sqrt(d),  dV_j = sum_i S_ij dA_i
- *   rows of dQ outside Zq and rows of dK, dV outside Zk = +0.0 (their gradient is dropped)
+ *   rows of dQ outside Zq and rows of dK, dV outside Zk = +0.0 (their gradient is dropped); with
+ *   SBP_FLAG_ATTN_KEPT_ROWS_ONLY those rows are not written at all - enough when the outputs feed an
+ *   sbp_linear_backward with the same keep list, which reads the kept rows only
  * Which subsets:
  *   Drop QKV (what the paper applies to image transformers): kv_rows = NULL, flags = 0: Zk = Zq = the kept tokens;
  *     the gradient path is attention among the kept tokens (the wrapped-operation reading of Algorithm 1; its maps

@@ -24,6 +24,7 @@ SBP_ACT_GELU = 0
 SBP_MASK_RANDOM, SBP_MASK_GRID, SBP_MASK_TEMPORAL, SBP_MASK_TEMPORAL_GRID = 0, 1, 2, 3
 SBP_FLAG_SHARE_MASK, SBP_FLAG_ACCUMULATE, SBP_FLAG_VALIDATE, SBP_FLAG_PLAIN_FMA = 1, 2, 4, 8
 SBP_FLAG_DY_COMPACT, SBP_FLAG_DX_COMPACT, SBP_FLAG_W_OUT_IN, SBP_FLAG_ATTN_ALL_KEYS = 16, 32, 64, 128
+SBP_FLAG_ATTN_KEPT_ROWS_ONLY = 256
 
 EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forward_cache", "sbp_linear_forward",
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",

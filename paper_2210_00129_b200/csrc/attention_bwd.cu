@@ -689,7 +689,7 @@ int64_t attention_max_tokens() { return kMaxTok; }
 cudaError_t launch_attention_backward(const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA, int64_t ld_da,
                                       const int32_t* q_rows, const int32_t* q_offs, const int32_t* k_rows, const int32_t* k_offs,
                                       int64_t B, int64_t N, int64_t heads, int64_t most_tokens, void* dQ, void* dK, void* dV,
-                                      int64_t ld_out, int32_t* status_word, cudaStream_t stream) {
+                                      int64_t ld_out, bool zero_other_rows, int32_t* status_word, cudaStream_t stream) {
     AttnParams prm;
     prm.Q = static_cast<const __nv_bfloat16*>(Q); prm.K = static_cast<const __nv_bfloat16*>(K);
     prm.V = static_cast<const __nv_bfloat16*>(V); prm.dA = static_cast<const __nv_bfloat16*>(dA);
@@ -701,7 +701,7 @@ cudaError_t launch_attention_backward(const void* Q, const void* K, const void* 
     prm.status_word = status_word;
     const int64_t problems = B * heads;
     // the zeros first: they touch only rows outside the lists, the products only rows inside them
-    if (q_rows != nullptr || k_rows != nullptr) {
+    if (zero_other_rows && (q_rows != nullptr || k_rows != nullptr)) {
         ZeroJob job;
         job.out[0] = prm.dQ; job.rows[0] = q_rows; job.total[0] = q_rows ? q_offs + B : nullptr;
         job.out[1] = prm.dK; job.rows[1] = k_rows; job.total[1] = k_rows ? k_offs + B : nullptr;

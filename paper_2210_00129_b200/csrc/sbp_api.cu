@@ -407,7 +407,7 @@ sbp_status sbp_attention_backward(sbp_dtype dt, const void* Q, const void* K, co
         return SBP_ERR_INVALID_ARG;
     if ((q_rows == nullptr) != (q_offsets == nullptr) || (kv_rows == nullptr) != (kv_offsets == nullptr))
         return SBP_ERR_INVALID_ARG;
-    if (flags & ~(uint32_t)SBP_FLAG_ATTN_ALL_KEYS) return SBP_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(SBP_FLAG_ATTN_ALL_KEYS | SBP_FLAG_ATTN_KEPT_ROWS_ONLY)) return SBP_ERR_INVALID_ARG;
     if ((flags & SBP_FLAG_ATTN_ALL_KEYS) && kv_rows != nullptr) return SBP_ERR_INVALID_ARG;
     const int64_t C = heads * head_dim;
     if (ld_qkv < C || ld_da < C || ld_out < C) return SBP_ERR_INVALID_ARG;
@@ -427,7 +427,8 @@ sbp_status sbp_attention_backward(sbp_dtype dt, const void* Q, const void* K, co
     const int64_t most = any_all ? N : max_kept;
     if (most > attention_max_tokens()) return SBP_ERR_UNSUPPORTED;
     const cudaError_t e = launch_attention_backward(Q, K, V, ld_qkv, dA, ld_da, q_rows, q_offsets, k_rows, k_offs, B, N, heads, most,
-                                                    dQ, dK, dV, ld_out, status_word, (cudaStream_t)stream);
+                                                    dQ, dK, dV, ld_out, (flags & SBP_FLAG_ATTN_KEPT_ROWS_ONLY) == 0, status_word,
+                                                    (cudaStream_t)stream);
     return e == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
 }
 

@@ -206,7 +206,7 @@ int64_t attention_max_tokens();
 cudaError_t launch_attention_backward(const void* Q, const void* K, const void* V, int64_t ld_qkv, const void* dA, int64_t ld_da,
                                       const int32_t* q_rows, const int32_t* q_offs, const int32_t* k_rows, const int32_t* k_offs,
                                       int64_t B, int64_t N, int64_t heads, int64_t most_tokens, void* dQ, void* dK, void* dV,
-                                      int64_t ld_out, int32_t* status_word, cudaStream_t stream);
+                                      int64_t ld_out, bool zero_other_rows, int32_t* status_word, cudaStream_t stream);
 
 // tcgen05 / TMEM bf16 products
 bool   tc_shapes_supported(int64_t M, int64_t M_keep_cap, int64_t C_in, int64_t C_out);

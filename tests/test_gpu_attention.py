@@ -108,6 +108,21 @@ def test_attention_backward_matches_the_oracle(B, H, W, heads, r, mode, variant,
     print(variant, r, errs)
 
 
+def test_kept_rows_only_leaves_the_other_rows_alone():
+    B, H, W, heads = 3, 14, 14, 2
+    N, M = H * W, B * H * W
+    Q, K, V, dA = _inputs(M, heads, 55, False)
+    rows_d, offs_d, cap = run_sample_keep(0, B, H, W, 0.5, seed=8)
+    keep = host(rows_d)[:int(host(offs_d)[-1])]
+    full = _run(B, N, heads, Q, K, V, dA, (rows_d, offs_d), None, 0, cap, False)
+    part = _run(B, N, heads, Q, K, V, dA, (rows_d, offs_d), None, sbp.SBP_FLAG_ATTN_KEPT_ROWS_ONLY, cap, False)
+    other = np.ones(M, dtype=bool); other[keep] = False
+    nan_bits = host(torch.full((1,), float("nan"), dtype=torch.bfloat16, device="cuda"))[0]
+    for a, b in zip(full, part):
+        assert np.array_equal(a[keep], b[keep])
+        assert (b[other] == nan_bits).all()              # untouched: still the fill value of the test's output buffers
+
+
 def test_attention_backward_is_deterministic_and_checks_its_arguments():
     B, H, W, heads = 2, 14, 14, 2
     N, M, C = H * W, B * H * W, heads * D
@@ -128,5 +143,6 @@ def test_attention_backward_is_deterministic_and_checks_its_arguments():
     assert call(cap=0) == sbp.SBP_ERR_INVALID_ARG
     assert call(cap=N + 1) == sbp.SBP_ERR_INVALID_ARG
     assert call(flags=1) == sbp.SBP_ERR_INVALID_ARG
+    assert call(flags=512) == sbp.SBP_ERR_INVALID_ARG
     assert call(N=400, cap=300) == sbp.SBP_ERR_UNSUPPORTED          # more than 256 kept tokens per sample
     assert call(N=400, flags=sbp.SBP_FLAG_ATTN_ALL_KEYS) == sbp.SBP_ERR_UNSUPPORTED
