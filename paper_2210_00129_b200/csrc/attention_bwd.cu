@@ -38,6 +38,7 @@ struct AttnParams {
     int B, N, heads;
     __nv_bfloat16 *dQ, *dK, *dV;
     float scale;
+    int zero_fill;                // 1: the rows of a sample that its list leaves out are written as zeros
     int32_t* status_word;
 };
 
@@ -61,6 +62,35 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Zeros for one head's 64 columns in the rows of sample b that an ascending token list leaves out.  `glob` holds the
+// global row of every listed token of the sample (shared memory, filled by the block before the barrier in front of
+// this call).  Eight threads share a row (one 128-byte line, 16 bytes each, so that a warp's store covers four whole
+// lines); such a group takes the runs of rows in front of listed token g, g + groups, ..., the run behind the last
+// token counting as one more.  Rows are clamped to the sample, so that a list that breaks the ascending order cannot
+// send a store anywhere else.  The stores are fire and forget: issued while the first products run.
+__device__ __forceinline__ void zero_gap_rows(__nv_bfloat16* out0, __nv_bfloat16* out1, int64_t ld, int col0, const int32_t* glob,
+                                              int count, int base_row, int N, int t, int threads) {
+    const int end = base_row + N;
+    const int chunk = (t & 7) * 8;
+    for (int g = t >> 3; g <= count; g += threads >> 3) {
+        int lo = g > 0 ? glob[g - 1] + 1 : base_row;
+        int hi = g < count ? glob[g] : end;
+        lo = lo < base_row ? base_row : lo;
+        hi = hi > end ? end : hi;
+        for (int r = lo; r < hi; ++r) {
+            ptx::st_global_v4(out0 + (int64_t)r * ld + col0 + chunk, 0u, 0u, 0u, 0u);
+            if (out1 != nullptr) ptx::st_global_v4(out1 + (int64_t)r * ld + col0 + chunk, 0u, 0u, 0u, 0u);
+        }
+    }
+}
+__device__ __forceinline__ void zero_unlisted_rows(const AttnParams& p, int prob, int nq, int nk, const int32_t* q_glob,
+                                                   const int32_t* k_glob, int t, int threads) {
+    if (!p.zero_fill) return;
+    const int b = prob / p.heads, col0 = (prob % p.heads) * kD;
+    if (p.q_rows != nullptr) zero_gap_rows(p.dQ, nullptr, p.ld_out, col0, q_glob, nq, b * p.N, p.N, t, threads);
+    if (p.k_rows != nullptr) zero_gap_rows(p.dK, p.dV, p.ld_out, col0, k_glob, nk, b * p.N, p.N, t, threads);
 }
 
 // What a thread needs to know about a problem before it can start its copies: the token counts, the global rows
@@ -151,11 +181,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
             load_rows_big(sK, p.K, p.ld_qkv, cur.kid, nk, col0);
             load_rows_big(sDA, p.dA, p.ld_da, cur.qid, nq, col0);
             load_rows_big(sV, p.V, p.ld_qkv, cur.kid, nk, col0);
-            sh.q_glob[threadIdx.x] = cur.q_glob;
-            sh.k_glob[threadIdx.x] = cur.k_glob;
         }
+        sh.q_glob[threadIdx.x] = cur.q_glob;
+        sh.k_glob[threadIdx.x] = cur.k_glob;
         cur = fetch_big_meta(p, prob + (int)gridDim.x);      // the next problem's indices travel while this one computes
-        if (nq <= 0 || nk <= 0) continue;
+        if (nq <= 0 || nk <= 0) {                            // nothing to compute: only the zeros of the unlisted rows
+            __syncthreads();
+            zero_unlisted_rows(p, prob, nq, nk, sh.q_glob, sh.k_glob, (int)threadIdx.x, kAttnThreads);
+            __syncthreads();
+            continue;
+        }
         const int QT = (nq + 127) >> 7, KT = (nk + 127) >> 7;
         const int keys_pad = (nk + 15) & ~15;               // accumulator columns of the first pass (a multiple of 16)
         ptx::cp_async_wait_all();
@@ -176,6 +211,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
                 }
                 ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
             }
+            if (qt == 0) zero_unlisted_rows(p, prob, nq, nk, sh.q_glob, sh.k_glob, (int)threadIdx.x, kAttnThreads);
             ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_s), n_s & 1u, abort_flag, p.status_word);
             ++n_s;
             ok = !__syncthreads_or(!ok);
@@ -183,20 +219,21 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
             ptx::tc_fence_after_sync();
             // this thread: row `row`, columns [128 half, 128 half + 128) below keys_pad; two sweeps (maximum; sums)
             const int cbeg = half * 128, cend = keys_pad < cbeg + 128 ? keys_pad : cbeg + 128;
-            float mx = -INFINITY;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four interleaved chains, not one long one
             for (int c = cbeg; c < cend; c += 32) {
                 float s[32];
                 ptx::tmem_ld_32x32(tmem + kColS1 + (uint32_t)c + lane_off, s);
                 ptx::tmem_ld_wait();
                 if (c + 32 <= nk) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) mx = fmaxf(mx, s[j]);
+                    for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], s[j]);
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) mx = fmaxf(mx, (c + j < nk) ? s[j] : -INFINITY);
+                    for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], (c + j < nk) ? s[j] : -INFINITY);
                 }
             }
-            float l = 0.f, u_acc = 0.f;
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            float l4[4] = {0.f, 0.f, 0.f, 0.f}, u4[4] = {0.f, 0.f, 0.f, 0.f};
             if (mx > -INFINITY) {
                 const float nm = -mx * sl2;
                 for (int c = cbeg; c < cend; c += 32) {
@@ -212,11 +249,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_bwd_kernel(const At
                             e = (c + j < nk) ? e : 0.f;
                             g = (c + j < nk) ? g : 0.f;
                         }
-                        l += e;
-                        u_acc = fmaf(e, g, u_acc);
+                        l4[j & 3] += e;
+                        u4[j & 3] = fmaf(e, g, u4[j & 3]);
                     }
                 }
             }
+            const float l = (l4[0] + l4[1]) + (l4[2] + l4[3]), u_acc = (u4[0] + u4[1]) + (u4[2] + u4[3]);
             sh.part[half][row][0] = mx; sh.part[half][row][1] = l; sh.part[half][row][2] = u_acc;
             ptx::tc_fence_before_sync();
             __syncthreads();
@@ -393,6 +431,7 @@ struct SmallShared {
     uint64_t bar_s, bar_o;
     uint32_t tmem_slot;
     int abort_flag;
+    int32_t q_glob[kSmallThreads], k_glob[kSmallThreads];   // global row of every query / key of the problem (-1: none)
 };
 
 // What a thread needs to know about a problem before it can start its copies: the token counts, the global rows
@@ -482,8 +521,17 @@ __global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(c
             load_rows_small(sDA, p.dA, p.ld_da, cur.qid, nq, col0);
             load_rows_small(sV, p.V, p.ld_qkv, cur.kid, nk, col0);
         }
+        if (p.zero_fill) {
+            sh.q_glob[threadIdx.x] = q_out;
+            sh.k_glob[threadIdx.x] = k_out;
+        }
         cur = fetch_meta(p, prob + (int)gridDim.x);          // the next problem's indices travel while this one computes
-        if (nq <= 0 || nk <= 0) continue;
+        if (nq <= 0 || nk <= 0) {                            // nothing to compute: only the zeros of the unlisted rows
+            __syncthreads();
+            zero_unlisted_rows(p, prob, nq, nk, sh.q_glob, sh.k_glob, (int)threadIdx.x, kSmallThreads);
+            __syncthreads();
+            continue;
+        }
         const uint32_t q_steps = (uint32_t)(nq + 15) >> 4, k_steps = (uint32_t)(nk + 15) >> 4;   // 16-row steps that hold tokens
         const uint32_t n_keys = k_steps * 16u;              // accumulator columns computed (a multiple of 16)
         ptx::cp_async_wait_all();
@@ -499,6 +547,7 @@ __global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(c
             }
             ptx::umma_commit(ptx::smem_addr(&sh.bar_s));
         }
+        zero_unlisted_rows(p, prob, nq, nk, sh.q_glob, sh.k_glob, (int)threadIdx.x, kSmallThreads);
         ok = ptx::mbar_wait(ptx::smem_addr(&sh.bar_s), n_s & 1u, abort_flag, p.status_word);
         ++n_s;
         ok = !__syncthreads_or(!ok);
@@ -507,21 +556,22 @@ __global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(c
         // ---- this thread's row of S and dS, three sweeps over the accumulators: the maximum; the sum and
         //      rowsum(e^(s - m) dS); then the S block to shared memory with dM kept in registers.  Columns from nk on
         //      (padding keys, stale columns past n_keys) are masked; only the chunk holding column nk pays for it. ----
-        float mx = -INFINITY;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four interleaved chains, not one of n_keys links
         for (uint32_t c = 0; c < n_keys; c += 32) {
             float s[32];
             ptx::tmem_ld_32x32(tmem + c + lane_off, s);
             ptx::tmem_ld_wait();
             if ((int)c + 32 <= nk) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, s[j]);
+                for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], s[j]);
             } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, ((int)c + j < nk) ? s[j] : -INFINITY);
+                for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], ((int)c + j < nk) ? s[j] : -INFINITY);
             }
         }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         const float nm = -mx * sl2;
-        float l = 0.f, u_acc = 0.f;
+        float l4[4] = {0.f, 0.f, 0.f, 0.f}, u4[4] = {0.f, 0.f, 0.f, 0.f};
         for (uint32_t c = 0; c < n_keys; c += 32) {
             float s[32], ds[32];
             ptx::tmem_ld_32x32(tmem + c + lane_off, s);
@@ -535,10 +585,11 @@ __global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(c
                     e = ((int)c + j < nk) ? e : 0.f;
                     g = ((int)c + j < nk) ? g : 0.f;
                 }
-                l += e;
-                u_acc = fmaf(e, g, u_acc);
+                l4[j & 3] += e;
+                u4[j & 3] = fmaf(e, g, u4[j & 3]);
             }
         }
+        const float l = (l4[0] + l4[1]) + (l4[2] + l4[3]), u_acc = (u4[0] + u4[1]) + (u4[2] + u4[3]);
         const float inv_l = 1.f / l;
         const float nds = -u_acc * inv_l * p.scale;         // -rowsum(S dS) / sqrt(d)
         uint32_t dm[64];
@@ -658,29 +709,6 @@ __global__ void __launch_bounds__(kSmallThreads, 2) attention_bwd_small_kernel(c
 
 // rows of an output [M, ld] (columns [0, cols)) that are not in its ascending list rows[0 .. *total) become +0.0:
 // entry m of the list owns the gap in front of it, one extra worker the tail; blockIdx.y picks the output
-struct ZeroJob {
-    __nv_bfloat16* out[3];
-    const int32_t* rows[3];
-    const int32_t* total[3];
-};
-__global__ void zero_rows_outside_kernel(const ZeroJob job, int64_t M, int64_t ld, int cols, const int32_t* status_word) {
-    pdl_launch_dependents();
-    pdl_wait();
-    if (status_word != nullptr && *reinterpret_cast<const volatile int32_t*>(status_word) != 0) return;
-    const int32_t* rows = job.rows[blockIdx.y];
-    if (rows == nullptr) return;
-    __nv_bfloat16* out = job.out[blockIdx.y];
-    const int64_t total = __ldg(job.total[blockIdx.y]);
-    const int lane = threadIdx.x & 31;
-    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t m = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); m <= total; m += warps) {
-        const int64_t lo = m > 0 ? (int64_t)__ldg(rows + m - 1) + 1 : 0;
-        const int64_t hi = m < total ? (int64_t)__ldg(rows + m) : M;
-        for (int64_t r = lo; r < hi; ++r)
-            for (int c = lane * 8; c < cols; c += 256) ptx::st_global_v4(out + r * ld + c, 0u, 0u, 0u, 0u);
-    }
-}
-
 }  // namespace
 
 bool attention_supported(sbp_dtype dt, int64_t head_dim) { return dt == SBP_BF16 && head_dim == kD; }
@@ -700,16 +728,8 @@ cudaError_t launch_attention_backward(const void* Q, const void* K, const void* 
     prm.scale = 1.0f / sqrtf((float)kD);
     prm.status_word = status_word;
     const int64_t problems = B * heads;
-    // the zeros first: they touch only rows outside the lists, the products only rows inside them
-    if (zero_other_rows && (q_rows != nullptr || k_rows != nullptr)) {
-        ZeroJob job;
-        job.out[0] = prm.dQ; job.rows[0] = q_rows; job.total[0] = q_rows ? q_offs + B : nullptr;
-        job.out[1] = prm.dK; job.rows[1] = k_rows; job.total[1] = k_rows ? k_offs + B : nullptr;
-        job.out[2] = prm.dV; job.rows[2] = k_rows; job.total[2] = k_rows ? k_offs + B : nullptr;
-        const cudaError_t e = launch_pdl(zero_rows_outside_kernel, dim3(kNumSMs, 3), dim3(256), 0, stream, job, B * N, ld_out,
-                                         (int)(heads * kD), (const int32_t*)status_word);
-        if (e != cudaSuccess) return e;
-    }
+    // the zeros for the rows outside the lists are written by the same kernel, between a problem's copies and its products
+    prm.zero_fill = (zero_other_rows && (q_rows != nullptr || k_rows != nullptr)) ? 1 : 0;
     if (most_tokens <= 128) {
         const cudaError_t opt = opt_in_dynamic_smem<attention_bwd_small_kernel>((int)kSmallSmem);
         if (opt != cudaSuccess) return opt;
