@@ -1054,6 +1054,17 @@ def run_probes(args):
                     per_kb = c / iters / acc                      # per accumulator chain and k-block
                     ideal = 128.0 * N * 64 / 4096.0
                     print(f"| {blocks} block(s) | {'MN-major' if mn else 'K-major'} | {N} | {acc} | {c / (iters * 4 * acc):.1f} | {per_kb:.0f} | {ideal:.0f} | {ideal / per_kb:.2f} |")
+    print("\n| tcgen05.mma.cta_group::2, M = 256 over two SMs, K = 16, bf16 | operands | N | clocks per instruction | ideal per SM (4096 MAC/clk) | fraction |")
+    print("|---|---|---|---|---|---|")
+    for pairs in (1, 74):
+        for mn in (0, 1):
+            for N in (64, 128, 256):
+                sbp.sbp_probe_mma_pair_rate(N, mn, iters, pairs, cyc, st)
+                sbp.sbp_probe_mma_pair_rate(N, mn, iters, pairs, cyc, st)
+                torch.cuda.synchronize()
+                c = int(cyc.item()) / (iters * 4)
+                ideal = 128.0 * N * 16 / 4096.0
+                print(f"| {pairs} pair(s) | {'MN-major' if mn else 'K-major'} | {N} | {c:.1f} | {ideal:.0f} | {ideal / c:.2f} |")
     assert int(st.item()) == 0, "device status word set by a probe"
 
 

@@ -405,12 +405,17 @@ sbp_status sbp_selftest_bounded_wait(double limit_ms, int32_t* status_word /* de
  *   16 up to 256, operands K-major or MN-major) into one accumulator, or alternating between two accumulators 256
  *   columns apart (accumulators = 2: 8 * iters instructions); cycles_out[0] (dev) receives the SM clocks from the
  *   first issue to the completion of the last instruction on block 0, or -1 if the bounded wait ran out.
+ * sbp_probe_mma_pair_rate: the same stream in the two-SM form: `pairs` clusters of two blocks, the first block's
+ *   thread issuing 4 * iters tcgen05.mma.cta_group::2 (M = 256 over the pair, N a multiple of 32 up to 256, each SM
+ *   supplying its 128 rows of A and N / 2 rows of B); cycles_out[0] as above.
  * SBP_ERR_INVALID_ARG for sizes outside these ranges and null / misaligned pointers.
  */
 sbp_status sbp_probe_gather_ring(const void* src /* dev */, int64_t row_bytes, const int32_t* rows /* dev */, int64_t n_rows,
                                  int threads, int stages, int blocks, int32_t* status_word /* dev, nullable */, void* stream);
 sbp_status sbp_probe_mma_rate(int N, int mn_major, int accumulators, int iters, int blocks, int64_t* cycles_out /* dev */,
                               int32_t* status_word /* dev, nullable */, void* stream);
+sbp_status sbp_probe_mma_pair_rate(int N, int mn_major, int iters, int pairs, int64_t* cycles_out /* dev */,
+                                   int32_t* status_word /* dev, nullable */, void* stream);
 
 #ifdef __cplusplus
 }

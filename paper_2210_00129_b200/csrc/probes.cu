@@ -6,7 +6,8 @@
 //                kernel gathers the kept rows of dY; a consumer thread frees each stage as soon as it has landed.
 //                Nothing is computed: the time is what the gather path alone can sustain.
 //   mma rate:    one thread per block issues a stream of tcgen05.mma (M = 128, K = 16, bf16) of a given width on
-//                constant operands and reports the clocks from the first issue to the completion of the last.
+//                constant operands and reports the clocks from the first issue to the completion of the last; the pair
+//                variant issues the two-SM form (cta_group::2) from a cluster of two blocks.
 #include "tc_ptx.cuh"
 
 namespace sbp {
@@ -127,6 +128,65 @@ probe_mma_kernel(int N, int mn_major, int accumulators, int iters, long long* cy
     }
 }
 
+// The same stream issued for a pair of SMs: a cluster of two blocks, tensor memory allocated for the pair, and block 0's
+// thread 0 issuing tcgen05.mma.cta_group::2 (M = 256 over the pair: 128 accumulator rows in each SM; each SM supplies
+// its 128 rows of A and N / 2 rows of B from its own shared memory).  Block 1 only provides its operands and stays until
+// block 0 has seen the last product finish (cluster barrier, reached on every path).
+__global__ void __launch_bounds__(128, 1)
+probe_mma_pair_kernel(int N, int mn_major, int iters, long long* cycles_out, int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ ProbeShared sh;
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    for (uint32_t i = threadIdx.x; i < 48 * 1024 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem_raw + (base - raw))[i] = 0x3F803F80u;
+    uint32_t cta_rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(cta_rank));
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_addr(&sh.done), 1);
+        sh.abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    ptx::fence_async_proxy();
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_addr(&sh.tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    ptx::tc_fence_before_sync();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_slot);
+    if (cta_rank == 0 && threadIdx.x == 0) {
+        const uint32_t a_addr = base, b_addr = base + 16 * 1024;
+        const uint32_t idesc = ptx::umma_idesc_bf16(256, N, mn_major != 0, mn_major != 0);
+        const uint32_t k_step = mn_major ? 16u * 128u : 32u;
+        const uint32_t lbo = mn_major ? 64u * 128u : 16u;
+        const long long c0 = clock64();
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (uint32_t u = 0; u < 4; ++u) {
+                const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, 1024);
+                const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, 1024);
+                const uint32_t acc = (it | (int)u) != 0;
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\t"
+                    "setp.ne.b32 p, %4, 0;\n\t"
+                    "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                    ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+            }
+        }
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(ptx::smem_addr(&sh.done)) : "memory");
+        const bool ok = ptx::mbar_wait(ptx::smem_addr(&sh.done), 0, &sh.abort_flag, status_word);
+        const long long c1 = clock64();
+        if (blockIdx.x == 0) cycles_out[0] = ok ? c1 - c0 : -1;
+    }
+    ptx::tc_fence_before_sync();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (threadIdx.x < 32) {
+        ptx::tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
 }  // namespace
 }  // namespace sbp
 
@@ -170,6 +230,28 @@ sbp_status sbp_probe_mma_rate(int N, int mn_major, int accumulators, int iters, 
     probe_mma_kernel<<<blocks, 128, 50 * 1024, (cudaStream_t)stream>>>(N, mn_major, accumulators, iters, reinterpret_cast<long long*>(cycles_out),
                                                                        status_word);
     return cudaGetLastError() == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
+}
+
+sbp_status sbp_probe_mma_pair_rate(int N, int mn_major, int iters, int pairs, int64_t* cycles_out, int32_t* status_word, void* stream) {
+    using namespace sbp;
+    if (cycles_out == nullptr || (reinterpret_cast<uintptr_t>(cycles_out) & 7u)) return SBP_ERR_INVALID_ARG;
+    if (N < 32 || N > 256 || N % 32 != 0 || iters < 1 || iters > 100000 || pairs < 1 || pairs > kNumSMs / 2) return SBP_ERR_INVALID_ARG;
+    const cudaError_t e = opt_in_dynamic_smem<probe_mma_pair_kernel>(50 * 1024);
+    if (e != cudaSuccess) return SBP_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 50 * 1024;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t l = cudaLaunchKernelEx(&cfg, probe_mma_pair_kernel, N, mn_major, iters, reinterpret_cast<long long*>(cycles_out), status_word);
+    return (l == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SBP_OK : SBP_ERR_CUDA;
 }
 
 }  // extern "C"
