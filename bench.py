@@ -1039,6 +1039,28 @@ def run_probes(args):
                 gbs = n * rb / us / 1e3
                 print(f"| | {source} | {n} x {rb} | {blocks} | {threads} | {stages} x 16 KB | {us:.1f} | {gbs:.0f} | {gbs / blocks:.1f} |")
         del src
+    print("\n| operand feed per stage (gathered rows x 128 B + TMA boxes of 16 KB; sources L2-resident unless noted) | blocks | ring | us | "
+          "GB/s gathered | GB/s by TMA | GB/s per SM | clocks per stage at 1.9 GHz |")
+    print("|---|---|---|---|---|---|---|---|")
+    M, rb = 24576, 1024
+    src = torch.ones(M * rb, dtype=torch.uint8, device="cuda")
+    rows = torch.cat([torch.nonzero(torch.rand(M, device="cuda", generator=gen) < 0.5).flatten().to(torch.int32) for _ in range(4)]).contiguous()
+    dense = torch.ones(6144, 2048, dtype=torch.bfloat16, device="cuda")          # 24 MB
+    big_src = torch.ones(200704 * rb, dtype=torch.uint8, device="cuda")          # 205 MB: the gathered rows come from DRAM
+    big_rows = torch.nonzero(torch.rand(200704, device="cuda", generator=gen) < 0.5).flatten().to(torch.int32).contiguous()
+    steps = 512
+    for label, g_src, g_rows in (("", src, rows), (", gathered rows from DRAM", big_src, big_rows)):
+        for g, boxes in ((128, 0), (0, 1), (0, 2), (0, 3), (128, 2), (128, 1), (64, 2), (64, 3)):
+            if label and g == 0:
+                continue
+            stage = g * 128 + boxes * 16384
+            stages = min(12, (192 * 1024) // stage)
+            for blocks in (148, 74):
+                us = time_us(lambda: sbp.sbp_probe_operand_feed(g_src, rb, g_rows, int(g_rows.numel()), g, dense, 6144, 2048, boxes, stages, steps, blocks, st))
+                gg, gt = blocks * steps * g * 128 / us / 1e3, blocks * steps * boxes * 16384 / us / 1e3
+                print(f"| {g} rows + {boxes} boxes{label} | {blocks} | {stages} x {stage // 1024} KB | {us:.1f} | {gg:.0f} | {gt:.0f} | {(gg + gt) / blocks:.1f} | {us * 1e-6 / steps * 1.9e9:.0f} |")
+    del src, dense, big_src
+
     print("\n| tcgen05.mma, M = 128, K = 16, bf16 | operands | N | accumulators | clocks per instruction | clocks per 64-deep k-block | ideal (4096 MAC/clk) | fraction |")
     print("|---|---|---|---|---|---|---|---|")
     cyc = torch.zeros(1, dtype=torch.int64, device="cuda")

@@ -401,6 +401,10 @@ sbp_status sbp_selftest_bounded_wait(double limit_ms, int32_t* status_word /* de
  *   (2..12) 16 KB shared-memory stages per block, `threads` (64, 128 or 256) copying threads and `blocks` blocks, the
  *   way the backward kernel gathers the kept rows of dY; a consumer frees each stage as it lands.  Nothing is written
  *   to global memory.
+ * sbp_probe_operand_feed: the same ring fed by both producers of the backward kernel: per stage 64 threads gather
+ *   `gather_rows` (0, 64 or 128) rows x 128 bytes as above and one thread issues `tma_boxes` (0..3) TMA loads of 128 rows
+ *   x 128 bytes at scattered places of the bf16 matrix `dense` [dense_rows (multiple of 128), dense_cols (multiple of
+ *   64)]; each of `blocks` blocks runs `steps` stages through a ring of `stages` stages (at most 192 KB).
  * sbp_probe_mma_rate: one thread per block issues 4 * iters tcgen05.mma (M = 128, K = 16, bf16, width N a multiple of
  *   16 up to 256, operands K-major or MN-major) into one accumulator, or alternating between two accumulators 256
  *   columns apart (accumulators = 2: 8 * iters instructions); cycles_out[0] (dev) receives the SM clocks from the
@@ -412,6 +416,9 @@ sbp_status sbp_selftest_bounded_wait(double limit_ms, int32_t* status_word /* de
  */
 sbp_status sbp_probe_gather_ring(const void* src /* dev */, int64_t row_bytes, const int32_t* rows /* dev */, int64_t n_rows,
                                  int threads, int stages, int blocks, int32_t* status_word /* dev, nullable */, void* stream);
+sbp_status sbp_probe_operand_feed(const void* src /* dev */, int64_t row_bytes, const int32_t* rows /* dev */, int64_t n_rows,
+                                  int gather_rows, const void* dense /* dev */, int64_t dense_rows, int64_t dense_cols, int tma_boxes,
+                                  int stages, int steps, int blocks, int32_t* status_word /* dev, nullable */, void* stream);
 sbp_status sbp_probe_mma_rate(int N, int mn_major, int accumulators, int iters, int blocks, int64_t* cycles_out /* dev */,
                               int32_t* status_word /* dev, nullable */, void* stream);
 sbp_status sbp_probe_mma_pair_rate(int N, int mn_major, int iters, int pairs, int64_t* cycles_out /* dev */,

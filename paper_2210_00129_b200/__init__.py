@@ -30,7 +30,7 @@ EXPORTS = ("sbp_status_string", "sbp_keep_count", "sbp_sample_keep", "sbp_forwar
            "sbp_linear_backward_workspace_bytes", "sbp_linear_backward", "sbp_linear_backward_kernel_count",
            "sbp_plan_search_count", "sbp_act_backward", "sbp_attention_backward", "sbp_patch_cache", "sbp_patch_scatter_workspace_bytes",
            "sbp_patch_scatter", "sbp_step_host_arena_bytes", "sbp_step_host", "sbp_bias_grad_static",
-           "sbp_selftest_bounded_wait", "sbp_probe_gather_ring", "sbp_probe_mma_rate", "sbp_probe_mma_pair_rate")
+           "sbp_selftest_bounded_wait", "sbp_probe_gather_ring", "sbp_probe_mma_rate", "sbp_probe_mma_pair_rate", "sbp_probe_operand_feed")
 
 _lib = None
 
@@ -83,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.sbp_probe_gather_ring.restype = ci
     lib.sbp_probe_mma_rate.argtypes = [ci, ci, ci, ci, ci, vp, vp, vp]
     lib.sbp_probe_mma_rate.restype = ci
+    lib.sbp_probe_operand_feed.argtypes = [vp, i64, vp, i64, ci, vp, i64, i64, ci, ci, ci, ci, vp, vp]
+    lib.sbp_probe_operand_feed.restype = ci
     lib.sbp_probe_mma_pair_rate.argtypes = [ci, ci, ci, ci, vp, vp, vp]
     lib.sbp_probe_mma_pair_rate.restype = ci
     lib.sbp_act_backward.argtypes = [ci, ci, vp, vp, vp, i64, i64, vp, vp, vp]
@@ -271,6 +273,16 @@ def sbp_probe_mma_rate(N, mn_major, accumulators, iters, blocks, cycles_out, sta
                                           _stream(stream))
     if check:
         _check(s, "sbp_probe_mma_rate")
+    return s
+
+
+def sbp_probe_operand_feed(src, row_bytes, rows, n_rows, gather_rows, dense, dense_rows, dense_cols, tma_boxes, stages, steps, blocks,
+                           status_word=None, stream=None, check=True) -> int:
+    """Diagnostic: the gather ring fed by cp.async gathers and TMA loads of a dense matrix together (nothing is computed)."""
+    s = load_library().sbp_probe_operand_feed(_ptr(src), row_bytes, _ptr(rows), n_rows, gather_rows, _ptr(dense), dense_rows, dense_cols,
+                                              tma_boxes, stages, steps, blocks, _ptr(status_word), _stream(stream))
+    if check:
+        _check(s, "sbp_probe_operand_feed")
     return s
 
 

@@ -5,6 +5,8 @@
 //                stages (128 rows x 128 bytes, 128-byte swizzle) behind full / empty mbarriers, exactly as the backward
 //                kernel gathers the kept rows of dY; a consumer thread frees each stage as soon as it has landed.
 //                Nothing is computed: the time is what the gather path alone can sustain.
+//   operand feed: the gather ring together with a TMA producer that streams 16 KB boxes of a dense matrix into the same
+//                stages: what shared memory can be fed with per SM when both producers of the backward kernel run.
 //   mma rate:    one thread per block issues a stream of tcgen05.mma (M = 128, K = 16, bf16) of a given width on
 //                constant operands and reports the clocks from the first issue to the completion of the last; the pair
 //                variant issues the two-SM form (cta_group::2) from a cluster of two blocks.
@@ -128,6 +130,92 @@ probe_mma_kernel(int N, int mn_major, int accumulators, int iters, long long* cy
     }
 }
 
+// Operand feed: what the backward kernel's two producers deliver together.  Per stage, 64 threads gather `gather_rows`
+// (0, 64 or 128) rows x 128 bytes with 16-byte cp.async, as above, and one thread issues `tma_boxes` (0..3) TMA loads of
+// 128 rows x 128 bytes (16 KB, 128-byte swizzle) at scattered places of a dense bf16 matrix; a consumer thread frees the
+// stage as soon as everything has landed.  Nothing is computed and nothing is written to global memory.
+__global__ void __launch_bounds__(128, 1)
+probe_feed_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __restrict__ src, const int32_t* __restrict__ rows, int n_rows,
+                  int row_bytes, int gather_rows, int dense_row_boxes, int dense_col_boxes, int tma_boxes, int stages, int steps,
+                  int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ ProbeShared sh;
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;
+    const uint32_t stage_bytes = (uint32_t)gather_rows * 128u + (uint32_t)tma_boxes * 16384u;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            ptx::mbar_init(ptx::smem_addr(&sh.full[s]), 1 + (gather_rows > 0 ? 64 : 0));
+            ptx::mbar_init(ptx::smem_addr(&sh.empty[s]), 1);
+        }
+        sh.abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&map);
+    }
+    __syncthreads();
+    volatile int* abort_flag = &sh.abort_flag;
+    if (warp == 3) {                                        // consumer
+        if (threadIdx.x == 96)
+            for (int it = 0; it < steps; ++it) {
+                const int s = it % stages;
+                if (!ptx::mbar_wait(ptx::smem_addr(&sh.full[s]), (it / stages) & 1u, abort_flag, status_word)) break;
+                ptx::mbar_arrive(ptx::smem_addr(&sh.empty[s]));
+            }
+    } else if (warp == 2) {                                 // TMA producer
+        if (threadIdx.x == 64) {
+            int it = 0;
+            bool ok = true;
+            for (; it < steps; ++it) {
+                const int s = it % stages;
+                ok = ptx::mbar_wait(ptx::smem_addr(&sh.empty[s]), ((it / stages) & 1u) ^ 1u, abort_flag, status_word);
+                if (!ok) break;
+                const uint32_t full = ptx::smem_addr(&sh.full[s]);
+                ptx::mbar_arrive_expect_tx(full, (uint32_t)tma_boxes * 16384u);
+                const uint32_t dst = ring + s * stage_bytes + (uint32_t)gather_rows * 128u;
+                for (int b = 0; b < tma_boxes; ++b) {
+                    const int x = ((it * 7 + (int)blockIdx.x) % dense_col_boxes) * 64;
+                    const int y = ((it * 13 + (int)blockIdx.x * 31 + b * 5) % dense_row_boxes) * 128;
+                    ptx::tma_load_2d(dst + b * 16384u, &map, x, y, full);
+                }
+            }
+            if (!ok)                                        // let the loads already issued land before shared memory goes away
+                for (int j = (it > stages ? it - stages : 0); j < it; ++j)
+                    for (int spin = 0; spin < (1 << 14); ++spin)
+                        if (ptx::mbar_try_wait(ptx::smem_addr(&sh.full[j % stages]), (j / stages) & 1u)) break;
+        }
+    } else if (gather_rows > 0) {                           // gather producers: 8 rows x 128 bytes per pass of the 64 threads
+        // as in the backward kernel a tile's row pointers are fetched once and serve all its 128-byte pieces
+        const uint32_t chunk = threadIdx.x & 7u, sub = threadIdx.x >> 3;
+        const int pieces = row_bytes / 128;
+        int it = 0;
+        bool ok = true;
+        const int tiles = n_rows / gather_rows;             // the list is walked again from its start when it runs out
+        for (int tile = (int)blockIdx.x % tiles; ok && it < steps; tile = (tile + (int)gridDim.x) % tiles) {
+            const uint8_t* p[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int m = tile * gather_rows + (i * 8 + (int)sub) % gather_rows;
+                p[i] = src + (size_t)__ldg(rows + m) * row_bytes + chunk * 16;
+            }
+            for (int piece = 0; piece < pieces && it < steps; ++piece, ++it) {
+                const int s = it % stages;
+                ok = ptx::mbar_wait(ptx::smem_addr(&sh.empty[s]), ((it / stages) & 1u) ^ 1u, abort_flag, status_word);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t dst = ring + s * stage_bytes;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const uint32_t r = i * 8 + sub;
+                    if ((int)r < gather_rows) ptx::cp_async_16(dst + r * 128 + ((chunk ^ (r & 7u)) << 4), p[i] + piece * 128, 16u);
+                }
+                ptx::cp_async_arrive_noinc(ptx::smem_addr(&sh.full[s]));
+            }
+        }
+        ptx::cp_async_wait_all();
+    }
+}
+
 // The same stream issued for a pair of SMs: a cluster of two blocks, tensor memory allocated for the pair, and block 0's
 // thread 0 issuing tcgen05.mma.cta_group::2 (M = 256 over the pair: 128 accumulator rows in each SM; each SM supplies
 // its 128 rows of A and N / 2 rows of B from its own shared memory).  Block 1 only provides its operands and stays until
@@ -216,6 +304,44 @@ sbp_status sbp_probe_gather_ring(const void* src, int64_t row_bytes, const int32
     }
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return SBP_ERR_CUDA;
     return SBP_OK;
+}
+
+sbp_status sbp_probe_operand_feed(const void* src, int64_t row_bytes, const int32_t* rows, int64_t n_rows, int gather_rows,
+                                  const void* dense, int64_t dense_rows, int64_t dense_cols, int tma_boxes, int stages, int steps,
+                                  int blocks, int32_t* status_word, void* stream) {
+    using namespace sbp;
+    if (src == nullptr || rows == nullptr || dense == nullptr || (reinterpret_cast<uintptr_t>(src) & 15u) ||
+        (reinterpret_cast<uintptr_t>(dense) & 15u) || (reinterpret_cast<uintptr_t>(rows) & 3u))
+        return SBP_ERR_INVALID_ARG;
+    if (row_bytes < 128 || row_bytes % 128 != 0 || row_bytes > (1 << 20) || n_rows < 128 || n_rows >= (1ll << 31)) return SBP_ERR_INVALID_ARG;
+    if ((gather_rows != 0 && gather_rows != 64 && gather_rows != 128) || tma_boxes < 0 || tma_boxes > 3 || (gather_rows == 0 && tma_boxes == 0))
+        return SBP_ERR_INVALID_ARG;
+    if (dense_rows < 128 || dense_rows % 128 != 0 || dense_cols < 64 || dense_cols % 64 != 0 || dense_rows >= (1ll << 31) || dense_cols >= (1ll << 31))
+        return SBP_ERR_INVALID_ARG;
+    const size_t stage_bytes = (size_t)gather_rows * 128 + (size_t)tma_boxes * 16384;
+    if (stages < 2 || stages > 12 || (size_t)stages * stage_bytes > 192 * 1024 || steps < 1 || steps > (1 << 20) || blocks < 1 || blocks > kNumSMs)
+        return SBP_ERR_INVALID_ARG;
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                 const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || fn == nullptr)
+        return SBP_ERR_CUDA;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)dense_cols, (cuuint64_t)dense_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)dense_cols * 2};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    if (reinterpret_cast<EncodeFn>(fn)(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(dense), dims, strides, box, elem_strides,
+                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return SBP_ERR_CUDA;
+    const cudaError_t e = opt_in_dynamic_smem<probe_feed_kernel>(197 * 1024);
+    if (e != cudaSuccess) return SBP_ERR_CUDA;
+    probe_feed_kernel<<<blocks, 128, (size_t)stages * stage_bytes + 1024, (cudaStream_t)stream>>>(
+        map, (const uint8_t*)src, rows, (int)n_rows, (int)row_bytes, gather_rows, (int)(dense_rows / 128), (int)(dense_cols / 64), tma_boxes, stages,
+        steps, status_word);
+    return cudaGetLastError() == cudaSuccess ? SBP_OK : SBP_ERR_CUDA;
 }
 
 sbp_status sbp_probe_mma_rate(int N, int mn_major, int accumulators, int iters, int blocks, int64_t* cycles_out, int32_t* status_word,
