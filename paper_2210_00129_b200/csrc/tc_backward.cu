@@ -73,6 +73,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory per block");
 struct TcControl {
     uint64_t full_bar[kStagesNarrow];    // 1 arrival carrying the TMA byte count + one arrival per gather thread
     uint64_t empty_bar[kStagesNarrow];   // 1 arrival: tcgen05.commit of the MMAs that read the stage
+    uint64_t gather_bar[kStagesNarrow];  // pairs of blocks, odd block: one arrival per gather thread (forwarded to the even block)
     uint64_t acc_full[2];          // 1 arrival: all MMAs of the tile in this accumulator have finished
     uint64_t acc_empty[2];         // 4 arrivals: each epilogue warp has read the accumulator out
     uint32_t tmem_slot;
@@ -117,15 +118,16 @@ struct Tile {
     uint32_t split, kb_begin, num_kb;
 };
 
-template <int BNX, int BNW>
+// kTM: accumulator rows one worker's tile spans - 128 for a block, 256 for a pair of blocks (each block then takes half)
+template <int BNX, int BNW, int kTM>
 __device__ __forceinline__ Schedule make_schedule(const TcParams& p, int64_t M_keep) {
     Schedule s;
     s.x_ntiles = (uint32_t)((p.C_in + BNX - 1) / BNX);
-    s.x_tiles = (p.dX != nullptr) ? (uint32_t)((M_keep + kBM - 1) / kBM) * s.x_ntiles : 0u;
+    s.x_tiles = (p.dX != nullptr) ? (uint32_t)((M_keep + kTM - 1) / kTM) * s.x_ntiles : 0u;
     s.x_kb = (uint32_t)((p.C_out + kBK - 1) / kBK);
     s.splits = (uint32_t)p.dw_splits;
     s.w_ctiles = (uint32_t)((p.C_in + BNW - 1) / BNW);
-    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_out + kBM - 1) / kBM) * s.w_ctiles * s.splits : 0u;
+    s.w_tiles = (p.dW_out != nullptr) ? (uint32_t)((p.C_out + kTM - 1) / kTM) * s.w_ctiles * s.splits : 0u;
     s.w_kb_total = (uint32_t)((M_keep + kBK - 1) / kBK);
     s.w_kb_per = (s.w_kb_total + s.splits - 1) / s.splits;
     s.w_first = s.w_kb_per >= s.x_kb;
@@ -162,8 +164,8 @@ __device__ __forceinline__ Tile decode_tile(const Schedule& s, uint32_t q) {
 
 // CTA b takes list positions b, 2G-1-b, 2G+b, 4G-1-b, ...: with the list sorted by cost this
 // evens out the load without any run-time counter.
-__device__ __forceinline__ uint32_t list_position(uint32_t pass) {
-    const uint32_t G = gridDim.x, b = blockIdx.x;
+// (G workers, this one is number b: the blocks of the grid, or its pairs of blocks)
+__device__ __forceinline__ uint32_t list_position(uint32_t pass, uint32_t G, uint32_t b) {
     return pass * G + ((pass & 1u) ? (G - 1u - b) : b);
 }
 
@@ -174,21 +176,20 @@ __device__ __forceinline__ uint32_t list_position(uint32_t pass) {
 // then the second of every slab, ...).  Both groups then move through every slab of kept rows from its start to its
 // end at the same time, so each kept row of dY comes from DRAM once: whichever product reaches a row second finds
 // it in L2 (and, being served from L2, catches up with the other).
-__device__ __forceinline__ bool next_tile(const Schedule& s, uint32_t pass, Tile& t) {
+__device__ __forceinline__ bool next_tile(const Schedule& s, uint32_t pass, Tile& t, uint32_t G, uint32_t b) {
     if (s.dw_ctas == 0u) {
-        const uint32_t q = list_position(pass);
+        const uint32_t q = list_position(pass, G, b);
         if (q >= s.total) return false;
         t = decode_tile(s, q);
         return true;
     }
-    const uint32_t b = blockIdx.x;
     if (b < s.dw_ctas) {
         const uint32_t q = b + pass * s.dw_ctas;
         if (q >= s.w_tiles) return false;
         t = decode_tile(s, s.w_first ? q : s.x_tiles + q);
         return true;
     }
-    const uint32_t q = (b - s.dw_ctas) + pass * (gridDim.x - s.dw_ctas);
+    const uint32_t q = (b - s.dw_ctas) + pass * (G - s.dw_ctas);
     if (q >= s.x_tiles) return false;
     const uint32_t tr = q / s.x_ntiles;               // position of the row tile in the interleaved order
     const uint32_t lim = s.slab_len * s.splits;       // positions below this: every slab still has a tile at this depth
@@ -271,14 +272,29 @@ __device__ __forceinline__ void zero_dropped_rows(const TcParams& p, const Tile&
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int BNX, int BNW, int kBiasDepth, bool kPacked>
+// kPair (wide tiles only): the grid is made of clusters of two blocks that share every tile through the two-SM tensor-core
+// instructions (tcgen05.mma.cta_group::2, issued by the even block).  A tile then spans 256 accumulator rows, 128 in each
+// block - each block gathers, reads out and stores its own half exactly as it would a tile of its own - and the 256
+// columns of the dense operand are split: each block loads only 128 of them, and the tensor cores exchange the halves.
+// Measured on B200 a one-SM instruction of width 256 takes 171 clocks where the two-SM form takes the ideal 128, and a
+// block reads a third less shared memory per k-block (64 KB instead of 96 KB written and read), which is what held the
+// one-block form back.  What crosses the pair: the odd block's TMA loads credit their bytes to the even block's `full`
+// barrier; its gather lands on a local barrier that its (otherwise idle) warp 5 forwards with one remote arrival;
+// tcgen05.commit signals `empty` and `accumulator full` in both blocks at once; the odd block's epilogue warps release an
+// accumulator with remote arrivals.  Both blocks meet at a cluster barrier before either leaves.
+template <int BNX, int BNW, int kBiasDepth, bool kPacked, bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                    const __grid_constant__ CUtensorMap map_dw, const TcParams p) {
-    // narrow layers (both tile kinds 128 wide) move 32 KB per stage: six stages then fill the ring
+    // narrow layers (both tile kinds 128 wide) and pairs (half of a 256-wide dense tile per block) move 32 KB per stage:
+    // six stages then fill the ring
     constexpr bool kNarrow = BNX <= 128 && BNW <= 128;
-    constexpr int kS = kNarrow ? kStagesNarrow : kStages;
-    constexpr uint32_t kSB = kABytes + (kNarrow ? 128u : 256u) * kRowBytes;
+    static_assert(!kPair || (BNX == 256 && BNW == 256), "pairs of blocks run the wide tiles only");
+    constexpr int kS = (kNarrow || kPair) ? kStagesNarrow : kStages;
+    constexpr uint32_t kDenseRows = (kNarrow || kPair) ? 128u : 256u;        // rows of the dense operand a block holds per stage
+    constexpr uint32_t kSB = kABytes + kDenseRows * kRowBytes;
+    const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;                // 0: the block that issues the MMAs
+    const uint32_t workers = kPair ? gridDim.x >> 1 : gridDim.x, worker = kPair ? blockIdx.x >> 1 : blockIdx.x;
     extern __shared__ uint8_t smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t raw_addr = ptx::smem_addr(smem_raw);
@@ -289,12 +305,13 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kS; ++s) {
-            ptx::mbar_init(ptx::smem_addr(&ctl->full_bar[s]), 1 + kGatherThreads);
+            ptx::mbar_init(ptx::smem_addr(&ctl->full_bar[s]), 1 + kGatherThreads + (kPair ? 1 : 0));
             ptx::mbar_init(ptx::smem_addr(&ctl->empty_bar[s]), 1);
+            ptx::mbar_init(ptx::smem_addr(&ctl->gather_bar[s]), kGatherThreads);
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ptx::smem_addr(&ctl->acc_full[a]), 1);
-            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), 4);
+            ptx::mbar_init(ptx::smem_addr(&ctl->acc_empty[a]), kPair ? 8 : 4);
         }
         ctl->abort_flag = 0;
         ptx::fence_mbar_init();
@@ -315,9 +332,13 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         }
         ptx::fence_async_proxy();                                    // read by the tensor core (async proxy)
     }
-    if (warp == 5) ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
+    if (warp == 5) {
+        if constexpr (kPair) ptx::tmem_alloc_pair(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
+        else ptx::tmem_alloc(ptx::smem_addr(&ctl->tmem_slot), 2 * kAccCols);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if constexpr (kPair) ptx::cluster_sync_all();                    // the peer's barriers exist before anything is sent to them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctl->tmem_slot);
     volatile int* abort_flag = &ctl->abort_flag;
@@ -326,8 +347,14 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     pdl_wait();                                                      // from here on global memory is read
     const bool skip_all = status_word != nullptr && *reinterpret_cast<volatile int32_t*>(status_word) != 0;
     const int64_t M_keep = load_m_keep(p.M_keep_dev, p.M_keep_cap);
-    const Schedule sched = make_schedule<BNX, BNW>(p, M_keep);
+    const Schedule sched = make_schedule<BNX, BNW, kPair ? 2 * kBM : kBM>(p, M_keep);
     const int C_in = p.C_in, C_out = p.C_out;
+    // this block's tile of round `pass`: a pair's tile covers two 128-row tiles, one for each of its blocks
+    auto fetch_tile = [&](uint32_t pass, Tile& t) {
+        if (!next_tile(sched, pass, t, workers, worker)) return false;
+        if constexpr (kPair) t.row_tile = t.row_tile * 2u + rank;
+        return true;
+    };
 
     if (skip_all) {
         // an earlier check failed: leave every output untouched
@@ -338,14 +365,27 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             bool ok = true;
             for (uint32_t pass = 0; ok; ++pass) {
                 Tile t;
-                if (!next_tile(sched, pass, t)) break;
+                if (!fetch_tile(pass, t)) break;
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
                     const int s = it % kS;
                     ok = ptx::mbar_wait(ptx::smem_addr(&ctl->empty_bar[s]), ((it / kS) & 1u) ^ 1u, abort_flag, status_word);
                     if (!ok) break;
                     const uint32_t full = ptx::smem_addr(&ctl->full_bar[s]);
                     const uint32_t a_dst = ring + s * kSB;
-                    if (t.is_dw) {                                   // X_keep tile: BNW/64 blocks of 64 columns x 64 kept rows
+                    if constexpr (kPair) {
+                        // this block's 128 of the tile's 256 dense rows; the bytes of both blocks are credited to the even
+                        // block's barrier, which expects them all
+                        const uint32_t full0 = ptx::map_to_cta(full, 0);
+                        if (rank == 0) ptx::mbar_arrive_expect_tx(full, 256u * kRowBytes);
+                        if (t.is_dw) {
+                            const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.col_tile * BNW) + (int)rank * 128;
+#pragma unroll
+                            for (int b = 0; b < 2; ++b)
+                                ptx::tma_load_2d_pair(a_dst + kABytes + b * kBlock64Bytes, &map_x, i0 + b * 64, row0, full0);
+                        } else {
+                            ptx::tma_load_2d_pair(a_dst + kABytes, &map_w, (int)(k * kBK), (int)(t.col_tile * BNX) + (int)rank * 128, full0);
+                        }
+                    } else if (t.is_dw) {                            // X_keep tile: BNW/64 blocks of 64 columns x 64 kept rows
                         const int row0 = (int)((t.kb_begin + k) * kBK), i0 = (int)(t.col_tile * BNW);
                         ptx::mbar_arrive_expect_tx(full, BNW * kRowBytes);
 #pragma unroll
@@ -357,7 +397,9 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     }
                 }
             }
-            if (!ok) {   // let the copies already issued land before shared memory goes away
+            if (!ok && kPair) {   // (pairs: the barrier may be the peer's; a fixed pause, far longer than any copy takes)
+                for (int i = 0; i < 64; ++i) __nanosleep(1000);
+            } else if (!ok) {   // let the copies already issued land before shared memory goes away
                 for (uint32_t j = (it > (uint32_t)kS ? it - kS : 0u); j < it; ++j) {
                     const uint32_t bar = ptx::smem_addr(&ctl->full_bar[j % kS]);
                     for (int spin = 0; spin < (1 << 14); ++spin)
@@ -367,13 +409,13 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         }
         __syncwarp();
     } else if (warp == 5) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer (of the pair: the even block's) ----------------
+        if (lane == 0 && rank == 0) {
             uint32_t it = 0, used = 0;                               // stage uses, accumulator uses
             bool ok = true;
             for (uint32_t pass = 0; ok; ++pass) {
                 Tile t;
-                if (!next_tile(sched, pass, t)) break;
+                if (!fetch_tile(pass, t)) break;
                 if (t.num_kb == 0) continue;
                 const uint32_t acc = used & 1u;
                 ok = ptx::mbar_wait(ptx::smem_addr(&ctl->acc_empty[acc]), ((used >> 1) & 1u) ^ 1u, abort_flag, status_word);
@@ -385,8 +427,9 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                 const uint32_t bias_tmem = kNarrow ? d_tmem + 128u : tmem_base + (acc ^ 1u) * kAccCols;
                 // K-major (dX): a 16-deep slice is 32 bytes along the swizzled row, 8-row groups 1024 B apart.
                 // MN-major (dW): a 16-deep slice is 16 rows (two atoms); 64-wide blocks of the MN extent 8 KB apart.
-                const uint32_t idesc = t.is_dw ? ptx::umma_idesc_bf16(kBM, BNW, true, true)
-                                               : ptx::umma_idesc_bf16(kBM, BNX, false, false);
+                constexpr int kMmaM = kPair ? 2 * kBM : kBM;
+                const uint32_t idesc = t.is_dw ? ptx::umma_idesc_bf16(kMmaM, BNW, true, true)
+                                               : ptx::umma_idesc_bf16(kMmaM, BNX, false, false);
                 const uint32_t k_step = t.is_dw ? kUmmaK * kRowBytes : kUmmaK * 2;
                 const uint32_t lbo = t.is_dw ? kBlock64Bytes : 16;
                 for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
@@ -400,16 +443,37 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     for (uint32_t u = 0; u < kBK / kUmmaK; ++u) {
                         const uint64_t da = ptx::umma_desc_sw128(a_addr + u * k_step, lbo, kAtomBytes);
                         const uint64_t db = ptx::umma_desc_sw128(b_addr + u * k_step, lbo, kAtomBytes);
-                        ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
-                        if (t.is_dw && t.col_tile == 0 && p.db_from_mma) {   // the bias column: 16 more accumulator columns, the first is db
+                        if constexpr (kPair) ptx::umma_bf16_pair(d_tmem, da, db, idesc, (k | u) != 0u);
+                        else ptx::umma_bf16(d_tmem, da, db, idesc, (k | u) != 0u);
+                        if (!kPair && t.is_dw && t.col_tile == 0 && p.db_from_mma) {   // the bias column: 16 more accumulator columns, the first is db
                             const uint64_t d1 = ptx::umma_desc_sw128(raw_addr + ones_off + u * k_step, kBlock64Bytes, kAtomBytes);
                             ptx::umma_bf16(bias_tmem, da, d1, ptx::umma_idesc_bf16(kBM, 16, true, true), (k | u) != 0u);
                         }
                     }
-                    ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));      // stage reusable once these MMAs retire
+                    // stage reusable once these MMAs retire (pairs: in both blocks)
+                    if constexpr (kPair) ptx::umma_commit_pair(ptx::smem_addr(&ctl->empty_bar[s]));
+                    else ptx::umma_commit(ptx::smem_addr(&ctl->empty_bar[s]));
                 }
-                if (ok) ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
+                if (ok) {
+                    if constexpr (kPair) ptx::umma_commit_pair(ptx::smem_addr(&ctl->acc_full[acc]));
+                    else ptx::umma_commit(ptx::smem_addr(&ctl->acc_full[acc]));
+                }
                 ++used;
+            }
+        } else if (kPair && lane == 0) {
+            // ---------------- odd block of a pair: tell the issuer when this block's gathered rows have landed ----------------
+            uint32_t it = 0;
+            bool ok = true;
+            for (uint32_t pass = 0; ok; ++pass) {
+                Tile t;
+                if (!fetch_tile(pass, t)) break;
+                for (uint32_t k = 0; k < t.num_kb; ++k, ++it) {
+                    const int s = it % kS;
+                    ok = ptx::mbar_wait(ptx::smem_addr(&ctl->gather_bar[s]), (it / kS) & 1u, abort_flag, status_word);
+                    if (!ok) break;
+                    ptx::fence_async_proxy();                        // this block's tensor core reads what its cp.async wrote
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->full_bar[s]), 0));
+                }
             }
         }
         __syncwarp();
@@ -420,7 +484,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         bool ok = true;
         for (uint32_t pass = 0; ok; ++pass) {
             Tile t;
-            if (!next_tile(sched, pass, t)) break;
+            if (!fetch_tile(pass, t)) break;
             if (!t.is_dw) {
                 // dX tile: 128 kept rows x 128 bytes per stage; one warp instruction moves 4 rows x 128 B
                 constexpr int kInstr = 32 / kGatherWarps;
@@ -446,7 +510,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                     for (int i = 0; i < kInstr; ++i)
                         ptx::cp_async_16(a_dst + swizzled((gw * kInstr + i) * 4 + sub, chunk), src[i] + off, bytes);
                     // the stage's barrier gets this thread's arrival when the copies above have landed
-                    ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
+                    ptx::cp_async_arrive_noinc(ptx::smem_addr(rank == 0 ? &ctl->full_bar[s] : &ctl->gather_bar[s]));
                 }
             } else {
                 // dW tile: 64 kept rows x 128 columns (256 B) of dY per stage; one warp instruction moves 2 rows
@@ -493,7 +557,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             ptx::cp_async_16(a_dst + (c >> 3) * kBlock64Bytes + swizzled(gw * kRows + rl, c & 7u),
                                              col_ptr + (live ? (int64_t)g * C_out : 0), live ? 16u : 0u);
                         }
-                        ptx::cp_async_arrive_noinc(ptx::smem_addr(&ctl->full_bar[s]));
+                        ptx::cp_async_arrive_noinc(ptx::smem_addr(rank == 0 ? &ctl->full_bar[s] : &ctl->gather_bar[s]));
                         ++it;
                     }
                 }
@@ -505,7 +569,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         if (p.dX != nullptr && M_keep > 0) {
             for (uint32_t pass = 0;; ++pass) {
                 Tile t;
-                if (!next_tile(sched, pass, t)) break;
+                if (!fetch_tile(pass, t)) break;
                 if (!t.is_dw) zero_dropped_rows<BNX, kPacked>(p, t, M_keep, warp - kBiasWarp0, lane);
             }
         }
@@ -582,7 +646,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         bool ok = true;
         for (uint32_t pass = 0; ok; ++pass) {
             Tile t;
-            if (!next_tile(sched, pass, t)) break;
+            if (!fetch_tile(pass, t)) break;
             const uint32_t acc = used & 1u;
             const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
             if (!t.is_dw) {
@@ -673,7 +737,7 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
                             else ptx::bulk_wait_read<0>();
                         }
                         ptx::bar_named<kEpiBarrier, 128>();
-                        if (threadIdx.x == 0) {
+                        if (threadIdx.x == 0 && j0 < C_out) {            // (a pair's second block may hold columns past the end of dW)
                             if (add_in) ptx::tma_reduce_add_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
                             else ptx::tma_store_3d(&map_dw, raw_addr + buf_off, j0, i0 + c * kEpiChunk, (int)t.split);
                             ptx::bulk_commit();
@@ -689,16 +753,21 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
             // this warp is done with the accumulator: hand it back to the MMA issuer
             ptx::tc_fence_before_sync();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
+            if (lane == 0) {
+                if constexpr (kPair) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_addr(&ctl->acc_empty[acc]), 0));
+                else ptx::mbar_arrive(ptx::smem_addr(&ctl->acc_empty[acc]));
+            }
             ++used;
         }
     }
     if (threadIdx.x == 0) ptx::bulk_wait_all();                      // the TMA stores of the dW epilogue have landed
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if constexpr (kPair) ptx::cluster_sync_all();                    // neither block leaves while the other may still reach into it
     if (warp == 5) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, 2 * kAccCols);
+        if constexpr (kPair) ptx::tmem_dealloc_pair(tmem_base, 2 * kAccCols);
+        else ptx::tmem_dealloc(tmem_base, 2 * kAccCols);
     }
 }
 
@@ -751,14 +820,15 @@ struct Plan {
     int bnx, bnw;          // accumulator width of dX / dW tiles
     int splits;            // pieces each dW tile's reduction over kept rows is cut into
     int dw_ctas;           // role split: blocks given to the dW pieces (0 = one list for all blocks)
-    int64_t tiles;         // upper bound of the tile count (from the capacity)
+    bool pair;             // pairs of blocks share 256-row tiles through the two-SM tensor-core instructions
+    int64_t tiles;         // upper bound of the tile count (from the capacity); tiles of pairs when pair is set
 };
 
 // Estimated run time of the tile list for a given split count, in units of one dX k-block: the
 // longest per-block total under the kernel's own static assignment (block b takes list positions
 // b, 2G-1-b, 2G+b, ...), the epilogue of that block's last tile, and the reduce launch that
 // splitting costs.  The weights are measured ratios on ViT-B shapes; they only rank candidates.
-double estimate_cost(int64_t x_tiles, int64_t x_kb, int64_t w_tiles, int64_t w_kb, int64_t splits, int64_t dw_elems) {
+double estimate_cost(int64_t x_tiles, int64_t x_kb, int64_t w_tiles, int64_t w_kb, int64_t splits, int64_t dw_elems, int64_t workers) {
     constexpr double kDwKb = 1.12;        // a dW k-block (two gathered MN-major operands) relative to a dX one
     constexpr double kTileSwitch = 0.5;   // per tile: pipeline hand-over
     constexpr double kTailDx = 9.0, kTailDw = 6.0;   // exposed epilogue of the last tile
@@ -766,7 +836,7 @@ double estimate_cost(int64_t x_tiles, int64_t x_kb, int64_t w_tiles, int64_t w_k
     const int64_t w_pieces = w_tiles * splits;
     const int64_t total = x_tiles + w_pieces;
     if (total == 0) return 0.0;
-    const int64_t G = total < kNumSMs ? total : kNumSMs;
+    const int64_t G = total < workers ? total : workers;
     const bool w_first = kb_per >= x_kb;
     const int64_t first = w_first ? w_pieces : x_tiles;
     double worst = 0.0;
@@ -812,12 +882,22 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     Plan pl;
     pl.bnx = (C_in >= 256) ? 256 : 128;
     pl.bnw = (C_in >= 256) ? 256 : 128;
-    const int64_t x_tiles = want_dx ? ((M_keep_cap + kBM - 1) / kBM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
+    int64_t x_tiles = want_dx ? ((M_keep_cap + kBM - 1) / kBM) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
     const int64_t x_kb = (C_out + kBK - 1) / kBK;
-    const int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
+    int64_t w_tiles = want_dw ? ((C_out + kBM - 1) / kBM) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
     const int64_t w_kb = (M_keep_cap + kBK - 1) / kBK;
     pl.splits = 1;
     pl.dw_ctas = 0;
+    // Wide layers with enough work for every pair run as pairs of blocks unless the role split below takes them (the
+    // memory-bound layers gain nothing from the faster tensor-core form).
+    const bool memory_bound = 2.0 * (double)M_keep_cap * (double)(2 * C_in + C_out) / 6.5e12 >=
+                              0.75 * 4.0 * (double)M_keep_cap * (double)C_in * (double)C_out / 1.4e15;
+    pl.pair = pl.bnx == 256 && pl.bnw == 256 && C_out >= 256 && M_keep_cap >= 2048 && !(want_dw && want_dx && !dy_packed && memory_bound);
+    if (pl.pair) {
+        x_tiles = want_dx ? ((M_keep_cap + 2 * kBM - 1) / (2 * kBM)) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
+        w_tiles = want_dw ? ((C_out + 2 * kBM - 1) / (2 * kBM)) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
+    }
+    const int64_t workers = pl.pair ? kNumSMs / 2 : kNumSMs;
     if (want_dw) {
         // The same answer for the same shape: every shape a process has asked about is remembered (a few
         // dozen bytes per layer shape, never evicted), so a model's layers do not push each other out.
@@ -841,7 +921,7 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
             const double t_flop = 4.0 * (double)M_keep_cap * (double)C_in * (double)C_out / 1.4e15;
             const double t_mem = 2.0 * (double)M_keep_cap * (double)(2 * C_in + C_out) / 6.5e12;
             bool role_split = false;
-            if (want_dx && !dy_packed && t_mem >= 0.75 * t_flop && w_tiles > 0 && w_tiles <= kNumSMs / 4) {
+            if (!pl.pair && want_dx && !dy_packed && t_mem >= 0.75 * t_flop && w_tiles > 0 && w_tiles <= kNumSMs / 4) {
                 const double dy = 2.0 * (double)M_keep_cap * (double)C_out, xk = 2.0 * (double)M_keep_cap * (double)C_in;
                 const double w_cols = (double)((C_in + pl.bnw - 1) / pl.bnw), w_rows = (double)((C_out + kBM - 1) / kBM);
                 const double bytes_w = dy * w_cols + xk * w_rows;
@@ -865,7 +945,7 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
                 while (max_s > 1 && (x_tiles + w_tiles * max_s) * max_s > (1 << 22)) max_s /= 2;
                 double best = 0.0;
                 for (int64_t sp = 1; sp <= max_s; ++sp) {
-                    const double c = estimate_cost(x_tiles, x_kb, w_tiles, w_kb, sp, C_in * C_out);
+                    const double c = estimate_cost(x_tiles, x_kb, w_tiles, w_kb, sp, C_in * C_out, workers);
                     if (sp == 1 || c < best * 0.995) { best = c; pl.splits = (int)sp; }
                 }
             }
@@ -878,28 +958,32 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     return pl;
 }
 
-template <int BNX, int BNW, int DEPTH, bool PACKED>
+template <int BNX, int BNW, int DEPTH, bool PACKED, bool PAIR>
 cudaError_t launch_fused_variant(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
                                  const CUtensorMap& map_dw, const TcParams& prm) {
-    const cudaError_t opt = opt_in_dynamic_smem<tc_backward_kernel<BNX, BNW, DEPTH, PACKED>>((int)kSmemBytes);
+    const cudaError_t opt = opt_in_dynamic_smem<tc_backward_kernel<BNX, BNW, DEPTH, PACKED, PAIR>>((int)kSmemBytes);
     if (opt != cudaSuccess) return opt;
-    return launch_pdl(tc_backward_kernel<BNX, BNW, DEPTH, PACKED>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x,
-                      map_dw, prm);
+    if constexpr (PAIR)
+        return launch_pdl_cluster(tc_backward_kernel<BNX, BNW, DEPTH, PACKED, PAIR>, grid, dim3(kTcThreads), kSmemBytes, 2u, stream, map_w,
+                                  map_x, map_dw, prm);
+    else
+        return launch_pdl(tc_backward_kernel<BNX, BNW, DEPTH, PACKED, PAIR>, grid, dim3(kTcThreads), kSmemBytes, stream, map_w, map_x,
+                          map_dw, prm);
 }
 
-template <int BNX, int BNW, int DEPTH>
+template <int BNX, int BNW, int DEPTH, bool PAIR>
 cudaError_t launch_fused_depth(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
                                const CUtensorMap& map_dw, const TcParams& prm) {
     const bool packed = prm.dy_rows == nullptr || prm.dx_rows == nullptr;
-    return packed ? launch_fused_variant<BNX, BNW, DEPTH, true>(grid, stream, map_w, map_x, map_dw, prm)
-                  : launch_fused_variant<BNX, BNW, DEPTH, false>(grid, stream, map_w, map_x, map_dw, prm);
+    return packed ? launch_fused_variant<BNX, BNW, DEPTH, true, PAIR>(grid, stream, map_w, map_x, map_dw, prm)
+                  : launch_fused_variant<BNX, BNW, DEPTH, false, PAIR>(grid, stream, map_w, map_x, map_dw, prm);
 }
 
-template <int BNX, int BNW>
+template <int BNX, int BNW, bool PAIR = false>
 cudaError_t launch_fused(dim3 grid, cudaStream_t stream, const CUtensorMap& map_w, const CUtensorMap& map_x,
                          const CUtensorMap& map_dw, const TcParams& prm, bool deep_side_queue) {
-    return deep_side_queue ? launch_fused_depth<BNX, BNW, 16>(grid, stream, map_w, map_x, map_dw, prm)
-                           : launch_fused_depth<BNX, BNW, 8>(grid, stream, map_w, map_x, map_dw, prm);
+    return deep_side_queue ? launch_fused_depth<BNX, BNW, 16, PAIR>(grid, stream, map_w, map_x, map_dw, prm)
+                           : launch_fused_depth<BNX, BNW, 8, PAIR>(grid, stream, map_w, map_x, map_dw, prm);
 }
 
 }  // namespace
@@ -942,8 +1026,9 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     // a product that is not requested still gets a valid map (of the other matrix): it is never used
     const void* w_base = want_dx ? W : X_keep;
     const void* x_base = want_dw ? X_keep : W;
-    if (!make_map(&map_w, w_base, want_dx ? C_in : M_keep_cap, want_dx ? C_out : C_in, want_dx ? (uint32_t)pl.bnx : 64u) ||
-        !make_map(&map_x, x_base, want_dw ? M_keep_cap : C_in, want_dw ? C_in : C_out, want_dw ? 64u : (uint32_t)pl.bnx))
+    const uint32_t w_box = pl.pair ? (uint32_t)pl.bnx / 2u : (uint32_t)pl.bnx;   // a block of a pair loads half of the tile's rows of W
+    if (!make_map(&map_w, w_base, want_dx ? C_in : M_keep_cap, want_dx ? C_out : C_in, want_dx ? w_box : 64u) ||
+        !make_map(&map_x, x_base, want_dw ? M_keep_cap : C_in, want_dw ? C_in : C_out, want_dw ? 64u : w_box))
         return SBP_ERR_CUDA;
     TcParams prm;
     prm.dY = static_cast<const __nv_bfloat16*>(dY);
@@ -975,6 +1060,10 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
     prm.dw_ctas = pl.dw_ctas;
     int64_t ctas = pl.tiles < kNumSMs ? pl.tiles : kNumSMs;
     if (ctas < 1) ctas = 1;
+    if (pl.pair) {                                                   // pl.tiles counts tiles of pairs
+        const int64_t pairs = pl.tiles < kNumSMs / 2 ? (pl.tiles < 1 ? 1 : pl.tiles) : kNumSMs / 2;
+        ctas = 2 * pairs;
+    }
     const dim3 grid((unsigned)ctas);
     // Bias sums on the side: 16-byte loads per side-warp thread against the time the main loop leaves them
     // (about 1.3 us per batch of loads in flight, 0.45 us per k-block).  The shallow queue is enough when it
@@ -990,7 +1079,8 @@ sbp_status launch_tc_backward(const void* X_keep, const void* dY, const void* W,
         deep_side = loads / 8.0 * 1.3 > 0.6 * loop_us;
     }
     cudaError_t e;
-    if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
+    if (pl.pair) e = launch_fused<256, 256, true>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
+    else if (pl.bnx == 256 && pl.bnw == 256) e = launch_fused<256, 256>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
     else if (pl.bnx == 128 && pl.bnw == 256) e = launch_fused<128, 256>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
     else if (pl.bnx == 256 && pl.bnw == 128) e = launch_fused<256, 128>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
     else e = launch_fused<128, 128>(grid, stream, map_w, map_x, map_dw, prm, deep_side);
