@@ -47,6 +47,7 @@ def _packed(dY, keep, cap, dtype):
     ("bf16", 5, 14, 14, 256, 384, 0.5, 0),       # tensor-core kernel, several tiles, ragged last row tile
     ("bf16", 3, 14, 14, 384, 136, 0.25, 37),     # capacity larger than the device-side count
     ("bf16", 9, 7, 7, 128, 512, 0.75, 5),
+    ("bf16", 100, 14, 14, 512, 776, 0.5, 29),    # enough kept rows for pairs of blocks; 7 column tiles of dY: a dead half
 ])
 def test_packed_forms_match_the_scattered_result(dtype, B, H, W, C_in, C_out, r, extra):
     M = B * H * W

@@ -8,7 +8,8 @@ drown in the norm of a 768 x 3072 matrix:
       a few 1e-6 rms per thousand accumulator updates)
   dX (one rounding to bf16):               |got - want| <= 2^-8 |want| + 1e-3 * rms(want)
 The shapes are chosen so that every block of the persistent kernels runs several tiles (five and more on
-the ConvNeXt and detection maps), with ragged last tiles and ragged per-sample counts among them.
+the ConvNeXt and detection maps), with ragged last tiles and ragged per-sample counts among them; the last two run
+the form that pairs blocks on the two-SM tensor-core instructions.
 """
 import numpy as np
 import pytest
@@ -31,6 +32,9 @@ CASES = [
     ("convnext_s4_pw2_grid_ragged", 64, 7, 7, 4096, 1024, 0.5, 1),
     ("detection_s1_pw1", 2, 200, 334, 128, 512, 0.5, 0),
     ("detection_s1_pw2", 2, 200, 334, 512, 128, 0.5, 0),
+    # from 8192 kept rows on wide layers run on pairs of SMs (256-row tiles, half of the dense operand per block)
+    ("vit_b16_fc1_b128_pairs", 128, 14, 14, 768, 3072, 0.5, 0),
+    ("pairs_odd_row_tiles_ragged_columns", 100, 14, 14, 768, 1160, 0.5, 0),     # 77 row tiles: the last pair has a dead half
 ]
 
 
