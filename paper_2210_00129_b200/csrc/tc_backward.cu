@@ -15,7 +15,7 @@
 // stages behind full/empty mbarriers) never drains between tiles, and the fp32 accumulator in
 // tensor memory is double-buffered, so the epilogue of one tile overlaps the MMAs of the next.
 // Warp roles: warps 0-3 epilogue (TMEM lane quadrant = warp id), warp 4 TMA producer of the dense
-// operand, warp 5 MMA issuer and TMEM owner, warps 6-7 gather producers, which copy the indexed
+// operand, warp 5 MMA issuer and TMEM owner, warps 6-9 gather producers, which copy the indexed
 // rows of dY with coalesced 16-byte cp.async into the swizzled layout the MMA reads; each thread's
 // copies signal the stage's barrier when they land (cp.async.mbarrier.arrive).  TMA tile::gather4
 // was measured at ~45 ns of issue time per instruction per SM whatever it fetches - far too slow
@@ -36,7 +36,8 @@ namespace sbp {
 namespace {
 
 constexpr int kGatherWarp0 = 6;          // first gather warp
-constexpr int kGatherWarps = 2;          // every gather thread adds an arrival per stage: keep them few
+constexpr int kGatherWarps = 4;          // four: the copy instructions of a stage are issue-bound in two warps (dW tiles: 800 of
+                                         // the 880 clocks of a k-block), and 448 threads still leave 128 registers each
 constexpr int kGatherThreads = 32 * kGatherWarps;
 constexpr int kBiasWarp0 = kGatherWarp0 + kGatherWarps;   // four bias warps ride along after the gather warps
 constexpr int kBiasThreads = 128;
