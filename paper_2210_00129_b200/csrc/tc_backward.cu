@@ -890,12 +890,18 @@ Plan make_plan(int64_t M_keep_cap, int64_t C_in, int64_t C_out, bool want_dw, bo
     pl.splits = 1;
     pl.dw_ctas = 0;
     // Wide layers with enough work for every pair run as pairs of blocks unless the role split below takes them (the
-    // memory-bound layers gain nothing from the faster tensor-core form).  Below some 8000 kept rows the list of the
-    // twice as large tiles is too short to balance over 74 pairs (ViT-B/16 at 6272 kept rows: 7-10 % slower, at 12544
-    // and more 5-9 % faster than single blocks).
+    // memory-bound layers gain nothing from the faster tensor-core form).  From some 4000 kept rows on the pairs win on
+    // every wide shape of the paper's models (ViT-B/16 at 6272 kept rows: backward 63 -> 55 us).  A call for dX alone has
+    // no dW pieces to even out its tile list, so there the pairs must fill their waves about as well as single blocks
+    // would (6272 kept rows x 768 columns: 75 tiles on 74 pairs, 43 us against 30 us).
     const bool memory_bound = 2.0 * (double)M_keep_cap * (double)(2 * C_in + C_out) / 6.5e12 >=
                               0.75 * 4.0 * (double)M_keep_cap * (double)C_in * (double)C_out / 1.4e15;
-    pl.pair = pl.bnx == 256 && pl.bnw == 256 && C_out >= 256 && M_keep_cap >= 8192 && !(want_dw && want_dx && !dy_packed && memory_bound);
+    pl.pair = pl.bnx == 256 && pl.bnw == 256 && C_out >= 256 && M_keep_cap >= 4096 && !(want_dw && want_dx && !dy_packed && memory_bound);
+    if (pl.pair && !want_dw) {
+        const int64_t pair_tiles = ((M_keep_cap + 2 * kBM - 1) / (2 * kBM)) * ((C_in + pl.bnx - 1) / pl.bnx);
+        const auto fill = [](int64_t tiles, int64_t workers) { return (double)tiles / (double)((tiles + workers - 1) / workers * workers); };
+        pl.pair = fill(pair_tiles, kNumSMs / 2) + 0.1 >= fill(x_tiles, kNumSMs);
+    }
     if (pl.pair) {
         x_tiles = want_dx ? ((M_keep_cap + 2 * kBM - 1) / (2 * kBM)) * ((C_in + pl.bnx - 1) / pl.bnx) : 0;
         w_tiles = want_dw ? ((C_out + 2 * kBM - 1) / (2 * kBM)) * ((C_in + pl.bnw - 1) / pl.bnw) : 0;
