@@ -1028,7 +1028,10 @@ def run_probes(args):
     print("| gather of random rows (every other row kept) | source | rows x bytes | blocks | copy threads | ring | us | GB/s | GB/s per SM |")
     print("|---|---|---|---|---|---|---|---|---|")
     gen = torch.Generator(device="cuda").manual_seed(3)
-    for source, M, rb, reps in (("DRAM (205 MB)", 200704, 1024, 1), ("DRAM (51 MB of 256-byte rows)", 200704, 256, 1), ("L2 (24 MB)", 24576, 1024, 8)):
+    # lists long enough (about 800 000 rows) for runs of 100 us and more: with five tiles per block the launch and the
+    # fill of the ring are half of the time
+    for source, M, rb, reps in (("DRAM (616 MB of 6 KB rows)", 100352, 6144, 16), ("DRAM / L2 (205 MB of 1 KB rows)", 200704, 1024, 8),
+                                ("DRAM / L2 (51 MB of 256-byte rows)", 200704, 256, 8), ("L2 (24 MB)", 24576, 1024, 64)):
         src = torch.ones(M * rb, dtype=torch.uint8, device="cuda")
         lists = [torch.nonzero(torch.rand(M, device="cuda", generator=gen) < 0.5).flatten().to(torch.int32) for _ in range(reps)]
         rows = torch.cat(lists).contiguous()
