@@ -42,6 +42,25 @@ constexpr int kGatherThreads = 32 * kGatherWarps;
 constexpr int kBiasWarp0 = kGatherWarp0 + kGatherWarps;   // four bias warps ride along after the gather warps
 constexpr int kBiasThreads = 128;
 constexpr int kTcThreads = 32 * kBiasWarp0 + kBiasThreads;
+// Which of the eight warps from kGatherWarp0 on gather and which work on the side.  Plain order (gather 6-9, side 10-13)
+// for the wide tiles.  For narrow layers the map is interleaved - gather 6, 7, 10, 11, side 8, 9, 12, 13: a warp's
+// scheduler is its number modulo 4, so the gather warps, which issue copies all the time, then share schedulers 2 and 3
+// with two epilogue warps only, and the TMA and MMA threads (warps 4 and 5) share theirs with side warps that fall idle
+// once the zero rows are written.  Measured on the same GPU: ConvNeXt stage-1 pw1 57.9 -> 52.9 us; the wide variants
+// gain nothing from it (ViT-B proj and ConvNeXt stage-2 pw1 lose 4-6 %), so they keep the plain order.
+static_assert(kGatherWarps == 4 && kBiasThreads == 128, "the warp maps below are written for 4 + 4 warps");
+template <bool kInterleaved> __device__ __forceinline__ bool is_gather_warp(int warp) {
+    const int w = warp - kGatherWarp0;
+    return w >= 0 && (kInterleaved ? (w & 2) == 0 : w < kGatherWarps);
+}
+template <bool kInterleaved> __device__ __forceinline__ int gather_index(int warp) {
+    const int w = warp - kGatherWarp0;
+    return kInterleaved ? (w & 1) + (w >> 2) * 2 : w;
+}
+template <bool kInterleaved> __device__ __forceinline__ int side_index(int warp) {
+    const int w = warp - kGatherWarp0;
+    return kInterleaved ? ((w - 2) & 1) + ((w - 2) >> 2) * 2 : w - kGatherWarps;
+}
 constexpr int kBM = 128;                 // accumulator rows per tile (= TMEM lanes)
 constexpr int kBK = 64;                  // reduction depth per stage: 64 bf16 = one 128-byte swizzle row
 constexpr uint32_t kUmmaK = 16;          // reduction depth of one tcgen05.mma for 16-bit operands
@@ -478,9 +497,9 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         __syncwarp();
-    } else if (warp >= kGatherWarp0 && warp < kBiasWarp0) {
+    } else if (is_gather_warp<kNarrow>(warp)) {
         // ---------------- gather producers ----------------
-        const int gw = warp - kGatherWarp0;
+        const int gw = gather_index<kNarrow>(warp);
         uint32_t it = 0;
         bool ok = true;
         for (uint32_t pass = 0; ok; ++pass) {
@@ -565,19 +584,19 @@ tc_backward_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
             }
         }
         ptx::cp_async_wait_all();
-    } else if (warp >= kBiasWarp0) {
+    } else if (warp >= kGatherWarp0) {
         // ---------------- side warps: zeros for the dropped rows of dX, then the bias sums ----------------
         if (p.dX != nullptr && M_keep > 0) {
             for (uint32_t pass = 0;; ++pass) {
                 Tile t;
                 if (!fetch_tile(pass, t)) break;
-                if (!t.is_dw) zero_dropped_rows<BNX, kPacked>(p, t, M_keep, warp - kBiasWarp0, lane);
+                if (!t.is_dw) zero_dropped_rows<BNX, kPacked>(p, t, M_keep, side_index<kNarrow>(warp), lane);
             }
         }
         // db partial of this CTA's share of the kept rows
         if (p.db_partial != nullptr && !p.db_from_mma) {
             float* red = reinterpret_cast<float*>(smem_raw + (ring - raw_addr) + kRingBytes + 256);
-            const int t = threadIdx.x - kBiasWarp0 * 32;
+            const int t = side_index<kNarrow>(warp) * 32 + lane;
             const int V = C_out >> 3;                                  // 16-byte column vectors per row
             int VT = 16;                                               // vectors covered per pass (power of two <= 128)
             while (VT < V && VT < kBiasThreads) VT <<= 1;
