@@ -44,7 +44,7 @@ METRIC = "sbp_backward_tflops_kept_rows"
 UNIT = "TFLOP/s"
 # dram__bytes_read + dram__bytes_write per launch of the dominant kernel (mean over the launches of one step), from
 # the ncu captures summarised in profiles/ (absent = never captured, or the kernel changed since)
-NCU_TRAFFIC_BYTES = {"vit_b16_block_b128": 176.0e6, "convnext_b_s1_block": 227.1e6}
+NCU_TRAFFIC_BYTES = {"vit_b16_block_b128": 176.0e6, "convnext_b_s1_block": 225.3e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
 
